@@ -1,0 +1,148 @@
+"""ctypes front end of the CPU oracle (oracle/tko.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+CPU-baseline leg of the benchmark.  The CUDA library never imports this module
+and this module never imports the CUDA library.
+
+The shared object is compiled with g++ on first use (or by build()).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tko.cpp")
+_LIB = os.path.join(_HERE, "libtko.so")
+_lock = threading.Lock()
+_lib: Optional[ctypes.CDLL] = None
+
+MASK, TOPK, TOPKMAG = 0, 1, 2
+FLAG_RESUM = 1          # solve every pooling sub-problem member by member
+FLAG_SINGLE_THREAD = 2  # no OpenMP over rows
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle/tko.cpp into oracle/libtko.so (no-op when up to date)."""
+    with _lock:
+        if (not force and os.path.exists(_LIB)
+                and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+            return _LIB
+        tmp = _LIB + f".tmp{os.getpid()}"
+        cmd = ["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-fopenmp",
+               "-ffp-contract=off", "-o", tmp, _SRC]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+        return _LIB
+
+
+def _load() -> ctypes.CDLL:
+    global _lib
+    if _lib is not None:
+        return _lib
+    build()
+    lib = ctypes.CDLL(_LIB)
+    f32p = ctypes.POINTER(ctypes.c_float)
+    f64p = ctypes.POINTER(ctypes.c_double)
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    i64 = ctypes.c_int64
+    lib.tko_num_threads.restype = ctypes.c_int
+    lib.tko_argsort.argtypes = [f32p, i64, i64, ctypes.c_int, i32p, f64p]
+    lib.tko_fwd.argtypes = [f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double, ctypes.c_int,
+                            ctypes.c_int, f64p, i32p, f64p, i32p, i32p]
+    lib.tko_vjp.argtypes = [f32p, f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double,
+                            ctypes.c_int, ctypes.c_int, f64p]
+    lib.tko_dykstra.argtypes = [f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double,
+                                ctypes.c_int, ctypes.c_int, ctypes.c_int, f64p, f64p]
+    for fn in (lib.tko_argsort, lib.tko_fwd, lib.tko_vjp, lib.tko_dykstra):
+        fn.restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def _f32(x) -> np.ndarray:
+    a = np.ascontiguousarray(np.asarray(x, dtype=np.float32))
+    if a.ndim == 1:
+        a = a[None, :]
+    if a.ndim != 2:
+        raise ValueError("theta must be (rows, n) or (n,)")
+    return a
+
+
+def _ptr(a: Optional[np.ndarray], ty):
+    if a is None:
+        return ctypes.cast(None, ctypes.POINTER(ty))
+    return a.ctypes.data_as(ctypes.POINTER(ty))
+
+
+def num_threads() -> int:
+    return int(_load().tko_num_threads())
+
+
+def argsort(theta, mode: int = MASK) -> Tuple[np.ndarray, np.ndarray]:
+    """(perm int32, sorted keys float64), both (rows, n)."""
+    x = _f32(theta)
+    rows, n = x.shape
+    perm = np.empty((rows, n), np.int32)
+    s = np.empty((rows, n), np.float64)
+    rc = _load().tko_argsort(_ptr(x, ctypes.c_float), rows, n, mode, _ptr(perm, ctypes.c_int32),
+                             _ptr(s, ctypes.c_double))
+    if rc:
+        raise ValueError("tko_argsort: invalid argument")
+    return perm, s
+
+
+def fwd(theta, k: int, p: float, lam: float, mode: int = MASK, flags: int = 0,
+        details: bool = False):
+    """Operator output (rows, n) float64.  details=True also returns a dict with
+    perm, v (isotonic solution, sorted coordinates), block_lo, block_hi."""
+    x = _f32(theta)
+    rows, n = x.shape
+    out = np.empty((rows, n), np.float64)
+    perm = v = blo = bhi = None
+    if details:
+        perm = np.empty((rows, n), np.int32)
+        v = np.empty((rows, n), np.float64)
+        blo = np.empty((rows, n), np.int32)
+        bhi = np.empty((rows, n), np.int32)
+    rc = _load().tko_fwd(_ptr(x, ctypes.c_float), rows, n, k, p, lam, mode, flags,
+                         _ptr(out, ctypes.c_double), _ptr(perm, ctypes.c_int32),
+                         _ptr(v, ctypes.c_double), _ptr(blo, ctypes.c_int32),
+                         _ptr(bhi, ctypes.c_int32))
+    if rc:
+        raise ValueError("tko_fwd: invalid argument")
+    if details:
+        return out, {"perm": perm, "v": v, "block_lo": blo, "block_hi": bhi}
+    return out
+
+
+def vjp(theta, gout, k: int, p: float, lam: float, mode: int = MASK, flags: int = 0) -> np.ndarray:
+    x = _f32(theta)
+    g = _f32(gout)
+    if g.shape != x.shape:
+        raise ValueError("cotangent shape differs from theta")
+    rows, n = x.shape
+    grad = np.empty((rows, n), np.float64)
+    rc = _load().tko_vjp(_ptr(x, ctypes.c_float), _ptr(g, ctypes.c_float), rows, n, k, p, lam,
+                         mode, flags, _ptr(grad, ctypes.c_double))
+    if rc:
+        raise ValueError("tko_vjp: invalid argument")
+    return grad
+
+
+def dykstra(theta, k: int, p: float, lam: float, mode: int = MASK, sweeps: int = 100,
+            flags: int = 0, return_v: bool = False):
+    x = _f32(theta)
+    rows, n = x.shape
+    out = np.empty((rows, n), np.float64)
+    v = np.empty((rows, n), np.float64) if return_v else None
+    rc = _load().tko_dykstra(_ptr(x, ctypes.c_float), rows, n, k, p, lam, mode, sweeps, flags,
+                             _ptr(out, ctypes.c_double), _ptr(v, ctypes.c_double))
+    if rc:
+        raise ValueError("tko_dykstra: invalid argument")
+    return (out, v) if return_v else out

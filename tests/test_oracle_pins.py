@@ -1,0 +1,551 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something
+that is not the oracle -- a closed form, a textbook special case, brute force
+over the permutahedron's vertices, an optimality condition of the defining
+problem, a limit the paper states, or finite differences.
+
+None of these tests needs a GPU.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+from scipy.optimize import minimize
+
+from oracle import tko
+
+P43 = 4.0 / 3.0
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --------------------------------------------------------------------------
+# independent helpers (none of them sorts-then-pools)
+# --------------------------------------------------------------------------
+def q_of(p):
+    return p / (p - 1.0)
+
+
+def rho_np(t, p, lam):
+    q = q_of(p)
+    return np.sign(t) * (np.abs(t) / lam) ** (q - 1.0)
+
+
+def mask_by_threshold(x, k, p, lam):
+    """KKT form of max_{y in [0,1]^n, sum y = k} <y,x> - (lam/p) sum y^p
+    (Sec. 3, P(1_k) is the capped simplex scaled by k): stationarity gives
+    y_i = clip(((x_i - tau)_+/lam)^(q-1), 0, 1) and tau is fixed by sum y = k.
+    For p = 2 this is the Euclidean projection of x/lam onto that polytope."""
+    x = np.asarray(x, np.float64)
+    q = q_of(p)
+
+    def total(tau):
+        return np.clip((np.maximum(x - tau, 0.0) / lam) ** (q - 1.0), 0.0, 1.0).sum()
+
+    lo, hi = x.min() - lam - 1.0, x.max()
+    for _ in range(300):
+        mid = 0.5 * (lo + hi)
+        if total(mid) > k:
+            lo = mid
+        else:
+            hi = mid
+    tau = 0.5 * (lo + hi)
+    return np.clip((np.maximum(x - tau, 0.0) / lam) ** (q - 1.0), 0.0, 1.0)
+
+
+def vertices(n, k):
+    out = []
+    for idx in itertools.combinations(range(n), k):
+        v = np.zeros(n)
+        v[list(idx)] = 1.0
+        out.append(v)
+    return np.array(out)
+
+
+def mask_by_vertex_hull(x, k, p, lam):
+    """max over the convex hull of all permutations of 1_k of <y,x> - R(y),
+    y = V^T a, a in the simplex (Sec. 3, definition of the permutahedron)."""
+    x = np.asarray(x, np.float64)
+    V = vertices(len(x), k)
+    m = len(V)
+
+    def neg(a):
+        y = a @ V
+        return -(y @ x) + lam / p * np.sum(np.abs(y) ** p)
+
+    def grad(a):
+        y = a @ V
+        gy = -x + lam * np.sign(y) * np.abs(y) ** (p - 1.0)
+        return V @ gy
+
+    best = None
+    for start in range(3):
+        rng = np.random.default_rng(start)
+        a0 = rng.dirichlet(np.ones(m))
+        res = minimize(neg, a0, jac=grad, method="SLSQP", bounds=[(0, 1)] * m,
+                       constraints=[{"type": "eq", "fun": lambda a: a.sum() - 1.0,
+                                     "jac": lambda a: np.ones(m)}],
+                       options={"ftol": 1e-15, "maxiter": 500})
+        if best is None or res.fun < best.fun:
+            best = res
+    return best.x @ V
+
+
+def primal_objective(x, u, k, p, lam, mag):
+    """R*(x - u) + f_phi(u, 1_k) of Prop. 2: sum of the k largest phi(u_i)."""
+    q = q_of(p)
+    rstar = np.sum(np.abs(x - u) ** q) / (q * lam ** (q - 1.0))
+    phi = 0.5 * u * u if mag else u
+    return rstar + np.sort(phi)[::-1][:k].sum()
+
+
+def mag_by_epigraph(x, k, p, lam):
+    """Prop. 2 for phi = x^2/2 solved with no sorting: min_u max_S of
+    R*(x-u) + 1/2 sum_{i in S} u_i^2 over all k-subsets S, as an epigraph
+    programme; then y = grad R*(x - u)."""
+    x = np.asarray(x, np.float64)
+    n = len(x)
+    q = q_of(p)
+    subsets = [list(s) for s in itertools.combinations(range(n), k)]
+
+    def rstar(u):
+        return np.sum(np.abs(x - u) ** q) / (q * lam ** (q - 1.0))
+
+    def drstar(u):
+        return -np.sign(x - u) * np.abs(x - u) ** (q - 1.0) / lam ** (q - 1.0)
+
+    cons = []
+    for S in subsets:
+        def fun(z, S=S):
+            u, t = z[:n], z[n]
+            return t - rstar(u) - 0.5 * np.sum(u[S] ** 2)
+
+        def jac(z, S=S):
+            u = z[:n]
+            g = -drstar(u)
+            g[S] -= u[S]
+            return np.concatenate([g, [1.0]])
+        cons.append({"type": "ineq", "fun": fun, "jac": jac})
+    u0 = x / (1.0 + lam)
+    z0 = np.concatenate([u0, [primal_objective(x, u0, k, p, lam, True) + 1.0]])
+    res = minimize(lambda z: z[n], z0, jac=lambda z: np.concatenate([np.zeros(n), [1.0]]),
+                   method="SLSQP", constraints=cons, options={"ftol": 1e-16, "maxiter": 1000})
+    u = res.x[:n]
+    return rho_np(x - u, p, lam), u
+
+
+def random_rows(rows, n, seed, scale=1.0):
+    return (np.random.default_rng(seed).standard_normal((rows, n)) * scale).astype(np.float32)
+
+
+# --------------------------------------------------------------------------
+# hard operators and the sort
+# --------------------------------------------------------------------------
+def test_hard_operator_example_from_paper():
+    spec = {}
+    with open(os.path.join(GOLDEN, "hard_operators_example.txt")) as fh:
+        for line in fh:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, *vals = line.split()
+            spec[key] = [int(v) for v in vals]
+    x = np.array([1.0, -3.0, 2.0], np.float32)   # x3 >= x1 >= x2 and |x2| >= |x3| >= |x1|
+    k = spec["k"][0]
+    perm, s = tko.argsort(x, tko.MASK)
+    assert (perm[0] + 1).tolist() == spec["argsort"]
+    assert s[0].tolist() == [2.0, 1.0, -3.0]
+    rank = np.empty(3, int)
+    rank[perm[0]] = np.arange(1, 4)
+    assert rank.tolist() == spec["rank"]
+    tiny = 1e-9   # lambda -> 0: the relaxed operators are the hard ones
+    assert np.allclose(tko.fwd(x, k, 2.0, tiny, tko.MASK)[0], spec["topkmask"], atol=1e-12)
+    assert np.allclose(tko.fwd(x, k, 2.0, tiny, tko.TOPK)[0], x * np.array(spec["topk_keep"]),
+                       atol=1e-8)
+    assert np.allclose(tko.fwd(x, k, 2.0, tiny, tko.TOPKMAG)[0], x * np.array(spec["topkmag_keep"]),
+                       atol=1e-8)
+
+
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPKMAG])
+def test_argsort_against_rank_count(mode):
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((40, 37)).astype(np.float32)
+    x[:, 5] = x[:, 20]            # exact ties
+    x[:, 7] = -x[:, 9]            # |.| ties in magnitude mode
+    x[3, 2], x[3, 30] = 0.0, -0.0  # signed zeros compare equal
+    perm, s = tko.argsort(x, mode)
+    key = np.abs(x) if mode == tko.TOPKMAG else x
+    for r in range(x.shape[0]):
+        kr = key[r].astype(np.float64)
+        # position of element i = #{j: key_j > key_i} + #{j < i: key_j == key_i}
+        pos = [(np.sum(kr > kr[i]) + np.sum(kr[:i] == kr[i])) for i in range(len(kr))]
+        expect = np.empty(len(kr), np.int32)
+        expect[pos] = np.arange(len(kr))
+        assert np.array_equal(perm[r], expect)
+        assert np.array_equal(s[r], kr[expect])
+        assert np.all(np.diff(s[r]) <= 0)
+
+
+# --------------------------------------------------------------------------
+# the mask: closed form, brute force, polytope, limits, invariances
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("p", [2.0, P43, 1.5])
+@pytest.mark.parametrize("lam", [0.1, 1.0, 3.0])
+def test_mask_equals_threshold_form(p, lam):
+    for seed, (n, k) in enumerate([(5, 2), (17, 4), (64, 2), (64, 8), (200, 20), (33, 33), (9, 1)]):
+        x = random_rows(6, n, 100 + seed)
+        y = tko.fwd(x, k, p, lam, tko.MASK)
+        for r in range(x.shape[0]):
+            ref = mask_by_threshold(x[r], k, p, lam)
+            assert np.max(np.abs(y[r] - ref)) < 1e-9
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_mask_equals_projection_on_vertex_hull(p):
+    rng = np.random.default_rng(11)
+    for n, k in [(3, 1), (4, 2), (5, 2), (6, 3), (6, 2)]:
+        for lam in (0.5, 1.5):
+            x = rng.standard_normal(n).astype(np.float32)
+            ref = mask_by_vertex_hull(x, k, p, lam)
+            y = tko.fwd(x, k, p, lam, tko.MASK)[0]
+            assert np.max(np.abs(y - ref)) < 2e-5, (n, k, lam)
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_mask_lies_in_the_polytope(p):
+    for lam in (0.01, 0.3, 1.0, 10.0):
+        x = random_rows(50, 40, 7, scale=2.0)
+        for k in (1, 5, 39, 40):
+            y = tko.fwd(x, k, p, lam, tko.MASK)
+            assert y.min() >= 0.0 and y.max() <= 1.0 + 1e-12   # rounding of rho(s - (s - lam))
+            assert np.max(np.abs(y.sum(axis=1) - k)) < 1e-11
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPK, tko.TOPKMAG])
+def test_small_lambda_gives_hard_operator(p, mode):
+    x = random_rows(20, 30, 3)
+    k = 6
+    key = np.abs(x) if mode == tko.TOPKMAG else x
+    order = np.argsort(-key, axis=1, kind="stable")
+    hard_mask = np.zeros_like(x, dtype=np.float64)
+    np.put_along_axis(hard_mask, order[:, :k], 1.0, axis=1)
+    gap = np.min(np.abs(np.diff(np.sort(key.astype(np.float64), axis=1), axis=1)))
+    lam = 0.05 * gap
+    y = tko.fwd(x, k, p, lam, mode)
+    # a top singleton's output is rho(s - (s - lam)): 1 up to the rounding of s - lam
+    slack = 8 * np.finfo(np.float64).eps * np.max(np.abs(x)) / lam
+    if mode == tko.MASK:
+        assert np.array_equal(y == 0.0, hard_mask == 0.0)
+        assert np.max(np.abs(y - hard_mask)) <= slack
+    elif mode == tko.TOPK:
+        assert np.array_equal(y == 0.0, hard_mask == 0.0)
+        assert np.max(np.abs(y - hard_mask * x)) <= slack * np.max(np.abs(x))
+    else:
+        hard = hard_mask * x
+        # error bound of Sec. 5 / App. A.6: ||topkmag_R - topkmag||_inf <= lam ||x||_inf
+        assert np.max(np.abs(y - hard)) <= lam * np.max(np.abs(x)) + slack * np.max(np.abs(x))
+        if p == 2.0:   # App. A.6, remark: y = w x / (lam w + 1)
+            assert np.allclose(y, hard / (1.0 + lam), rtol=0, atol=slack * np.max(np.abs(x)))
+        assert np.array_equal(y == 0.0, hard_mask == 0.0)
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_large_lambda_mask_goes_to_k_over_n(p):
+    x = random_rows(5, 12, 4)
+    y = tko.fwd(x, 3, p, 1e7, tko.MASK)
+    assert np.max(np.abs(y - 3.0 / 12.0)) < 1e-5      # Sec. 7, limit lambda -> infinity
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_mask_invariances(p):
+    rng = np.random.default_rng(9)
+    x = random_rows(8, 21, 9)
+    k, lam = 4, 0.7
+    y = tko.fwd(x, k, p, lam, tko.MASK)
+    # permutation equivariance
+    perm = rng.permutation(21)
+    assert np.max(np.abs(tko.fwd(x[:, perm], k, p, lam, tko.MASK) - y[:, perm])) < 1e-12
+    # shift invariance (exactly representable shift)
+    assert np.max(np.abs(tko.fwd(x + np.float32(2.0), k, p, lam, tko.MASK) - y)) < 1e-6
+    # mask_lam(x) = mask_1(x / lam): use a power of two so x/lam is exact in fp32
+    y2 = tko.fwd(x * np.float32(4.0), k, p, 4.0 * lam, tko.MASK)
+    assert np.max(np.abs(y2 - y)) < 1e-12
+    # topkmag with p = 2 is positively homogeneous of degree 1
+    z = tko.fwd(x, k, 2.0, lam, tko.TOPKMAG)
+    z2 = tko.fwd(x * np.float32(8.0), k, 2.0, lam, tko.TOPKMAG)
+    assert np.max(np.abs(z2 - 8.0 * z)) < 1e-12
+
+
+# --------------------------------------------------------------------------
+# Figure 1 (k = 2, theta(s) = (3, 1, -1+s, s), lambda = 1)
+# --------------------------------------------------------------------------
+def figure1_rows(points=101):
+    """points=101: the grid s = -3 + 0.06 j; points=97: step 1/16, on which s and
+    s - 1 are exact in fp32 so that the tie v_2 = v_3 at s >= 2 is exact too."""
+    s = np.linspace(-3.0, 3.0, points)
+    x = np.stack([np.full_like(s, 3.0), np.full_like(s, 1.0), s - 1.0, s], axis=1)
+    return s, x.astype(np.float32)
+
+
+def test_figure1_p2_closed_form():
+    # With y_1 = 1 and y_3 = 0 on this range, y_2 + y_4 = 1 with y_2 = 1 - tau,
+    # y_4 = s - tau  =>  tau = s/2 and y_2 = clamp(1 - s/2, 0, 1).
+    s, x = figure1_rows()
+    y = tko.fwd(x, 2, 2.0, 1.0, tko.MASK)
+    f = y[:, 1] + y[:, 2]
+    sf = x[:, 3].astype(np.float64)
+    assert np.max(np.abs(f - np.clip(1.0 - sf / 2.0, 0.0, 1.0))) < 1e-6
+    assert np.allclose(y[:, 0], 1.0)
+    s, x = figure1_rows(97)
+    y = tko.fwd(x, 2, 2.0, 1.0, tko.MASK)
+    f = y[:, 1] + y[:, 2]
+    assert np.array_equal(f, np.clip(1.0 - s / 2.0, 0.0, 1.0))   # exact on the dyadic grid
+    assert np.all(f[s >= 2.0] == 0.0)             # sparse: exactly zero
+
+
+def test_figure1_p43_closed_form():
+    # p = 4/3: y_2 = a^3, y_4 = (a + s - 1)^3 with a = 1 - tau and a^3 + (a+s-1)^3 = 1.
+    for points in (101, 97):
+        check_figure1_p43(points)
+
+
+def check_figure1_p43(points):
+    s, x = figure1_rows(points)
+    y = tko.fwd(x, 2, P43, 1.0, tko.MASK)
+    f = y[:, 1] + y[:, 2]
+    sf = x[:, 3].astype(np.float64)
+    for fi, si in zip(f, sf):
+        if si <= 0.0:
+            assert abs(fi - 1.0) < 1e-12
+        elif si >= 2.0:
+            # on the 101-point grid fl(s - 1) and fl(s) - 1 differ in the last bit
+            assert fi == 0.0 if points == 97 else abs(fi) < 1e-12
+        else:
+            lo, hi = 0.0, 1.0
+            for _ in range(200):
+                a = 0.5 * (lo + hi)
+                if a ** 3 + max(a + si - 1.0, 0.0) ** 3 > 1.0:
+                    hi = a
+                else:
+                    lo = a
+            assert abs(fi - (0.5 * (lo + hi)) ** 3) < 1e-9
+    if points == 97:
+        mid = np.argmin(np.abs(sf - 1.0))
+        assert sf[mid] == 1.0 and abs(f[mid] - 0.5) < 1e-12     # 2 a^3 = 1 at s = 1
+        # f(1 + d) + f(1 - d) = 1: the equation for a is symmetric under s -> 2 - s, a <-> a + s - 1
+        for j, sj in enumerate(sf):
+            if -1.0 <= sj <= 3.0:
+                jj = int(np.argmin(np.abs(sf - (2.0 - sj))))
+                assert sf[jj] == 2.0 - sj and abs(f[j] + f[jj] - 1.0) < 1e-12
+
+
+def test_figure3_is_sparse_and_continuous():
+    # x = (x1, x2, 1/2, 1), phi = x^2/2, k = 2, lambda = 0.3: output_1 + output_2 is
+    # exactly 0 around the origin and continuous (Figure 3 caption).
+    grid = np.linspace(-2.0, 2.0, 81)
+    for p in (2.0, P43):
+        rows = np.array([[a, b, 0.5, 1.0] for a in grid for b in grid], np.float32)
+        y = tko.fwd(rows, 2, p, 0.3, tko.TOPKMAG)
+        tot = (y[:, 0] + y[:, 1]).reshape(81, 81)
+        inner = (np.abs(grid)[:, None] < 0.25) & (np.abs(grid)[None, :] < 0.25)
+        assert np.all(tot[inner] == 0.0)
+        # continuity along a line: |d out_i / d x_j| <= rho' <= (q-1)/lam on [0,1]-valued
+        # pieces, so a step of 1e-3 moves the sum of two outputs by < 2 * 1e-3 * 3 / lam + slack;
+        # the unregularised operator jumps by about 0.5 on the same line.
+        line = np.linspace(-2.0, 2.0, 4001)
+        rows = np.array([[a, 0.7, 0.5, 1.0] for a in line], np.float32)
+        y = tko.fwd(rows, 2, p, 0.3, tko.TOPKMAG)
+        assert np.max(np.abs(np.diff(y[:, 0] + y[:, 1]))) < 0.025
+
+
+# --------------------------------------------------------------------------
+# magnitude operator: brute force and optimality of u*
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_topkmag_equals_epigraph_solution(p):
+    rng = np.random.default_rng(21)
+    for n, k in [(3, 1), (4, 2), (5, 2), (5, 3)]:
+        for lam in (0.3, 1.0):
+            x = rng.standard_normal(n).astype(np.float32)
+            ref, _ = mag_by_epigraph(x, k, p, lam)
+            y = tko.fwd(x, k, p, lam, tko.TOPKMAG)[0]
+            assert np.max(np.abs(y - ref)) < 5e-5, (n, k, lam, y, ref)
+
+
+@pytest.mark.parametrize("p", [2.0, P43, 1.5])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPKMAG])
+def test_u_star_minimises_the_primal(p, mode):
+    rng = np.random.default_rng(31)
+    mag = mode == tko.TOPKMAG
+    for n, k, lam in [(6, 2, 0.5), (12, 3, 1.0), (30, 7, 0.2), (30, 29, 2.0)]:
+        x = rng.standard_normal((3, n)).astype(np.float32)
+        _, det = tko.fwd(x, k, p, lam, mode, details=True)
+        for r in range(3):
+            v = det["v"][r]
+            u = np.empty(n)
+            u[det["perm"][r]] = v
+            xr = x[r].astype(np.float64)
+            if mag:
+                u *= np.where(np.signbit(xr) & (xr != 0), -1.0, 1.0)
+            f0 = primal_objective(xr, u, k, p, lam, mag)
+            for scale in (1e-1, 1e-2, 1e-3, 1e-4, 1e-5):
+                for _ in range(200):
+                    d = rng.standard_normal(n) * scale
+                    if rng.random() < 0.5:       # sparse directions probe single coordinates
+                        d *= rng.random(n) < 0.2
+                    assert primal_objective(xr, u + d, k, p, lam, mag) >= f0 - 1e-13
+
+
+# --------------------------------------------------------------------------
+# internals of the isotonic solution
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("p", [2.0, P43, 1.5])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPKMAG])
+def test_isotonic_solution_structure(p, mode):
+    mag = mode == tko.TOPKMAG
+    for n, k, lam, seed in [(50, 5, 1.0, 1), (50, 25, 0.3, 2), (128, 16, 1.0, 3), (10, 10, 1.0, 4)]:
+        x = random_rows(10, n, seed)
+        if seed == 2:
+            x[:, 3] = x[:, 11]
+        _, det = tko.fwd(x, k, p, lam, mode, details=True)
+        perm, s = tko.argsort(x, mode)
+        for r in range(x.shape[0]):
+            v, lo, hi = det["v"][r], det["block_lo"][r], det["block_hi"][r]
+            assert np.all(np.diff(v) <= 1e-15)                      # v in the monotone cone
+            if mag:
+                assert v.min() >= 0.0
+            pooled = 0
+            i = 0
+            while i < n:
+                a, b = lo[i], hi[i]
+                assert a == i and b > a
+                g = v[a]
+                assert np.all(v[a:b] == g)
+                w = (np.arange(a, b) < k).astype(float)
+                resid = np.sum(-rho_np(s[r][a:b] - g, p, lam) + w * (g if mag else 1.0))
+                assert abs(resid) < 1e-9 * max(1.0, b - a)           # block stationarity
+                pooled += (b - a) > 1
+                if b - a > 1:
+                    assert a < k < b                                  # the pooled block straddles rank k
+                i = b
+            assert pooled <= 1                                        # w = 1_k: at most one pooled block
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPK, tko.TOPKMAG])
+def test_member_resolve_matches_closed_form_solves(p, mode):
+    x = random_rows(12, 300, 8)
+    g = random_rows(12, 300, 9)
+    a = tko.fwd(x, 30, p, 1.0, mode)
+    b = tko.fwd(x, 30, p, 1.0, mode, flags=tko.FLAG_RESUM)
+    assert np.max(np.abs(a - b)) < 1e-11
+    ga = tko.vjp(x, g, 30, p, 1.0, mode)
+    gb = tko.vjp(x, g, 30, p, 1.0, mode, flags=tko.FLAG_RESUM)
+    assert np.max(np.abs(ga - gb)) < 1e-8
+
+
+# --------------------------------------------------------------------------
+# alternating projections
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("p", [2.0, P43])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPKMAG])
+def test_dykstra_converges_to_pav(p, mode):
+    x = random_rows(8, 24, 13)
+    for k, lam in [(3, 1.0), (12, 0.4)]:
+        exact, det = tko.fwd(x, k, p, lam, mode, details=True)
+        out, v = tko.dykstra(x, k, p, lam, mode, sweeps=6000, return_v=True)
+        assert np.max(np.abs(v - det["v"])) < 1e-9
+        assert np.max(np.abs(out - exact)) < 1e-8
+
+
+def test_dykstra_single_element_is_s_minus_lambda_w():
+    # n = 1: no constraint, so the iteration must return the unconstrained
+    # minimiser s - lambda w (phi = x) after any number of sweeps.
+    x = np.array([[0.75]], np.float32)
+    for sweeps in (0, 1, 5):
+        _, v = tko.dykstra(x, 1, 2.0, 0.5, tko.MASK, sweeps=sweeps, return_v=True)
+        assert v[0, 0] == 0.75 - 0.5
+
+
+def test_dykstra_hundred_sweeps_small_block():
+    # Sec. 5: 100 iterations reproduce PAV (small pooled blocks)
+    x = random_rows(64, 16, 17)
+    exact = tko.fwd(x, 2, 2.0, 0.3, tko.MASK)
+    out = tko.dykstra(x, 2, 2.0, 0.3, tko.MASK, sweeps=100)
+    assert np.max(np.abs(out - exact)) < 1e-6
+
+
+# --------------------------------------------------------------------------
+# VJP
+# --------------------------------------------------------------------------
+def jacobian_fd(x, k, p, lam, mode, h=1e-3):
+    """central differences in fp32-representable steps (inputs are fp32)."""
+    n = len(x)
+    J = np.empty((n, n))
+    for j in range(n):
+        xp = x.copy(); xm = x.copy()
+        xp[j] = np.float32(x[j] + h); xm[j] = np.float32(x[j] - h)
+        step = float(xp[j]) - float(xm[j])
+        J[:, j] = (tko.fwd(xp, k, p, lam, mode)[0] - tko.fwd(xm, k, p, lam, mode)[0]) / step
+    return J
+
+
+def jacobian_vjp(x, k, p, lam, mode):
+    n = len(x)
+    J = np.empty((n, n))
+    for i in range(n):
+        e = np.zeros(n, np.float32); e[i] = 1.0
+        J[i, :] = tko.vjp(x, e, k, p, lam, mode)[0]
+    return J
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPK, tko.TOPKMAG])
+def test_vjp_matches_finite_differences(p, mode):
+    rng = np.random.default_rng(41)
+    checked = 0
+    for trial in range(12):
+        n, k, lam = 9, 3, 0.8
+        x = (rng.standard_normal(n) * 1.0).astype(np.float32)
+        # keep away from kinks: block membership must not change within +-h
+        _, d0 = tko.fwd(x, k, p, lam, mode, details=True)
+        stable = True
+        for j in range(n):
+            for sgn in (-1, 1):
+                xx = x.copy(); xx[j] = np.float32(xx[j] + sgn * 2e-3)
+                _, d1 = tko.fwd(xx, k, p, lam, mode, details=True)
+                if not (np.array_equal(d0["perm"], d1["perm"]) and
+                        np.array_equal(d0["block_lo"], d1["block_lo"]) and
+                        np.array_equal(d0["block_hi"], d1["block_hi"])):
+                    stable = False
+        if not stable:
+            continue
+        J = jacobian_vjp(x, k, p, lam, mode)
+        Jfd = jacobian_fd(x, k, p, lam, mode)
+        tol = 1e-8 if p == 2.0 else 2e-5      # p = 2 is piecewise linear: differences are exact
+        assert np.max(np.abs(J - Jfd)) < tol * max(1.0, np.max(np.abs(J)))
+        checked += 1
+    assert checked >= 4
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_mask_jacobian_is_symmetric_with_zero_row_sums(p):
+    x = random_rows(1, 14, 51)[0]
+    J = jacobian_vjp(x, 4, p, 1.0, tko.MASK)
+    assert np.max(np.abs(J - J.T)) < 1e-12
+    assert np.max(np.abs(J.sum(axis=0))) < 1e-12 and np.max(np.abs(J.sum(axis=1))) < 1e-12
+    assert np.max(np.abs(J)) > 0.01
+
+
+def test_topkmag_p2_top_singletons_have_slope_one_over_one_plus_lambda():
+    x = np.array([[5.0, -4.0, 0.1, 0.05, -0.02]], np.float32)
+    lam = 0.25
+    g = np.ones((1, 5), np.float32)
+    grad = tko.vjp(x, g, 2, 2.0, lam, tko.TOPKMAG)[0]
+    assert np.allclose(grad[:2], 1.0 / (1.0 + lam)) and np.all(grad[2:] == 0.0)
+
+
+def test_invalid_arguments_are_rejected():
+    x = np.zeros((1, 4), np.float32)
+    for k, p, lam in [(0, 2.0, 1.0), (5, 2.0, 1.0), (2, 1.0, 1.0), (2, 2.0, 0.0)]:
+        with pytest.raises(ValueError):
+            tko.fwd(x, k, p, lam, tko.MASK)
