@@ -1,0 +1,129 @@
+/* tk.h -- C ABI of the sm_100a library for p-norm-regularised (smoothed) top-k
+ * operators: the batched forward pass and vector-Jacobian product of
+ *   topkmask_R, topk_R, topkmag_R   with   R(y) = (lambda/p) * sum_i |y_i|^p,
+ * p = 2 or p = 4/3, w = 1_k (k ones followed by zeros).
+ *
+ * Per row the library sorts theta (or |theta|), solves the isotonic problem the
+ * operator reduces to, maps the solution back through grad R*, and un-permutes.
+ * Paper references are to "Fast, Differentiable and Sparse Top-k: a Convex
+ * Analysis Perspective": Sec. 3 = Background, Sec. 4 = Proposed generalized
+ * framework, Sec. 5 = Algorithms, App. A = proofs.
+ *
+ * Conventions shared by every entry point
+ *  - All data pointers are DEVICE pointers owned by the caller; row r of a
+ *    [rows, n] tensor occupies elements [r*n, r*n + n) (row-major, contiguous).
+ *    fp32 values, int32 permutations.
+ *  - The library never allocates, frees or synchronises; all work is enqueued
+ *    on `stream`.  Scratch memory, when a configuration needs it, is passed in
+ *    tk_opts.workspace (size from tk_workspace_bytes).
+ *  - Arguments are checked on the host before any launch.  The return value is
+ *    a tk_status; nothing throws, exits or traps.  rows == 0 returns TK_OK
+ *    without a launch.
+ *  - 1 <= k <= n, lambda > 0, p > 1 with q = p/(p-1) within 1e-6 of 2 or 4
+ *    (other p: TK_ERR_UNSUPPORTED).  Outputs must not alias inputs.
+ *  - Inputs must be finite.  A NaN/Inf sets TK_FLAG_NONFINITE in *status_out
+ *    (when given); that row's output is unspecified, the call still completes.
+ */
+#ifndef TK_H_
+#define TK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque stream handle: a cudaStream_t passed as a pointer (NULL = default stream). */
+typedef void *tk_stream;
+
+typedef enum {
+  TK_MASK = 0,    /* phi(x) = x:      relaxed top-k mask (Sec. 4, "a relaxed top-k mask")   */
+  TK_TOPK = 1,    /* theta * mask_R(theta): relaxed top-k values of a signed input; the hard
+                     operator of Sec. 3 with the relaxed mask substituted                   */
+  TK_TOPKMAG = 2  /* phi(x) = x^2/2:  relaxed top-k in magnitude (Sec. 4, topkmag_R)        */
+} tk_mode;
+
+typedef enum {
+  TK_SOLVER_AUTO = 0,
+  TK_SOLVER_PAV = 1,      /* exact pooling of adjacent violators (Sec. 5, App. B.2)          */
+  TK_SOLVER_DYKSTRA = 2   /* alternating projections on odd/even pairs (Algorithm 1; for
+                             p != 2 the dual block coordinate ascent of App. A.8)            */
+} tk_solver;
+
+typedef enum {
+  TK_OK = 0,
+  TK_ERR_INVALID_ARG = 1,   /* null pointer, k out of range, lambda <= 0, p <= 1, ...        */
+  TK_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for                    */
+  TK_ERR_WORKSPACE = 3,     /* workspace missing or smaller than tk_workspace_bytes          */
+  TK_ERR_CUDA = 4,          /* a CUDA runtime call (launch, attribute) failed                */
+  TK_ERR_NOT_CONVERGED = 5
+} tk_status;
+
+/* bits OR-ed into *tk_opts.status_out by the kernels */
+#define TK_FLAG_NONFINITE 1      /* some input was NaN or Inf                                */
+#define TK_FLAG_NOT_CONVERGED 2  /* an iterative solve stopped at its iteration cap          */
+
+/* What the forward pass found for one row, enough to run the VJP without
+ * sorting again.  With s the keys in descending order, ranks [a, b) form the
+ * single pooled block of the isotonic solution (w = 1_k admits at most one),
+ * whose common value is gamma = pivot + offset; pivot is the k-th largest key
+ * (kept apart from offset so that key - gamma can be formed without
+ * cancellation).  a == b == k means no pooled block: every rank < k is a top
+ * singleton, every other rank a bottom singleton.                              */
+typedef struct {
+  float pivot;
+  float offset;
+  int32_t a;
+  int32_t b;
+} tk_rowstate;
+
+typedef struct {
+  int solver;              /* tk_solver; AUTO = PAV                                           */
+  int sweeps;              /* Dykstra sweeps; <= 0 means 100 (the count used in Sec. 5)       */
+  int32_t *perm_out;       /* [rows*n] sorted rank -> original index, or NULL                 */
+  tk_rowstate *state_out;  /* tk_fwd_ex: [rows] written.  tk_vjp: [rows] read (saved by a
+                              forward call with identical arguments), or NULL = recompute    */
+  void *workspace;         /* device scratch, 256-byte aligned, or NULL                       */
+  size_t workspace_bytes;
+  int32_t *status_out;     /* one device word, OR of TK_FLAG_*; the caller zeroes it          */
+} tk_opts;
+
+/* Scratch bytes tk_fwd_ex / tk_vjp / tk_argsort need for this shape (0 when the
+ * row is solved on chip).  solver as in tk_opts.                               */
+size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver);
+
+/* Forward pass (Prop. 2 with Prop. 5 / Prop. 6): out[r, :] = operator(theta[r, :]).
+ * theta, out: device, [rows*n] fp32.  Fails with TK_ERR_WORKSPACE for shapes that
+ * need scratch (use tk_fwd_ex).                                                 */
+tk_status tk_fwd(const float *theta, int64_t rows, int64_t n, int64_t k, double p, double lambda,
+                 int mode, float *out, tk_stream stream);
+
+/* Forward pass with options (solver choice, permutation / row state outputs,
+ * workspace, status word).  opts may be NULL (= tk_fwd).                        */
+tk_status tk_fwd_ex(const float *theta, int64_t rows, int64_t n, int64_t k, double p,
+                    double lambda, int mode, float *out, const tk_opts *opts, tk_stream stream);
+
+/* Vector-Jacobian product (Prop. 7 chained through y = grad R*(x - u)):
+ * grad_theta[r, :] = J(theta[r, :])^T grad_out[r, :].  All device, [rows*n] fp32.
+ * With opts->state_out from a forward call the rows are not sorted again.       */
+tk_status tk_vjp(const float *theta, const float *grad_out, int64_t rows, int64_t n, int64_t k,
+                 double p, double lambda, int mode, float *grad_theta, const tk_opts *opts,
+                 tk_stream stream);
+
+/* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
+ * perm_out[i] = index of the i-th largest key (theta, or |theta| for
+ * TK_TOPKMAG), equal keys in ascending index, -0 == +0.  sorted_out (may be
+ * NULL) receives the keys in that order.  opts may carry a workspace.           */
+tk_status tk_argsort(const float *theta, int64_t rows, int64_t n, int mode, int32_t *perm_out,
+                     float *sorted_out, const tk_opts *opts, tk_stream stream);
+
+const char *tk_status_string(int status);
+
+/* Library build tag, e.g. "tk 0.1 sm_100a".                                     */
+const char *tk_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TK_H_ */

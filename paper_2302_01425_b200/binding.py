@@ -1,0 +1,153 @@
+"""Thin ctypes binding of libtk.so: argument marshalling only.
+
+Every function here has the name and the arguments of its C counterpart in
+include/tk.h; tensors are torch CUDA tensors used purely as device buffers and
+work is enqueued on torch's current stream.  There is no CPU path: loading
+fails loudly when the library has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libtk.so")
+
+TK_MASK, TK_TOPK, TK_TOPKMAG = 0, 1, 2
+TK_SOLVER_AUTO, TK_SOLVER_PAV, TK_SOLVER_DYKSTRA = 0, 1, 2
+TK_OK = 0
+TK_ERR_INVALID_ARG, TK_ERR_UNSUPPORTED, TK_ERR_WORKSPACE, TK_ERR_CUDA, TK_ERR_NOT_CONVERGED = 1, 2, 3, 4, 5
+TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
+ROWSTATE_BYTES = 16
+
+EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
+           "tk_argsort")
+
+
+class TkOpts(ctypes.Structure):
+    _fields_ = [
+        ("solver", ctypes.c_int),
+        ("sweeps", ctypes.c_int),
+        ("perm_out", ctypes.c_void_p),
+        ("state_out", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
+        ("status_out", ctypes.c_void_p),
+    ]
+
+
+class TkError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libtk.so; raises if it is missing (there is no fallback)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2302_01425_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, dbl, vp, ci = ctypes.c_int64, ctypes.c_double, ctypes.c_void_p, ctypes.c_int
+    lib.tk_version.restype = ctypes.c_char_p
+    lib.tk_status_string.restype = ctypes.c_char_p
+    lib.tk_status_string.argtypes = [ci]
+    lib.tk_workspace_bytes.restype = ctypes.c_size_t
+    lib.tk_workspace_bytes.argtypes = [i64, i64, i64, dbl, ci, ci]
+    lib.tk_fwd.restype = ci
+    lib.tk_fwd.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, vp]
+    lib.tk_fwd_ex.restype = ci
+    lib.tk_fwd_ex.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_vjp.restype = ci
+    lib.tk_vjp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_argsort.restype = ci
+    lib.tk_argsort.argtypes = [vp, i64, i64, ci, vp, vp, ctypes.POINTER(TkOpts), vp]
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().tk_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return load().tk_version().decode()
+
+
+def _dev(t: Optional[torch.Tensor], dtype, what: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{what}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _opts(solver=TK_SOLVER_AUTO, sweeps=0, perm_out=None, state=None, workspace=None,
+          status_out=None) -> TkOpts:
+    o = TkOpts()
+    o.solver, o.sweeps = int(solver), int(sweeps)
+    o.perm_out = _dev(perm_out, torch.int32, "perm_out")
+    o.state_out = None if state is None else _dev(state, torch.uint8, "state")
+    o.workspace = None if workspace is None else _dev(workspace, torch.uint8, "workspace")
+    o.workspace_bytes = 0 if workspace is None else workspace.numel()
+    o.status_out = _dev(status_out, torch.int32, "status_out")
+    return o
+
+
+def new_state(rows: int, device="cuda") -> torch.Tensor:
+    """Device buffer for `rows` tk_rowstate records."""
+    return torch.empty(rows * ROWSTATE_BYTES, dtype=torch.uint8, device=device)
+
+
+def tk_workspace_bytes(rows: int, n: int, k: int, p: float, mode: int, solver: int = 0) -> int:
+    return int(load().tk_workspace_bytes(rows, n, k, p, mode, solver))
+
+
+def tk_fwd(theta: torch.Tensor, rows: int, n: int, k: int, p: float, lam: float, mode: int,
+           out: torch.Tensor) -> None:
+    rc = load().tk_fwd(_dev(theta, torch.float32, "theta"), rows, n, k, p, lam, mode,
+                       _dev(out, torch.float32, "out"), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_fwd")
+
+
+def tk_fwd_ex(theta, rows, n, k, p, lam, mode, out, *, solver=TK_SOLVER_AUTO, sweeps=0,
+              perm_out=None, state_out=None, workspace=None, status_out=None) -> None:
+    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out)
+    rc = load().tk_fwd_ex(_dev(theta, torch.float32, "theta"), rows, n, k, p, lam, mode,
+                          _dev(out, torch.float32, "out"), ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_fwd_ex")
+
+
+def tk_vjp(theta, grad_out, rows, n, k, p, lam, mode, grad_theta, *, state=None, workspace=None,
+           status_out=None) -> None:
+    o = _opts(state=state, workspace=workspace, status_out=status_out)
+    rc = load().tk_vjp(_dev(theta, torch.float32, "theta"), _dev(grad_out, torch.float32, "grad_out"),
+                       rows, n, k, p, lam, mode, _dev(grad_theta, torch.float32, "grad_theta"),
+                       ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_vjp")
+
+
+def tk_argsort(theta, rows, n, mode, perm_out, sorted_out=None, *, workspace=None,
+               status_out=None) -> None:
+    o = _opts(workspace=workspace, status_out=status_out)
+    rc = load().tk_argsort(_dev(theta, torch.float32, "theta"), rows, n, mode,
+                           _dev(perm_out, torch.int32, "perm_out"),
+                           _dev(sorted_out, torch.float32, "sorted_out"), ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_argsort")

@@ -1,0 +1,145 @@
+// tk_api.cu -- the C ABI: argument checks and dispatch.  Declarations and the
+// meaning of every argument are in include/tk.h.
+#include <math.h>
+
+#include "tk_common.cuh"
+
+namespace tk {
+// on-chip row kernels (tk_cta.cu)
+cudaError_t launch_cta(const Problem& P, cudaStream_t stream);
+int cta_padded_length(int n);
+// VJP from saved row state (tk_vjp_state.cu)
+cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
+
+constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
+}  // namespace tk
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// q = p/(p-1) must be 2 or 4 (p = 2 or p = 4/3).
+tk_status classify_p(double p, int* q4) {
+  if (!(p > 1.0) || !isfinite(p)) return TK_ERR_INVALID_ARG;
+  double q = p / (p - 1.0);
+  if (fabs(q - 2.0) <= 1e-6) { *q4 = 0; return TK_OK; }
+  if (fabs(q - 4.0) <= 1e-6) { *q4 = 1; return TK_OK; }
+  return TK_ERR_UNSUPPORTED;
+}
+
+tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, double p,
+                       double lambda, int mode, int* q4) {
+  if (rows < 0 || n < 1 || k < 1 || k > n) return TK_ERR_INVALID_ARG;
+  if (mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
+  if (!(lambda > 0.0) || !isfinite(lambda)) return TK_ERR_INVALID_ARG;
+  tk_status s = classify_p(p, q4);
+  if (s != TK_OK) return s;
+  if (rows > 0 && theta == nullptr) return TK_ERR_INVALID_ARG;
+  if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
+  return TK_OK;
+}
+
+void fill(tk::Problem& P, const float* theta, int64_t rows, int64_t n, int64_t k, int q4,
+          double lambda, int mode) {
+  P = tk::Problem{};
+  P.theta = theta;
+  P.rows = rows; P.n = (int)n; P.k = (int)k; P.q4 = q4; P.mode = mode;
+  P.lam = (float)lambda;
+  P.inv_lam = (float)(1.0 / lambda);
+  P.lam3 = (float)(lambda * lambda * lambda);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tk_version(void) { return "tk 0.1 sm_100a"; }
+
+const char* tk_status_string(int status) {
+  switch (status) {
+    case TK_OK: return "ok";
+    case TK_ERR_INVALID_ARG: return "invalid argument";
+    case TK_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TK_ERR_WORKSPACE: return "workspace missing or too small";
+    case TK_ERR_CUDA: return "CUDA runtime error";
+    case TK_ERR_NOT_CONVERGED: return "iteration cap reached";
+    default: return "unknown status";
+  }
+}
+
+size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver) {
+  (void)rows; (void)k; (void)p; (void)mode; (void)solver;
+  if (n <= tk::kMaxOnChipN) return 0;
+  return 0;
+}
+
+tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
+                    double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
+  int q4 = 0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4);
+  if (s != TK_OK) return s;
+  if (rows == 0) return TK_OK;
+  if (out == nullptr) return TK_ERR_INVALID_ARG;
+  int solver = opts ? opts->solver : TK_SOLVER_AUTO;
+  if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_DYKSTRA) return TK_ERR_INVALID_ARG;
+  if (solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
+  if (n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
+  tk::Problem P;
+  fill(P, theta, rows, n, k, q4, lambda, mode);
+  P.out = out;
+  P.what = tk::W_FWD;
+  if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
+  P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
+  cudaError_t e = tk::launch_cta(P, (cudaStream_t)stream);
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_fwd(const float* theta, int64_t rows, int64_t n, int64_t k, double p, double lambda,
+                 int mode, float* out, tk_stream stream) {
+  return tk_fwd_ex(theta, rows, n, k, p, lambda, mode, out, nullptr, stream);
+}
+
+tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_t n, int64_t k,
+                 double p, double lambda, int mode, float* grad_theta, const tk_opts* opts,
+                 tk_stream stream) {
+  int q4 = 0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4);
+  if (s != TK_OK) return s;
+  if (rows == 0) return TK_OK;
+  if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
+  tk::Problem P;
+  fill(P, theta, rows, n, k, q4, lambda, mode);
+  P.gout = grad_out;
+  P.out = grad_theta;
+  P.what = tk::W_VJP;
+  if (opts) P.status = opts->status_out;
+  P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(grad_out) && aligned16(grad_theta);
+  cudaError_t e;
+  if (opts && opts->state_out) {
+    P.state_in = opts->state_out;
+    e = tk::launch_vjp_state(P, (cudaStream_t)stream);
+  } else {
+    if (n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
+    e = tk::launch_cta(P, (cudaStream_t)stream);
+  }
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int32_t* perm_out,
+                     float* sorted_out, const tk_opts* opts, tk_stream stream) {
+  if (rows < 0 || n < 1 || mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
+  if (rows == 0) return TK_OK;
+  if (theta == nullptr || perm_out == nullptr) return TK_ERR_INVALID_ARG;
+  if (n > tk::kMaxOnChipN || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
+  tk::Problem P;
+  fill(P, theta, rows, n, 1, 0, 1.0, mode);
+  P.what = tk::W_ARGSORT;
+  P.perm_out = perm_out;
+  P.sorted_out = sorted_out;
+  if (opts) P.status = opts->status_out;
+  P.vec4 = (n % 4 == 0) && aligned16(theta);
+  cudaError_t e = tk::launch_cta(P, (cudaStream_t)stream);
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+}  // extern "C"

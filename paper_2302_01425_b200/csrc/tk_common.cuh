@@ -1,0 +1,162 @@
+// tk_common.cuh -- shared device helpers of the smoothed top-k kernels.
+//
+// Notation (Sec. 5 of the paper): s = keys in descending order, w = 1_k,
+// h_i(v) = r*(s_i - v) + w_i phi(v), r*(t) = |t|^q / (q lambda^(q-1)),
+// rho(t) = (r*)'(t) = sign(t) (|t|/lambda)^(q-1), q = p/(p-1) in {2, 4}.
+// All arithmetic near the pooled block is done relative to the pivot
+// c = k-th largest key: d_i = s_i - c, gamma = c + u.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tk.h"
+
+namespace tk {
+
+enum What { W_FWD = 0, W_VJP = 1, W_ARGSORT = 2 };
+
+struct Problem {
+  const float* theta;
+  const float* gout;        // cotangent (VJP only)
+  float* out;               // operator output (forward) or grad_theta (VJP)
+  int32_t* perm_out;
+  float* sorted_out;
+  tk_rowstate* state_out;
+  const tk_rowstate* state_in;
+  int32_t* status;
+  long long rows;
+  int n, k;
+  int N;                    // padded row length held on chip
+  int q4;                   // 1: q = 4 (p = 4/3); 0: q = 2
+  int mode;                 // tk_mode
+  int what;                 // What
+  int vec4;                 // rows may be accessed as float4
+  float lam, inv_lam, lam3; // lambda, 1/lambda, lambda^3
+  int sweeps;               // Dykstra path
+};
+
+// ---------------------------------------------------------------- keys
+// Order-preserving map float -> uint32 (larger float, larger integer).
+__device__ __forceinline__ uint32_t f2key(float x) {
+  uint32_t b = __float_as_uint(x);
+  return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float key2f(uint32_t u) {
+  uint32_t b = u ^ ((u >> 31) ? 0x80000000u : 0xFFFFFFFFu);
+  return __uint_as_float(b);
+}
+// The sort key of an input: theta or |theta|, with -0 folded onto +0.
+__device__ __forceinline__ float sort_key(float x, bool mag) {
+  float k = mag ? fabsf(x) : x;
+  return (k == 0.0f) ? 0.0f : k;
+}
+
+// ---------------------------------------------------------------- scalar math
+struct Math {
+  float lam, inv_lam, lam3;
+  bool q4, mag;
+
+  __device__ __forceinline__ float rho(float t) const {
+    float a = t * inv_lam;
+    return q4 ? a * a * a : a;
+  }
+  __device__ __forceinline__ float drho(float t) const {
+    float a = t * inv_lam;
+    return q4 ? 3.0f * a * a * inv_lam : inv_lam;
+  }
+  // z >= 0 with z^3 + lam z = s (s >= 0): z = (s - v)/lam at the minimiser v of
+  // h(v) = v^2/2 + (s - v)^4 / (4 lam^3).  Newton from the right of the root on
+  // a convex increasing function: monotone convergence.
+  __device__ __forceinline__ float cubic_z(float s) const {
+    if (!(s > 0.0f)) return 0.0f;
+    float z = fminf(cbrtf(s), s * inv_lam);
+#pragma unroll 1
+    for (int it = 0; it < 16; ++it) {
+      float f = fmaf(z * z + lam, z, -s);
+      float dz = f / fmaf(3.0f * z, z, lam);
+      z -= dz;
+      if (fabsf(dz) <= 6e-8f * z) break;
+    }
+    return z;
+  }
+  // Minimiser of h_i for a rank < k (w_i = 1) singleton with key s.
+  __device__ __forceinline__ float vtop(float s) const {
+    if (!mag) return s - lam;
+    if (!q4) return s / (1.0f + lam);
+    float z = cubic_z(s);
+    float lz = lam * z;
+    return (lz < 0.5f * s) ? s - lz : z * z * z;
+  }
+  // Key distance above gamma = tau at which a rank < k element stops being
+  // pooled: rho(width) = phi'(tau).
+  __device__ __forceinline__ float width(float tau) const {
+    if (!mag) return lam;
+    float t = fmaxf(tau, 0.0f);
+    return q4 ? lam * cbrtf(t) : lam * t;
+  }
+  // d/ds of the output of a top singleton (phi even): rho' / (rho' + 1).
+  __device__ __forceinline__ float top_slope(float s) const {
+    if (!mag) return 0.0f;
+    if (!q4) return 1.0f / (1.0f + lam);
+    float z = cubic_z(s);              // z = (s - v)/lam, rho' = 3 z^2 / lam
+    float r = 3.0f * z * z * inv_lam;
+    return r / (r + 1.0f);
+  }
+};
+
+__device__ __forceinline__ Math make_math(const Problem& P) {
+  Math m;
+  m.lam = P.lam; m.inv_lam = P.inv_lam; m.lam3 = P.lam3;
+  m.q4 = P.q4 != 0; m.mag = P.mode == TK_TOPKMAG;
+  return m;
+}
+
+// Root u of the pooled block's stationarity equation, from the block's power
+// sums D_m = sum_B d_i^m (cnt members, m of them with w = 1), pivot c:
+//   q = 2, phi = x   : sum (d_i - u)/lam = m            -> closed form
+//   q = 2, phi even  : sum (d_i - u)/lam = m (c + u)    -> closed form (Sec. 5 example)
+//   q = 4, phi = x   : sum (d_i - u)^3 = lam^3 m        (App. A.6 cubic)
+//   q = 4, phi even  : sum (d_i - u)^3 = lam^3 m (c+u)
+// The cubic is convex and decreasing in u left of the root; Newton from a point
+// left of the root converges monotonically.  u_left must satisfy g(u_left) >= 0.
+__device__ __forceinline__ double solve_block_u(bool q4, bool mag, double lam, double c, double cnt,
+                                                double m, double D1, double D2, double D3,
+                                                double u_left, int* not_converged) {
+  if (!q4) {
+    return mag ? (D1 - lam * m * c) / (cnt + lam * m) : (D1 - lam * m) / cnt;
+  }
+  const double l3m = lam * lam * lam * m;
+  double u = u_left;
+  bool ok = false;
+#pragma unroll 1
+  for (int it = 0; it < 64; ++it) {
+    double g = ((-cnt * u + 3.0 * D1) * u - 3.0 * D2) * u + D3 - (mag ? l3m * (c + u) : l3m);
+    double gp = -3.0 * ((cnt * u - 2.0 * D1) * u + D2) - (mag ? l3m : 0.0);
+    if (!(gp < 0.0)) { ok = true; break; }
+    double du = -g / gp;
+    u += du;
+    if (fabs(du) <= 1e-13 * (fabs(u) + lam)) { ok = true; break; }
+  }
+  if (!ok && not_converged) *not_converged = 1;
+  return u;
+}
+
+// ---------------------------------------------------------------- warp helpers
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace tk

@@ -1,0 +1,175 @@
+// tk_vjp_state.cu -- VJP from the row state saved by the forward pass.
+//
+// Prop. 7 makes the Jacobian of the isotonic solution block diagonal with one
+// rank-one block per pooled block; with w = 1_k there is at most one pooled
+// block per row, and its members are exactly the keys strictly between gamma
+// and gamma + width (width: the key distance at which rho reaches phi'(gamma)).
+// Membership is therefore decided from the key alone and no permutation is
+// needed: two row reductions (A = sum rho' chi g, D = sum rho') and one
+// elementwise pass.  Traffic: theta and g in, grad out (12 B per element).
+#include "tk_common.cuh"
+
+namespace tk {
+
+namespace {
+
+struct RowCtx {
+  float pivot, offset, wid;
+  bool has_block;
+  int m;            // members of the pooled block with w = 1 (ranks a..k-1)
+};
+
+__device__ __forceinline__ RowCtx load_ctx(const Problem& P, const Math& M, long long row) {
+  tk_rowstate st = P.state_in[row];
+  RowCtx c;
+  c.pivot = st.pivot; c.offset = st.offset;
+  c.has_block = st.b > st.a;
+  c.wid = c.has_block ? M.width(st.pivot + st.offset) : 0.0f;
+  c.m = P.k - st.a;
+  return c;
+}
+
+// class of an element: 0 bottom singleton, 1 pooled, 2 top singleton; tt = key - gamma clamped
+__device__ __forceinline__ int classify(const RowCtx& c, float key, float& tt) {
+  float d = key - c.pivot;
+  if (!c.has_block) { tt = 0.0f; return d >= 0.0f ? 2 : 0; }
+  float t = d - c.offset;
+  tt = fminf(fmaxf(t, 0.0f), c.wid);
+  if (t >= c.wid) return 2;
+  return t > 0.0f ? 1 : 0;
+}
+
+__device__ __forceinline__ void accumulate(const Problem& P, const Math& M, const RowCtx& c, float x,
+                                           float g, float& A, float& D) {
+  float tt;
+  float key = sort_key(x, M.mag);
+  if (classify(c, key, tt) == 1) {
+    float dr = M.drho(tt);
+    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
+    D += dr;
+    A += dr * chi * g;
+  }
+}
+
+__device__ __forceinline__ float finish(const Problem& P, const Math& M, const RowCtx& c, float x,
+                                        float g, float ratio) {
+  float tt;
+  float key = sort_key(x, M.mag);
+  int cls = classify(c, key, tt);
+  float sgn = (M.mag && signbit(x)) ? -1.0f : 1.0f;
+  float chi = M.mag ? sgn : (P.mode == TK_TOPK ? x : 1.0f);
+  float o = 0.0f;
+  if (cls == 1) o = M.drho(tt) * (chi * g - ratio);
+  else if (cls == 2 && M.mag) o = chi * g * M.top_slope(key);
+  o *= sgn;
+  if (P.mode == TK_TOPK) {
+    float y = cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f);
+    o += g * y;
+  }
+  return o;
+}
+
+// one warp per row
+__global__ void __launch_bounds__(256) tk_vjp_state_warp(const Problem P) {
+  const Math M = make_math(P);
+  const int lane = threadIdx.x & 31;
+  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= P.rows) return;
+  const int n = P.n;
+  const RowCtx c = load_ctx(P, M, row);
+  const float* x_row = P.theta + row * (long long)n;
+  const float* g_row = P.gout + row * (long long)n;
+  float* o_row = P.out + row * (long long)n;
+  float A = 0.f, D = 0.f;
+  if (c.has_block) {
+    if (P.vec4) {
+      const float4* x4 = reinterpret_cast<const float4*>(x_row);
+      const float4* g4 = reinterpret_cast<const float4*>(g_row);
+      for (int v = lane; 4 * v < n; v += 32) {
+        float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
+        accumulate(P, M, c, x.x, g.x, A, D); accumulate(P, M, c, x.y, g.y, A, D);
+        accumulate(P, M, c, x.z, g.z, A, D); accumulate(P, M, c, x.w, g.w, A, D);
+      }
+    } else {
+      for (int i = lane; i < n; i += 32) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+    }
+    A = warp_sum(A); D = warp_sum(D);
+    if (M.mag) D += (float)c.m;
+  }
+  const float ratio = D > 0.0f ? A / D : 0.0f;
+  if (P.vec4) {
+    const float4* x4 = reinterpret_cast<const float4*>(x_row);
+    const float4* g4 = reinterpret_cast<const float4*>(g_row);
+    float4* o4 = reinterpret_cast<float4*>(o_row);
+    for (int v = lane; 4 * v < n; v += 32) {
+      float4 x = __ldg(x4 + v), g = __ldg(g4 + v), o;
+      o.x = finish(P, M, c, x.x, g.x, ratio); o.y = finish(P, M, c, x.y, g.y, ratio);
+      o.z = finish(P, M, c, x.z, g.z, ratio); o.w = finish(P, M, c, x.w, g.w, ratio);
+      o4[v] = o;
+    }
+  } else {
+    for (int i = lane; i < n; i += 32) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+  }
+}
+
+// one thread block per row
+__global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
+  __shared__ float red[2][8];
+  const Math M = make_math(P);
+  const int t = threadIdx.x, T = blockDim.x, lane = t & 31, warp = t >> 5;
+  const long long row = blockIdx.x;
+  const int n = P.n;
+  const RowCtx c = load_ctx(P, M, row);
+  const float* x_row = P.theta + row * (long long)n;
+  const float* g_row = P.gout + row * (long long)n;
+  float* o_row = P.out + row * (long long)n;
+  float A = 0.f, D = 0.f;
+  if (c.has_block) {           // uniform per row
+    if (P.vec4) {
+      const float4* x4 = reinterpret_cast<const float4*>(x_row);
+      const float4* g4 = reinterpret_cast<const float4*>(g_row);
+      for (int v = t; 4 * v < n; v += T) {
+        float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
+        accumulate(P, M, c, x.x, g.x, A, D); accumulate(P, M, c, x.y, g.y, A, D);
+        accumulate(P, M, c, x.z, g.z, A, D); accumulate(P, M, c, x.w, g.w, A, D);
+      }
+    } else {
+      for (int i = t; i < n; i += T) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+    }
+    A = warp_sum(A); D = warp_sum(D);
+    if (lane == 0) { red[0][warp] = A; red[1][warp] = D; }
+    __syncthreads();
+    A = 0.f; D = 0.f;
+    for (int w = 0; w < (T >> 5); ++w) { A += red[0][w]; D += red[1][w]; }
+    if (M.mag) D += (float)c.m;
+  }
+  const float ratio = D > 0.0f ? A / D : 0.0f;
+  if (P.vec4) {
+    const float4* x4 = reinterpret_cast<const float4*>(x_row);
+    const float4* g4 = reinterpret_cast<const float4*>(g_row);
+    float4* o4 = reinterpret_cast<float4*>(o_row);
+    for (int v = t; 4 * v < n; v += T) {
+      float4 x = __ldg(x4 + v), g = __ldg(g4 + v), o;
+      o.x = finish(P, M, c, x.x, g.x, ratio); o.y = finish(P, M, c, x.y, g.y, ratio);
+      o.z = finish(P, M, c, x.z, g.z, ratio); o.w = finish(P, M, c, x.w, g.w, ratio);
+      o4[v] = o;
+    }
+  } else {
+    for (int i = t; i < n; i += T) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
+  if (P.n <= 512) {
+    const int warps = 8;
+    long long blocks = (P.rows + warps - 1) / warps;
+    tk_vjp_state_warp<<<(unsigned)blocks, warps * 32, 0, stream>>>(P);
+  } else {
+    tk_vjp_state_cta<<<(unsigned)P.rows, 256, 0, stream>>>(P);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace tk

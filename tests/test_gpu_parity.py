@@ -1,0 +1,130 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2302_01425_b200 import binding as tk, build, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+P43 = 4.0 / 3.0
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    build.build()
+    tk.load()
+
+
+def rows_of(n, rows, seed, scale=1.0):
+    return wl.normal_rows(rows, n, seed, scale)
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_small_shapes_all_modes(mode, p):
+    from parity import run_case
+    for n, k, lam, seed in [(1, 1, 1.0, 1), (2, 1, 0.5, 2), (3, 2, 1.0, 3), (5, 5, 1.0, 4),
+                            (32, 4, 1.0, 5), (33, 7, 0.3, 6), (64, 2, 0.1, 7), (100, 10, 2.0, 8),
+                            (127, 126, 1.0, 9), (129, 1, 1.0, 10), (257, 40, 0.05, 11)]:
+        x = rows_of(n, 37, seed)
+        g = wl.cotangent_like(x, seed)
+        run_case(x, k, p, lam, mode, g, label=f"n={n} k={k} lam={lam} mode={mode} p={p}")
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_multi_tile_rows_with_ragged_tail(mode, p):
+    from parity import run_case
+    for n, k, lam, seed in [(1000, 5, 0.5, 21), (1500, 150, 1.0, 22), (4096, 512, 1.0, 23),
+                            (5000, 77, 0.2, 24), (10007, 1000, 1.0, 25), (16384, 2048, 1.0, 26)]:
+        rows = 6 if n > 4096 else 12
+        x = rows_of(n, rows, seed)
+        g = wl.cotangent_like(x, seed)
+        run_case(x, k, p, lam, mode, g, label=f"n={n} k={k} lam={lam} mode={mode} p={p}")
+
+
+def test_ties_and_signed_zeros():
+    from parity import run_case
+    x = wl.class_logit_rows(64, 1000, seed=2, scale=3.0)
+    g = wl.cotangent_like(x, 2)
+    run_case(x, 5, P43, 0.5, tk.TK_TOPK, g, label="class-logit ties")
+    y = rows_of(200, 16, 31)
+    y[:, 10:20] = 0.0
+    y[:, 20:25] = -0.0
+    y[:, 30:60] = y[:, 90:120]
+    y[:, 130:150] = -y[:, 150:170]
+    for mode in (tk.TK_MASK, tk.TK_TOPKMAG):
+        for p in (2.0, P43):
+            run_case(y, 40, p, 0.7, mode, None, label=f"ties mode={mode} p={p}")
+    const = np.full((4, 77), 1.25, np.float32)
+    run_case(const, 7, 2.0, 1.0, tk.TK_MASK, None, label="constant row")
+    run_case(const, 7, P43, 1.0, tk.TK_TOPKMAG, None, label="constant row mag")
+
+
+def test_tiny_config_and_figure1():
+    from parity import run_case
+    for case in wl.tiny_cases():
+        x = case.theta()
+        g = case.cotangent(x)
+        run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
+
+
+def test_extreme_lambda_and_outliers():
+    from parity import run_case
+    x = rows_of(96, 20, 41)
+    for lam in (1e-6, 1e-3, 50.0, 1e4):
+        for p in (2.0, P43):
+            run_case(x, 9, p, lam, tk.TK_MASK, None, label=f"lam={lam} p={p}")
+            run_case(x, 9, p, lam, tk.TK_TOPKMAG, None, label=f"mag lam={lam} p={p}")
+    z = rows_of(300, 10, 42)
+    z[:, 0] = 1e6
+    z[:, 1] = -1e6
+    for p in (2.0, P43):
+        run_case(z, 30, p, 1.0, tk.TK_MASK, wl.cotangent_like(z, 42), label=f"outliers p={p}")
+
+
+def test_argsort_entry_point():
+    from oracle import tko
+    for mode in (tk.TK_MASK, tk.TK_TOPKMAG):
+        for n in (1, 7, 64, 1000, 4099):
+            x = rows_of(n, 9, 50 + n)
+            if n > 10:
+                x[:, 3] = x[:, 9]
+                x[:, 5] = -x[:, 6]
+            th = torch.from_numpy(x).cuda()
+            perm = torch.empty((9, n), dtype=torch.int32, device="cuda")
+            srt = torch.empty((9, n), dtype=torch.float32, device="cuda")
+            tk.tk_argsort(th, 9, n, mode, perm, srt)
+            torch.cuda.synchronize()
+            rp, rs = tko.argsort(x, mode)
+            assert np.array_equal(perm.cpu().numpy(), rp)
+            assert np.array_equal(srt.cpu().numpy().astype(np.float64), rs)
+
+
+def test_nonfinite_input_sets_status_and_returns():
+    x = rows_of(64, 8, 61)
+    x[3, 5] = np.nan
+    x[5, 0] = np.inf
+    th = torch.from_numpy(x).cuda()
+    out = torch.empty_like(th)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    tk.tk_fwd_ex(th, 8, 64, 4, 2.0, 1.0, tk.TK_MASK, out, status_out=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) & tk.TK_FLAG_NONFINITE
+    from oracle import tko
+    ok = [0, 1, 2, 4, 6, 7]
+    ref = tko.fwd(x[ok], 4, 2.0, 1.0, tko.MASK)
+    assert np.max(np.abs(out.cpu().numpy()[ok] - ref)) <= 1e-5
+
+
+def test_runs_are_bit_reproducible():
+    x = rows_of(2048, 32, 71)
+    th = torch.from_numpy(x).cuda()
+    a = torch.empty_like(th)
+    b = torch.empty_like(th)
+    for p in (2.0, P43):
+        tk.tk_fwd(th, 32, 2048, 100, p, 1.0, tk.TK_MASK, a)
+        tk.tk_fwd(th, 32, 2048, 100, p, 1.0, tk.TK_MASK, b)
+        torch.cuda.synchronize()
+        assert torch.equal(a, b)
