@@ -473,8 +473,19 @@ cudaError_t launch_cta(const Problem& P0, cudaStream_t stream) {
     case 8: kern = tk_cta_kernel<8, 256>; break;
     default: kern = (T > 512) ? tk_cta_kernel<16, 1024> : tk_cta_kernel<16, 512>; break;
   }
-  err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  // The opt-in to large dynamic shared memory is per function and per device; it is raised
+  // once to the largest size this file ever asks for.
+  static bool configured[4][64] = {};
+  int dev = 0;
+  err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
+  const int slot = (E == 4) ? 0 : (E == 8) ? 1 : (T > 512 ? 3 : 2);
+  if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
+    const int max_smem = (int)cta_smem_bytes(16384, 1024);
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (err != cudaSuccess) return err;
+    if (dev >= 0 && dev < 64) configured[slot][dev] = true;
+  }
   dim3 grid((unsigned)P.rows), block((unsigned)T);
   kern<<<grid, block, smem, stream>>>(P);
   return cudaGetLastError();
