@@ -8,10 +8,17 @@ namespace tk {
 // on-chip row kernels (tk_cta.cu)
 cudaError_t launch_cta(const Problem& P, cudaStream_t stream);
 int cta_padded_length(int n);
+// sub-warp row kernels for n <= 256 (tk_group.cu)
+cudaError_t launch_group(const Problem& P, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
+constexpr int kMaxGroupN = 256;      // longest row a single warp holds in registers
+
+inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
+  return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
+}
 }  // namespace tk
 
 namespace {
@@ -90,7 +97,7 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
   P.what = tk::W_FWD;
   if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
-  cudaError_t e = tk::launch_cta(P, (cudaStream_t)stream);
+  cudaError_t e = tk::launch_on_chip(P, (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 
@@ -120,7 +127,7 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
     e = tk::launch_vjp_state(P, (cudaStream_t)stream);
   } else {
     if (n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
-    e = tk::launch_cta(P, (cudaStream_t)stream);
+    e = tk::launch_on_chip(P, (cudaStream_t)stream);
   }
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
@@ -138,7 +145,7 @@ tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int3
   P.sorted_out = sorted_out;
   if (opts) P.status = opts->status_out;
   P.vec4 = (n % 4 == 0) && aligned16(theta);
-  cudaError_t e = tk::launch_cta(P, (cudaStream_t)stream);
+  cudaError_t e = tk::launch_on_chip(P, (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 

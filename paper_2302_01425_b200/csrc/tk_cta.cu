@@ -23,20 +23,6 @@ namespace {
 constexpr int PAD_SHIFT = 4;   // one spare 8-byte slot every 16 keeps blocked accesses conflict-free
 __device__ __forceinline__ int pad(int i) { return i + (i >> PAD_SHIFT); }
 
-// packed element: high word = order-preserving key, low word = (0xFFFF - index) << 1 | sign(theta).
-// Larger packed value sorts first; equal keys sort by ascending index.
-__device__ __forceinline__ unsigned long long pack(float x, int idx, bool mag, int n) {
-  if (idx >= n) return (unsigned long long)(((0xFFFFu - (uint32_t)idx) << 1));  // padding sorts last
-  uint32_t hi = f2key(sort_key(x, mag));
-  uint32_t lo = ((0xFFFFu - (uint32_t)idx) << 1) | (__float_as_uint(x) >> 31);
-  return ((unsigned long long)hi << 32) | lo;
-}
-__device__ __forceinline__ float un_key(unsigned long long e) { return key2f((uint32_t)(e >> 32)); }
-__device__ __forceinline__ int un_idx(unsigned long long e) {
-  return 0xFFFF - (int)(((uint32_t)e >> 1) & 0xFFFFu);
-}
-__device__ __forceinline__ bool un_neg(unsigned long long e) { return ((uint32_t)e & 1u) != 0; }
-
 template <int E>
 __device__ __forceinline__ void sort_registers(unsigned long long (&r)[E]) {
   // bitonic network, fully unrolled, descending
