@@ -69,12 +69,16 @@ __device__ __forceinline__ float finish(const Problem& P, const Math& M, const R
   return o;
 }
 
-// one warp per row
-__global__ void __launch_bounds__(256) tk_vjp_state_warp(const Problem P) {
+// G lanes of a warp per row (G = 1..32, power of two), 32/G rows per warp
+template <int G>
+__global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
   const Math M = make_math(P);
   const int lane = threadIdx.x & 31;
-  const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= P.rows) return;
+  const int lig = lane % G;
+  const long long row = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + lane / G;
+  if (row >= P.rows) return;          // whole groups leave together
+  constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
+  const unsigned mask = kGroupBits << (lane / G * G);
   const int n = P.n;
   const RowCtx c = load_ctx(P, M, row);
   const float* x_row = P.theta + row * (long long)n;
@@ -85,15 +89,19 @@ __global__ void __launch_bounds__(256) tk_vjp_state_warp(const Problem P) {
     if (P.vec4) {
       const float4* x4 = reinterpret_cast<const float4*>(x_row);
       const float4* g4 = reinterpret_cast<const float4*>(g_row);
-      for (int v = lane; 4 * v < n; v += 32) {
+      for (int v = lig; 4 * v < n; v += G) {
         float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
         accumulate(P, M, c, x.x, g.x, A, D); accumulate(P, M, c, x.y, g.y, A, D);
         accumulate(P, M, c, x.z, g.z, A, D); accumulate(P, M, c, x.w, g.w, A, D);
       }
     } else {
-      for (int i = lane; i < n; i += 32) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+      for (int i = lig; i < n; i += G) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
     }
-    A = warp_sum(A); D = warp_sum(D);
+#pragma unroll
+    for (int o = G >> 1; o > 0; o >>= 1) {
+      A += __shfl_xor_sync(mask, A, o);
+      D += __shfl_xor_sync(mask, D, o);
+    }
     if (M.mag) D += (float)c.m;
   }
   const float ratio = D > 0.0f ? A / D : 0.0f;
@@ -101,14 +109,14 @@ __global__ void __launch_bounds__(256) tk_vjp_state_warp(const Problem P) {
     const float4* x4 = reinterpret_cast<const float4*>(x_row);
     const float4* g4 = reinterpret_cast<const float4*>(g_row);
     float4* o4 = reinterpret_cast<float4*>(o_row);
-    for (int v = lane; 4 * v < n; v += 32) {
+    for (int v = lig; 4 * v < n; v += G) {
       float4 x = __ldg(x4 + v), g = __ldg(g4 + v), o;
       o.x = finish(P, M, c, x.x, g.x, ratio); o.y = finish(P, M, c, x.y, g.y, ratio);
       o.z = finish(P, M, c, x.z, g.z, ratio); o.w = finish(P, M, c, x.w, g.w, ratio);
       o4[v] = o;
     }
   } else {
-    for (int i = lane; i < n; i += 32) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+    for (int i = lig; i < n; i += G) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
   }
 }
 
@@ -163,9 +171,19 @@ __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
   if (P.n <= 512) {
-    const int warps = 8;
-    long long blocks = (P.rows + warps - 1) / warps;
-    tk_vjp_state_warp<<<(unsigned)blocks, warps * 32, 0, stream>>>(P);
+    // lanes per row: one float4 (or 4 scalars) per lane and pass where possible
+    int G = 1;
+    while (G < 32 && G * 4 < P.n) G <<= 1;
+    const long long rows_per_block = 8 * (32 / G);
+    const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
+    switch (G) {
+      case 1: tk_vjp_state_group<1><<<blocks, 256, 0, stream>>>(P); break;
+      case 2: tk_vjp_state_group<2><<<blocks, 256, 0, stream>>>(P); break;
+      case 4: tk_vjp_state_group<4><<<blocks, 256, 0, stream>>>(P); break;
+      case 8: tk_vjp_state_group<8><<<blocks, 256, 0, stream>>>(P); break;
+      case 16: tk_vjp_state_group<16><<<blocks, 256, 0, stream>>>(P); break;
+      default: tk_vjp_state_group<32><<<blocks, 256, 0, stream>>>(P); break;
+    }
   } else {
     tk_vjp_state_cta<<<(unsigned)P.rows, 256, 0, stream>>>(P);
   }
