@@ -12,6 +12,13 @@ int cta_padded_length(int n);
 cudaError_t launch_group(const Problem& P, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
+cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream);
+// rows held in global memory (tk_long.cu)
+size_t long_workspace_bytes(long long rows, int n);
+cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_dst, bool skip_map,
+                        cudaStream_t stream);
+tk_rowstate* long_workspace_state(void* workspace, long long rows, int n);
+void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
 constexpr int kMaxGroupN = 256;      // longest row a single warp holds in registers
@@ -24,6 +31,15 @@ inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Long rows need the caller's scratch: present, 256-byte aligned and large enough.
+tk_status check_workspace(const tk_opts* opts, int64_t rows, int64_t n) {
+  if (rows > 65535) return TK_ERR_UNSUPPORTED;            // rows ride on gridDim.y there
+  if (!opts || !opts->workspace) return TK_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(opts->workspace) & 255u) return TK_ERR_WORKSPACE;
+  if (opts->workspace_bytes < tk::long_workspace_bytes(rows, (int)n)) return TK_ERR_WORKSPACE;
+  return TK_OK;
+}
 
 // q = p/(p-1) must be 2 or 4 (p = 2 or p = 4/3).
 tk_status classify_p(double p, int* q4) {
@@ -75,9 +91,9 @@ const char* tk_status_string(int status) {
 }
 
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver) {
-  (void)rows; (void)k; (void)p; (void)mode; (void)solver;
-  if (n <= tk::kMaxOnChipN) return 0;
-  return 0;
+  (void)k; (void)p; (void)mode; (void)solver;
+  if (rows <= 0 || n <= tk::kMaxOnChipN || n > 0x7fffffff) return 0;
+  return tk::long_workspace_bytes(rows, (int)n);
 }
 
 tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
@@ -90,13 +106,18 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
   int solver = opts ? opts->solver : TK_SOLVER_AUTO;
   if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_DYKSTRA) return TK_ERR_INVALID_ARG;
   if (solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
-  if (n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, lambda, mode);
   P.out = out;
   P.what = tk::W_FWD;
   if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
+  if (n > tk::kMaxOnChipN) {
+    s = check_workspace(opts, rows, n);
+    if (s != TK_OK) return s;
+    cudaError_t el = tk::launch_long(P, opts->workspace, opts->state_out, false, (cudaStream_t)stream);
+    return el == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+  }
   cudaError_t e = tk::launch_on_chip(P, (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
@@ -122,11 +143,23 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (opts) P.status = opts->status_out;
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(grad_out) && aligned16(grad_theta);
   cudaError_t e;
-  if (opts && opts->state_out) {
+  if (n > tk::kMaxOnChipN) {
+    s = check_workspace(opts, rows, n);
+    if (s != TK_OK) return s;
+    P.state_in = opts->state_out;
+    if (!P.state_in) {      // no saved state: sort and solve again, keep only the row state
+      tk::Problem F = P;
+      F.what = tk::W_FWD; F.out = nullptr; F.gout = nullptr;
+      e = tk::launch_long(F, opts->workspace, nullptr, true, (cudaStream_t)stream);
+      if (e != cudaSuccess) return TK_ERR_CUDA;
+      P.state_in = tk::long_workspace_state(opts->workspace, rows, (int)n);
+    }
+    e = tk::launch_vjp_state_long(P, tk::long_workspace_partials(opts->workspace, rows, (int)n),
+                                  (cudaStream_t)stream);
+  } else if (opts && opts->state_out) {
     P.state_in = opts->state_out;
     e = tk::launch_vjp_state(P, (cudaStream_t)stream);
   } else {
-    if (n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
     e = tk::launch_on_chip(P, (cudaStream_t)stream);
   }
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
@@ -137,7 +170,7 @@ tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int3
   if (rows < 0 || n < 1 || mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
   if (rows == 0) return TK_OK;
   if (theta == nullptr || perm_out == nullptr) return TK_ERR_INVALID_ARG;
-  if (n > tk::kMaxOnChipN || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
+  if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
   tk::Problem P;
   fill(P, theta, rows, n, 1, 0, 1.0, mode);
   P.what = tk::W_ARGSORT;
@@ -145,6 +178,12 @@ tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int3
   P.sorted_out = sorted_out;
   if (opts) P.status = opts->status_out;
   P.vec4 = (n % 4 == 0) && aligned16(theta);
+  if (n > tk::kMaxOnChipN) {
+    tk_status s = check_workspace(opts, rows, n);
+    if (s != TK_OK) return s;
+    cudaError_t el = tk::launch_long(P, opts->workspace, nullptr, true, (cudaStream_t)stream);
+    return el == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+  }
   cudaError_t e = tk::launch_on_chip(P, (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }

@@ -16,6 +16,8 @@ namespace tk {
 
 enum What { W_FWD = 0, W_VJP = 1, W_ARGSORT = 2 };
 
+constexpr int kLongTile = 4096;   // elements per thread block in the kernels for rows held in global memory
+
 struct Problem {
   const float* theta;
   const float* gout;        // cotangent (VJP only)

@@ -167,7 +167,72 @@ __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
   }
 }
 
+// Rows held in global memory: per-tile partial sums, then every block re-reduces them
+// (no atomics, so results do not depend on scheduling) and finishes its own tile.
+__global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, float2* partial, int tiles) {
+  __shared__ float red[2][8];
+  const Math M = make_math(P);
+  const long long row = blockIdx.y;
+  const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
+  const RowCtx c = load_ctx(P, M, row);
+  float A = 0.f, D = 0.f;
+  if (c.has_block) {
+    const float* x_row = P.theta + row * (long long)n;
+    const float* g_row = P.gout + row * (long long)n;
+    const int start = tile * kLongTile;
+#pragma unroll 4
+    for (int j = 0; j < kLongTile / 256; ++j) {
+      const int i = start + j * 256 + t;
+      if (i < n) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+    }
+  }
+  A = warp_sum(A); D = warp_sum(D);
+  if ((t & 31) == 0) { red[0][t >> 5] = A; red[1][t >> 5] = D; }
+  __syncthreads();
+  if (t == 0) {
+    float a = 0.f, d = 0.f;
+    for (int w = 0; w < 8; ++w) { a += red[0][w]; d += red[1][w]; }
+    partial[row * (long long)tiles + tile] = make_float2(a, d);
+  }
+}
+
+__global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const float2* partial, int tiles) {
+  __shared__ double red[2][8];
+  const Math M = make_math(P);
+  const long long row = blockIdx.y;
+  const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
+  const RowCtx c = load_ctx(P, M, row);
+  double A = 0.0, D = 0.0;
+  for (int i = t; i < tiles; i += 256) { float2 v = partial[row * (long long)tiles + i]; A += v.x; D += v.y; }
+  A = warp_sum(A); D = warp_sum(D);
+  if ((t & 31) == 0) { red[0][t >> 5] = A; red[1][t >> 5] = D; }
+  __syncthreads();
+  A = 0.0; D = 0.0;
+  for (int w = 0; w < 8; ++w) { A += red[0][w]; D += red[1][w]; }
+  if (M.mag && c.has_block) D += (double)c.m;
+  const float ratio = D > 0.0 ? (float)(A / D) : 0.0f;
+  const float* x_row = P.theta + row * (long long)n;
+  const float* g_row = P.gout + row * (long long)n;
+  float* o_row = P.out + row * (long long)n;
+  const int start = tile * kLongTile;
+#pragma unroll 4
+  for (int j = 0; j < kLongTile / 256; ++j) {
+    const int i = start + j * 256 + t;
+    if (i < n) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+  }
+}
+
 }  // namespace
+
+// scratch: rows * ceil(n / kLongTile) * 8 bytes
+cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream) {
+  const int tiles = (P.n + kLongTile - 1) / kLongTile;
+  const dim3 grid((unsigned)tiles, (unsigned)P.rows);
+  float2* partial = static_cast<float2*>(scratch);
+  tk_vjp_long_partial<<<grid, 256, 0, stream>>>(P, partial, tiles);
+  tk_vjp_long_finish<<<grid, 256, 0, stream>>>(P, partial, tiles);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
   if (P.n <= 512) {

@@ -128,3 +128,50 @@ def test_runs_are_bit_reproducible():
         tk.tk_fwd(th, 32, 2048, 100, p, 1.0, tk.TK_MASK, b)
         torch.cuda.synchronize()
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_rows_held_in_global_memory(mode, p):
+    from parity import run_case
+    for n, k, lam, rows, seed in [(16385, 1638, 1.0, 3, 81), (20011, 77, 0.3, 2, 82), (40000, 4000, 1.0, 2, 83),
+                                  (70001, 35000, 0.05, 1, 84)]:
+        x = rows_of(n, rows, seed)
+        if seed == 82:
+            x[:, 100:400] = x[:, 5000:5300]        # exact ties across tiles
+        g = wl.cotangent_like(x, seed)
+        run_case(x, k, p, lam, mode, g, label=f"long n={n} k={k} lam={lam} mode={mode} p={p}")
+
+
+def test_long_rows_need_a_workspace():
+    n = 20000
+    th = torch.zeros((1, n), device="cuda")
+    out = torch.empty_like(th)
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd(th, 1, n, 10, 2.0, 1.0, tk.TK_MASK, out)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+    need = tk.tk_workspace_bytes(1, n, 10, 2.0, tk.TK_MASK)
+    assert need > 0
+    small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 1, n, 10, 2.0, 1.0, tk.TK_MASK, out, workspace=small)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+
+
+def test_pruning_config_full_size():
+    from parity import run_case
+    case = wl.pruning_case()
+    x = case.theta()
+    g = case.cotangent(x)
+    res = run_case(x, case.k, case.p, case.lam, case.mode, g, label="pruning 1 x 4194304")
+    print("pruning", res)
+
+
+def test_sweep_n32768_sampled_rows():
+    from parity import run_case
+    for case in wl.shape_sweep_cases():
+        if case.n != 32768:
+            continue
+        x = case.theta(rows=3)
+        g = case.cotangent(x)
+        run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
