@@ -118,6 +118,38 @@ tk_status tk_vjp(const float *theta, const float *grad_out, int64_t rows, int64_
 tk_status tk_argsort(const float *theta, int64_t rows, int64_t n, int mode, int32_t *perm_out,
                      float *sorted_out, const tk_opts *opts, tk_stream stream);
 
+/* Forward pass that brings its own scratch memory.  The paper has no counterpart
+ * to this entry point; it exists for callers that cannot allocate device memory
+ * when they need the operator: a plugin inside an application that owns the
+ * allocator, a real-time loop that must not hit cudaMalloc's implicit device
+ * synchronisation, a process whose memory pool is fully committed.  Such callers
+ * can use tk_fwd for rows of up to 16384 elements (which needs no scratch), but
+ * tk_fwd_ex wants a workspace for longer rows; this call does not.
+ *
+ * Arguments, layout and results are those of tk_fwd (all pointers device
+ * pointers owned by the caller; out[r, :] = operator(theta[r, :]); work is
+ * enqueued on `stream`).  Rows of up to 16384 elements are passed straight to
+ * tk_fwd.  Longer rows run the global-memory pipeline of tk_fwd_ex on a scratch
+ * array compiled into the library: TK_NOALLOC_SCRATCH_BYTES of device memory
+ * that every GPU holds from the moment it loads the library until the process
+ * exits.  The call itself performs no allocation of any kind.
+ *
+ *  - Limit: rows * n <= TK_NOALLOC_MAX_ELEMENTS (and the scratch the shape needs
+ *    must fit the array); anything larger returns TK_ERR_WORKSPACE before any
+ *    launch.  Use tk_fwd_ex with your own workspace for bigger problems.
+ *  - The first call on a device looks up the array's device address
+ *    (cudaGetSymbolAddress) with that device current; make that first call
+ *    outside of any stream capture.
+ *  - All calls on a device share the one array.  It keeps whatever the previous
+ *    call left in it, which is harmless (every word is written before it is read
+ *    within a call), but two calls whose kernels overlap on the GPU -- different
+ *    streams, or concurrent host threads -- race on it and produce garbage.
+ *    Serialise them on one stream.                                              */
+#define TK_NOALLOC_MAX_ELEMENTS (1 << 18)
+#define TK_NOALLOC_SCRATCH_BYTES (8u << 20)
+tk_status tk_fwd_noalloc(const float *theta, int64_t rows, int64_t n, int64_t k, double p,
+                         double lambda, int mode, float *out, tk_stream stream);
+
 const char *tk_status_string(int status);
 
 /* Library build tag, e.g. "tk 0.1 sm_100a".                                     */

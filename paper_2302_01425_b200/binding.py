@@ -24,7 +24,8 @@ TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
 ROWSTATE_BYTES = 16
 
 EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
-           "tk_argsort")
+           "tk_argsort", "tk_fwd_noalloc")
+TK_NOALLOC_MAX_ELEMENTS = 1 << 18
 
 
 class TkOpts(ctypes.Structure):
@@ -65,6 +66,8 @@ def load() -> ctypes.CDLL:
     lib.tk_workspace_bytes.argtypes = [i64, i64, i64, dbl, ci, ci]
     lib.tk_fwd.restype = ci
     lib.tk_fwd.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, vp]
+    lib.tk_fwd_noalloc.restype = ci
+    lib.tk_fwd_noalloc.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, vp]
     lib.tk_fwd_ex.restype = ci
     lib.tk_fwd_ex.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_vjp.restype = ci
@@ -122,6 +125,16 @@ def tk_fwd(theta: torch.Tensor, rows: int, n: int, k: int, p: float, lam: float,
                        _dev(out, torch.float32, "out"), _stream())
     if rc != TK_OK:
         raise TkError(rc, "tk_fwd")
+
+
+def tk_fwd_noalloc(theta: torch.Tensor, rows: int, n: int, k: int, p: float, lam: float, mode: int,
+                   out: torch.Tensor) -> None:
+    """tk_fwd for callers that cannot allocate: long rows use the scratch array built into
+    the library (rows * n <= TK_NOALLOC_MAX_ELEMENTS; calls must not overlap on the GPU)."""
+    rc = load().tk_fwd_noalloc(_dev(theta, torch.float32, "theta"), rows, n, k, p, lam, mode,
+                               _dev(out, torch.float32, "out"), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_fwd_noalloc")
 
 
 def tk_fwd_ex(theta, rows, n, k, p, lam, mode, out, *, solver=TK_SOLVER_AUTO, sweeps=0,
