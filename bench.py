@@ -216,6 +216,8 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--rows", type=int, default=0, help="profiling aid: only the leading ROWS rows of every variant")
     ap.add_argument("--no-e2e", action="store_true", help="profiling aid: skip the host-buffer leg")
+    ap.add_argument("--no-clocks", action="store_true", help="profiling aid: no clock sampling (and no "
+                    "extra replays to give the sampler time)")
     args = ap.parse_args()
     global ROWS_LIMIT
     ROWS_LIMIT = max(0, args.rows)
@@ -248,7 +250,8 @@ def main():
         torch.cuda.synchronize()
 
     res = measure(args.workload, args.steps, max(args.warmup, 3), dev, tk, torch,
-                  graph=not args.no_graph, barrier=barrier, sample_clocks=True, e2e=not args.no_e2e)
+                  graph=not args.no_graph, barrier=barrier, sample_clocks=not args.no_clocks,
+                  e2e=not args.no_e2e)
     if args.no_e2e:
         res.update(e2e_ms_total=float("nan"), e2e_steps=0, h2d_bytes_per_step=0, d2h_bytes_per_step=0)
     ms_total = res["ms_total"]
