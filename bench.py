@@ -306,10 +306,13 @@ def main():
                         r = measure(name, 10, 3, dev, tk, torch, graph=False, barrier=barrier,
                                     sample_clocks=False, e2e=False)
                         v2 = r["elements_per_step"] * r["steps"] / (r["ms_total"] * 1e-3)
-                        extra.append({"workload": name, "value": v2, "unit": UNIT,
-                                      "ms_per_step": r["ms_total"] / r["steps"],
-                                      "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
-                                      "kernels": r["kernels"], "config": r["config"]})
+                        entry = {"workload": name, "value": v2, "unit": UNIT,
+                                 "ms_per_step": r["ms_total"] / r["steps"],
+                                 "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
+                                 "kernels": r["kernels"], "config": r["config"]}
+                        if name.startswith("sweep_n") and int(name[7:]) <= 4096:
+                            entry["dykstra_forward_100_sweeps"] = time_dykstra_forward(name, dev, tk, torch)
+                        extra.append(entry)
                     except tk.TkError as e:
                         extra.append({"workload": name, "unavailable": str(e)})
                 line["other_workloads"] = extra
@@ -317,6 +320,28 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def time_dykstra_forward(workload, dev, tk, torch, sweeps=100, launches=3):
+    """Forward pass through the alternating-projection solver (fixed sweeps), per variant."""
+    out = []
+    for c in workload_cases(workload):
+        th = torch.from_numpy(c.theta()).to(dev)
+        y = torch.empty_like(th)
+        run = lambda: tk.tk_fwd_ex(th, c.rows, c.n, c.k, c.p, c.lam, c.mode, y,
+                                   solver=tk.TK_SOLVER_DYKSTRA, sweeps=sweeps)
+        run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(launches):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / launches
+        out.append({"p": round(c.p, 6), "avg_us": us, "elements_per_s": c.elements / (us * 1e-6)})
+        del th, y
+    return out
 
 
 def measure(workload, steps, warmup, dev, tk, torch, graph, barrier, sample_clocks, e2e):

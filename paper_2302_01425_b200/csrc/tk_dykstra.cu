@@ -1,0 +1,287 @@
+// tk_dykstra.cu -- the alternating-projection solver path (Algorithm 1 and
+// App. A.8 of the paper) for rows held on chip, a fixed number of sweeps.
+//
+// After the same sort as the exact path, the isotonic problem is iterated on
+// the two families of adjacent pairs C1 = {(1,2),(3,4),..}, C2 = {(2,3),(4,5),..}:
+//
+//  p = 2: Dykstra's projection of z onto C1 n C2 in the metric c, with
+//    z_i = s_i - lambda w_i, c_i = 1          (phi = x)
+//    z_i = s_i / c_i,        c_i = 1 + lambda w_i   (phi = x^2/2; completing the
+//    square of h_i).  The linear term is applied once, through z (the printed
+//    iteration, which subtracts w in both half-steps, converges to the
+//    projection of s - 2w).  The correction kept for a pair (a, b) is one scalar
+//    delta >= 0: the pair's corrections are (-c_b delta, +c_a delta).
+//  p = 4/3, phi = x: block coordinate ascent on the duals alpha_j >= 0 of
+//    v_j >= v_{j+1}; each coordinate solves its two-variable problem in closed
+//    form (depressed cubic t^3 + 3 d^2 t + B = 0 by Cardano, one Newton step),
+//    odd coordinates then even coordinates.  The output needs no cube root:
+//    rho(s_i - v_i) = w_i - alpha_i + alpha_{i-1}.
+//
+// Each thread (lane) owns an even number of consecutive sorted ranks, so every C1
+// pair is thread-local and one C2 pair per thread crosses to the next thread.
+#include "tk_common.cuh"
+#include "tk_cta_sort.cuh"
+#include "tk_group_sort.cuh"
+
+namespace tk {
+
+namespace {
+
+// One Dykstra step on a pair in the metric (ca, cb): a, b are the current iterate, delta the
+// stored correction; on return a >= b holds and delta is the new correction.
+__device__ __forceinline__ void dyk_pair(float& a, float& b, float& delta, float ca, float cb) {
+  const float ta = a - cb * delta, tb = b + ca * delta;
+  const float d = fmaxf(0.0f, (tb - ta) / (ca + cb));
+  a = ta + cb * d;
+  b = tb - ca * d;
+  delta = d;
+}
+
+// Dual coordinate of the constraint between keys s1 >= s2 (weights w1, w2), neighbours' duals fixed.
+__device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w2, float a_prev,
+                                           float a_next, const Math& M) {
+  const float c1 = w1 + a_prev, c2 = w2 - a_next;
+  const float v1 = s1 - M.lam * cbrtf(c1), v2 = s2 - M.lam * cbrtf(c2);
+  if (v1 >= v2) return 0.0f;
+  const float d = 0.5f * (s1 - s2), m = 0.5f * (s1 + s2);
+  const float B = 0.5f * M.lam3 * (c1 + c2);
+  const float d2 = d * d;
+  const float R = sqrtf(0.25f * B * B + d2 * d2 * d2);
+  const float big = -copysignf(cbrtf(0.5f * fabsf(B) + R), B);
+  float t = (big != 0.0f) ? big - d2 / big : 0.0f;
+  {   // one Newton step on the increasing cubic t^3 + 3 d^2 t + B
+    const float f = fmaf(t * t + 3.0f * d2, t, B), fp = 3.0f * (t * t + d2);
+    if (fp > 0.0f) t -= f / fp;
+  }
+  const float z = (s1 - (m + t)) * M.inv_lam;
+  return fmaxf(0.0f, c1 - z * z * z);
+}
+
+// The solver on E consecutive ranks per thread.  Exchange with the neighbouring threads goes
+// through the two callables: next0(x) returns the NEXT thread's x, prev_last(x) the PREVIOUS thread's.
+// On return y[i] = rho(s_i - v_i).
+template <int E, typename NextF, typename PrevF, typename SyncF>
+__device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
+                                            bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
+                                            SyncF sync, float (&y)[E]) {
+  const int n = P.n, k = P.k;
+  const int sweeps = P.sweeps > 0 ? P.sweeps : 100;
+  const float s_next = next_of(s[0]);                      // key of the next thread's first rank
+  sync();
+  const bool cross = has_next && (rank0 + E) < n;          // pair (rank0 + E - 1, rank0 + E) exists
+  auto wgt = [&](int rk) -> float { return rk < k ? 1.0f : 0.0f; };
+  if (!M.q4) {
+    float v[E], c[E], pd[E / 2], qd[E / 2];
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const float w = wgt(rank0 + i);
+      c[i] = M.mag ? 1.0f + M.lam * w : 1.0f;
+      v[i] = M.mag ? s[i] / c[i] : s[i] - M.lam * w;
+    }
+#pragma unroll
+    for (int j = 0; j < E / 2; ++j) { pd[j] = 0.0f; qd[j] = 0.0f; }
+    const float c_next = M.mag ? 1.0f + M.lam * wgt(rank0 + E) : 1.0f;
+#pragma unroll 1
+    for (int it = 0; it < sweeps; ++it) {
+#pragma unroll
+      for (int j = 0; j < E / 2; ++j)
+        if (rank0 + 2 * j + 1 < n) dyk_pair(v[2 * j], v[2 * j + 1], pd[j], c[2 * j], c[2 * j + 1]);
+      // C2: the pair that crosses to the next thread, then the thread-local ones
+      float nb = next_of(v[0]);
+      float mine = v[E - 1];
+      if (cross) dyk_pair(mine, nb, qd[E / 2 - 1], c[E - 1], c_next);
+      v[E - 1] = mine;
+#pragma unroll
+      for (int j = 0; j < E / 2 - 1; ++j)
+        if (rank0 + 2 * j + 2 < n) dyk_pair(v[2 * j + 1], v[2 * j + 2], qd[j], c[2 * j + 1], c[2 * j + 2]);
+      sync();
+      const float back = prev_of(nb);                      // what the previous thread made of my first rank
+      if (has_prev && rank0 < n) v[0] = back;
+      sync();
+    }
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const float vi = M.mag ? fmaxf(v[i], 0.0f) : v[i];
+      y[i] = (s[i] - vi) * M.inv_lam;
+    }
+  } else {
+    // alpha of constraint (rank0 + i, rank0 + i + 1): i even -> ao[i/2], i odd -> ae[i/2]
+    float ao[E / 2], ae[E / 2];
+#pragma unroll
+    for (int j = 0; j < E / 2; ++j) { ao[j] = 0.0f; ae[j] = 0.0f; }
+    float prev_e = 0.0f;                                   // previous thread's last even-family dual
+#pragma unroll 1
+    for (int it = 0; it < sweeps; ++it) {
+#pragma unroll
+      for (int j = 0; j < E / 2; ++j) {
+        const int rk = rank0 + 2 * j;
+        if (rk + 1 < n) {
+          const float a_prev = (j == 0) ? prev_e : ae[j - 1];
+          ao[j] = bca_alpha(s[2 * j], s[2 * j + 1], wgt(rk), wgt(rk + 1), a_prev, ae[j], M);
+        }
+      }
+      const float next_o = next_of(ao[0]);
+      sync();
+#pragma unroll
+      for (int j = 0; j < E / 2; ++j) {
+        const int rk = rank0 + 2 * j + 1;
+        if (j < E / 2 - 1) {
+          if (rk + 1 < n) ae[j] = bca_alpha(s[2 * j + 1], s[2 * j + 2], wgt(rk), wgt(rk + 1), ao[j], ao[j + 1], M);
+        } else if (cross) {
+          const float a_next = (rk + 2 < n) ? next_o : 0.0f;
+          ae[j] = bca_alpha(s[E - 1], s_next, wgt(rk), wgt(rk + 1), ao[j], a_next, M);
+        }
+      }
+      const float pe = prev_of(ae[E / 2 - 1]);
+      prev_e = has_prev ? pe : 0.0f;
+      sync();
+    }
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const float a_i = (i & 1) ? ae[i / 2] : ao[i / 2];
+      const float a_im1 = (i == 0) ? prev_e : ((i & 1) ? ao[i / 2] : ae[i / 2 - 1]);
+      y[i] = wgt(rank0 + i) - a_i + a_im1;
+    }
+  }
+}
+
+// ------------------------------------------------------------------ rows of up to 256 elements
+template <int G>
+__global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) {
+  constexpr int N = G * EPL;
+  constexpr int GROUPS = 128 / G;
+  constexpr int STRIDE = N + (N >> 3) + 1;
+  __shared__ float stage_all[GROUPS][STRIDE];
+  const int tid = threadIdx.x;
+  const int grp = tid / G, lig = tid % G;
+  const long long row = (long long)blockIdx.x * GROUPS + grp;
+  if (row >= P.rows) return;
+  constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
+  const unsigned mask = kGroupBits << ((tid & 31) / G * G);
+  const int n = P.n;
+  const Math M = make_math(P);
+  const float* x_row = P.theta + row * (long long)n;
+  unsigned long long r[EPL];
+  bool bad = false;
+  group_load_pack(P, x_row, lig, M.mag, r, bad);
+  group_sort<G>(r, lig, mask);
+  if (P.perm_out) {
+    int32_t* pr = P.perm_out + row * (long long)n;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) if (EPL * lig + i < n) pr[EPL * lig + i] = un_idx(r[i]);
+  }
+  float s[EPL], y[EPL];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) s[i] = un_key(r[i]);
+  auto next_of = [&](float x) -> float { return __shfl_down_sync(mask, x, 1, G); };
+  auto prev_of = [&](float x) -> float { return __shfl_up_sync(mask, x, 1, G); };
+  auto sync = [&]() {};
+  solve_pairs<EPL>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync, y);
+
+  float* stage = stage_all[grp];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int idx = un_idx(r[i]);
+    if (EPL * lig + i < n && idx < n) stage[pad8(idx)] = (M.mag && un_neg(r[i])) ? -y[i] : y[i];
+  }
+  __syncwarp(mask);
+  float* o_row = P.out + row * (long long)n;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int idx = EPL * lig + i;
+    if (idx < n) { float q = stage[pad8(idx)]; if (P.mode == TK_TOPK) q *= __ldg(x_row + idx); o_row[idx] = q; }
+  }
+  if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
+}
+
+// ------------------------------------------------------------------ rows of up to 16384 elements
+template <int E, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const int T = blockDim.x, t = threadIdx.x, n = P.n, N = P.N;
+  const long long row = blockIdx.x;
+  const Math M = make_math(P);
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
+  float* stage = reinterpret_cast<float*>(smem_raw);
+  float* xch = reinterpret_cast<float*>(keys + pad(N) + 1);   // T + 2 floats
+  const float* x_row = P.theta + row * (long long)n;
+  unsigned long long r[E];
+  bool bad = false;
+  cta_load_sort<E>(P, x_row, keys, r, bad);
+  if (P.perm_out) {
+    int32_t* pr = P.perm_out + row * (long long)n;
+    for (int i = t; i < n; i += T) pr[i] = un_idx(keys[pad(i)]);
+  }
+  float s[E], y[E];
+#pragma unroll
+  for (int i = 0; i < E; ++i) s[i] = un_key(r[i]);
+  // neighbour exchange through xch[]: write own value, barrier, read the neighbour's slot.  The
+  // solver calls sync() after every exchange before the next one overwrites the buffer.
+  auto next_of = [&](float x) -> float { xch[t] = x; __syncthreads(); return (t + 1 < T) ? xch[t + 1] : 0.0f; };
+  auto prev_of = [&](float x) -> float { xch[t] = x; __syncthreads(); return (t > 0) ? xch[t - 1] : 0.0f; };
+  auto sync = [&]() { __syncthreads(); };
+  solve_pairs<E>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, y);
+
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < E; ++i) {
+    const int idx = un_idx(r[i]);
+    if (t * E + i < n && idx < n) stage[idx] = (M.mag && un_neg(r[i])) ? -y[i] : y[i];
+  }
+  __syncthreads();
+  float* o_row = P.out + row * (long long)n;
+  for (int i = t; i < n; i += T) { float q = stage[i]; if (P.mode == TK_TOPK) q *= __ldg(x_row + i); o_row[i] = q; }
+  if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
+}
+
+}  // namespace
+
+int cta_padded_length(int n);
+
+cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
+  Problem P = P0;
+  if (P.n <= 256) {
+    int G = 1;
+    while (G * EPL < P.n) G <<= 1;
+    P.N = G * EPL;
+    const long long groups = 128 / G;
+    const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
+    switch (G) {
+      case 1: tk_group_dykstra_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
+      case 2: tk_group_dykstra_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
+      case 4: tk_group_dykstra_kernel<4><<<blocks, 128, 0, stream>>>(P); break;
+      case 8: tk_group_dykstra_kernel<8><<<blocks, 128, 0, stream>>>(P); break;
+      case 16: tk_group_dykstra_kernel<16><<<blocks, 128, 0, stream>>>(P); break;
+      default: tk_group_dykstra_kernel<32><<<blocks, 128, 0, stream>>>(P); break;
+    }
+    return cudaGetLastError();
+  }
+  P.N = cta_padded_length(P.n);
+  const int E = P.N >= 4096 ? 16 : (P.N >= 1024 ? 8 : 4);
+  const int T = P.N / E;
+  const size_t smem = (size_t)(P.N + (P.N >> PAD_SHIFT) + 1) * 8 + (size_t)(T + 2) * 4 + 16;
+  void (*kern)(const Problem) = nullptr;
+  int slot;
+  switch (E) {
+    case 4: kern = tk_cta_dykstra_kernel<4, 128>; slot = 0; break;
+    case 8: kern = tk_cta_dykstra_kernel<8, 256>; slot = 1; break;
+    default:
+      if (T > 512) { kern = tk_cta_dykstra_kernel<16, 1024>; slot = 3; }
+      else { kern = tk_cta_dykstra_kernel<16, 512>; slot = 2; }
+      break;
+  }
+  static bool configured[4][64] = {};
+  int dev = 0;
+  cudaError_t err = cudaGetDevice(&dev);
+  if (err != cudaSuccess) return err;
+  if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
+    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 1) * 8 + (1024 + 2) * 4 + 16;
+    err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+    if (err != cudaSuccess) return err;
+    if (dev >= 0 && dev < 64) configured[slot][dev] = true;
+  }
+  kern<<<(unsigned)P.rows, (unsigned)T, smem, stream>>>(P);
+  return cudaGetLastError();
+}
+
+}  // namespace tk

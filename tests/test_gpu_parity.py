@@ -175,3 +175,52 @@ def test_sweep_n32768_sampled_rows():
         x = case.theta(rows=3)
         g = case.cotangent(x)
         run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_dykstra_path_matches_oracle_sweeps(p):
+    """Alternating projections with a fixed sweep count: same count in the oracle, <= 1e-5."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    modes = [tk.TK_MASK, tk.TK_TOPK] + ([tk.TK_TOPKMAG] if p == 2.0 else [])
+    shapes = [(1, 1, 1.0), (2, 1, 0.5), (7, 3, 1.0), (8, 8, 1.0), (33, 7, 0.3), (64, 2, 0.1), (64, 8, 1.0),
+              (200, 20, 1.0), (256, 100, 2.0), (257, 40, 0.5), (1000, 5, 0.5), (4096, 512, 1.0), (5000, 77, 0.2)]
+    for mode in modes:
+        for n, k, lam in shapes:
+            for sweeps in (1, 10, 100):
+                if n > 1000 and sweeps == 1:
+                    continue
+                rows = 9 if n <= 1000 else 3
+                x = rows_of(n, rows, 300 + n)
+                th = torch.from_numpy(x).cuda()
+                out = torch.full_like(th, float("nan"))
+                perm = torch.empty((rows, n), dtype=torch.int32, device="cuda")
+                tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=sweeps,
+                             perm_out=perm)
+                torch.cuda.synchronize()
+                ref = tko.dykstra(x, k, p, lam, mode, sweeps=sweeps)
+                got = out.cpu().numpy()
+                assert np.isfinite(got).all()
+                assert np.array_equal(perm.cpu().numpy(), tko.argsort(x, mode)[0])
+                err = rel_err(got, ref).max()
+                assert err <= TOL, (mode, n, k, lam, sweeps, err)
+
+
+def test_dykstra_default_sweeps_and_limits():
+    from oracle import tko
+    x = rows_of(64, 16, 77)
+    th = torch.from_numpy(x).cuda()
+    out = torch.empty_like(th)
+    tk.tk_fwd_ex(th, 16, 64, 2, 2.0, 0.3, tk.TK_MASK, out, solver=tk.TK_SOLVER_DYKSTRA)   # sweeps = 0 -> 100
+    torch.cuda.synchronize()
+    ref = tko.dykstra(x, 2, 2.0, 0.3, tko.MASK, sweeps=100)
+    assert np.max(np.abs(out.cpu().numpy() - ref)) <= 1e-5
+    exact = tko.fwd(x, 2, 2.0, 0.3, tko.MASK)
+    assert np.max(np.abs(out.cpu().numpy() - exact)) <= 1e-4       # small blocks: 100 sweeps reach PAV
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 16, 64, 2, P43, 0.3, tk.TK_TOPKMAG, out, solver=tk.TK_SOLVER_DYKSTRA)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 16, 64, 2, 2.0, 0.3, tk.TK_MASK, out, solver=tk.TK_SOLVER_DYKSTRA,
+                     state_out=tk.new_state(16))
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
