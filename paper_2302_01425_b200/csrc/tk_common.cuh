@@ -70,6 +70,29 @@ __device__ __forceinline__ int un_idx(unsigned long long e) {
 }
 __device__ __forceinline__ bool un_neg(unsigned long long e) { return ((uint32_t)e & 1u) != 0; }
 
+// Branch-free compare-exchange and selection on packed elements.  Written as setp/selp so that
+// the sorting networks compile to predicated selects (no divergent branches).
+__device__ __forceinline__ void ce_desc(unsigned long long& a, unsigned long long& b) {   // a >= b after
+  unsigned long long hi, lo;
+  asm("{\n\t.reg .pred p;\n\tsetp.gt.u64 p, %2, %3;\n\tselp.b64 %0, %2, %3, p;\n\tselp.b64 %1, %3, %2, p;\n\t}"
+      : "=l"(hi), "=l"(lo) : "l"(a), "l"(b));
+  a = hi; b = lo;
+}
+// the larger (keepmax) or the smaller of r and o
+__device__ __forceinline__ unsigned long long pick64(unsigned long long r, unsigned long long o, bool keepmax) {
+  unsigned long long out;
+  asm("{\n\t.reg .pred p, q;\n\tsetp.gt.u64 p, %2, %1;\n\tsetp.ne.u32 q, %3, 0;\n\txor.pred p, p, q;\n\t"
+      "selp.b64 %0, %1, %2, p;\n\t}"
+      : "=l"(out) : "l"(r), "l"(o), "r"((unsigned)keepmax));
+  return out;
+}
+__device__ __forceinline__ unsigned long long sel64(bool c, unsigned long long x, unsigned long long y) {   // c ? x : y
+  unsigned long long out;
+  asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %3, 0;\n\tselp.b64 %0, %1, %2, p;\n\t}"
+      : "=l"(out) : "l"(x), "l"(y), "r"((unsigned)c));
+  return out;
+}
+
 // ---------------------------------------------------------------- scalar math
 struct Math {
   float lam, inv_lam, lam3;

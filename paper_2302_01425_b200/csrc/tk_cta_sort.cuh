@@ -22,11 +22,7 @@ __device__ __forceinline__ void sort_registers(unsigned long long (&r)[E]) {
       for (int i = 0; i < E; ++i) {
         int j = i ^ stride;
         if (j > i) {
-          bool desc = (i & size) == 0;
-          unsigned long long a = r[i], b = r[j];
-          bool sw = desc ? (a < b) : (a > b);
-          r[i] = sw ? b : a;
-          r[j] = sw ? a : b;
+          if ((i & size) == 0) ce_desc(r[i], r[j]); else ce_desc(r[j], r[i]);
         }
       }
     }
@@ -75,21 +71,31 @@ __device__ __forceinline__ void cta_load_sort(const Problem& P, const float* x_r
     const int diag = pos - base;
     const unsigned long long* A = keys;      // run A = [base, base+L), run B = [base+L, base+2L)
     int lo = max(0, diag - L), hi = min(diag, L);
-    while (lo < hi) {
-      int mid = (lo + hi) >> 1;
-      unsigned long long a = A[pad(base + mid)];
-      unsigned long long b = A[pad(base + L + diag - 1 - mid)];
-      if (a > b) lo = mid + 1; else hi = mid;
+    // merge path: the same number of halving steps in every thread (no divergence)
+    for (int span = L; span > 0; span >>= 1) {
+      const bool go = lo < hi;
+      const int mid = go ? (lo + hi) >> 1 : 0;
+      const int ib_probe = go ? diag - 1 - mid : 0;
+      const unsigned long long a = A[pad(base + mid)];
+      const unsigned long long b = A[pad(base + L + ib_probe)];
+      const bool up = a > b;
+      lo = (go && up) ? mid + 1 : lo;
+      hi = (go && !up) ? mid : hi;
     }
     int ia = lo, ib = diag - lo;
     unsigned long long a = (ia < L) ? A[pad(base + ia)] : 0ull;
     unsigned long long b = (ib < L) ? A[pad(base + L + ib)] : 0ull;
 #pragma unroll
     for (int i = 0; i < E; ++i) {
-      bool takeA = a > b;
-      r[i] = takeA ? a : b;
-      if (takeA) { ++ia; a = (ia < L) ? A[pad(base + ia)] : 0ull; }
-      else       { ++ib; b = (ib < L) ? A[pad(base + L + ib)] : 0ull; }
+      const bool takeA = a > b;
+      r[i] = sel64(takeA, a, b);
+      ia += takeA ? 1 : 0;
+      ib += takeA ? 0 : 1;
+      const int nxt = takeA ? ia : L + ib;                 // one load per step, from the run that advanced
+      const bool in = takeA ? (ia < L) : (ib < L);
+      const unsigned long long v = in ? A[pad(base + nxt)] : 0ull;
+      a = sel64(takeA, v, a);
+      b = sel64(takeA, b, v);
     }
     __syncthreads();
 #pragma unroll

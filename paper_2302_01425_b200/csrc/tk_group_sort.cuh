@@ -11,10 +11,7 @@ namespace tk {
 constexpr int EPL = 8;   // elements per lane
 __device__ __forceinline__ int pad8(int i) { return i + (i >> 3); }
 
-__device__ __forceinline__ void ce(unsigned long long& a, unsigned long long& b) {   // a >= b after
-  unsigned long long hi = a > b ? a : b, lo = a > b ? b : a;
-  a = hi; b = lo;
-}
+__device__ __forceinline__ void ce(unsigned long long& a, unsigned long long& b) { ce_desc(a, b); }
 
 __device__ __forceinline__ void sort8(unsigned long long (&r)[EPL]) {
   // 19-comparator network for 8 inputs (descending)
@@ -44,10 +41,7 @@ __device__ __forceinline__ void group_sort(unsigned long long (&r)[EPL], int lig
 #pragma unroll
       for (int i = 0; i < EPL; ++i) o[i] = __shfl_xor_sync(mask, r[EPL - 1 - i], size - 1);
 #pragma unroll
-      for (int i = 0; i < EPL; ++i) {
-        bool take = keepmax ? (o[i] > r[i]) : (o[i] < r[i]);
-        r[i] = take ? o[i] : r[i];
-      }
+      for (int i = 0; i < EPL; ++i) r[i] = pick64(r[i], o[i], keepmax);
     }
 #pragma unroll
     for (int s = size >> 2; s >= 1; s >>= 1) {
@@ -55,8 +49,7 @@ __device__ __forceinline__ void group_sort(unsigned long long (&r)[EPL], int lig
 #pragma unroll
       for (int i = 0; i < EPL; ++i) {
         unsigned long long o = __shfl_xor_sync(mask, r[i], s);
-        bool take = keepmax ? (o > r[i]) : (o < r[i]);
-        r[i] = take ? o : r[i];
+        r[i] = pick64(r[i], o, keepmax);
       }
     }
     merge8(r);
