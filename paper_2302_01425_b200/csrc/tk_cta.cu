@@ -69,7 +69,7 @@ struct RowSolve {       // per-row scalars shared by all threads
 };
 
 template <int E, int MAXT>
-__global__ void __launch_bounds__(MAXT, 1)
+__global__ void __launch_bounds__(MAXT, MAXT == 512 ? 2 : 1)
 tk_cta_kernel(const Problem P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int T = blockDim.x;
@@ -357,7 +357,9 @@ size_t cta_smem_bytes(int N, int T) {
 }
 
 // Picks items-per-thread for a padded row length.
-static int pick_items(int N) { return N >= 4096 ? 16 : (N >= 1024 ? 8 : 4); }
+// Items per thread.  The merge rounds are latency-bound, so the choice favours resident warps:
+// 8 items from N = 512 (64-thread blocks, many per SM), 16 from N = 4096 with registers capped at 64.
+static int pick_items(int N) { return N >= 4096 ? 16 : (N >= 512 ? 8 : 4); }
 
 int cta_padded_length(int n) {
   int N = 128;
@@ -375,7 +377,7 @@ cudaError_t launch_cta(const Problem& P0, cudaStream_t stream) {
   void (*kern)(const Problem) = nullptr;
   switch (E) {
     case 4: kern = tk_cta_kernel<4, 128>; break;
-    case 8: kern = tk_cta_kernel<8, 256>; break;
+    case 8: kern = tk_cta_kernel<8, 512>; break;
     default: kern = (T > 512) ? tk_cta_kernel<16, 1024> : tk_cta_kernel<16, 512>; break;
   }
   // The opt-in to large dynamic shared memory is per function and per device; it is raised
