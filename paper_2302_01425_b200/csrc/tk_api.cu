@@ -23,7 +23,7 @@ tk_rowstate* long_workspace_state(void* workspace, long long rows, int n);
 void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
-constexpr int kMaxGroupN = 256;      // longest row a single warp holds in registers
+constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers
 
 inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);

@@ -168,7 +168,24 @@ __device__ __forceinline__ double solve_block_u(bool q4, bool mag, double lam, d
     return mag ? (D1 - lam * m * c) / (cnt + lam * m) : (D1 - lam * m) / cnt;
   }
   const double l3m = lam * lam * lam * m;
+  // Starting point: with mu = D1/cnt and central moments m2, m3 the equation is the depressed
+  // cubic w^3 + P w + Q = 0 in w = u - mu, P >= 0, solved in fp32 by Cardano (stable form: the
+  // two cube roots multiply to -P/3).  Newton in fp64 then needs a couple of steps; it is safe
+  // from any start (a start right of the root steps to its left, then converges monotonically).
   double u = u_left;
+  {
+    const double mu = D1 / cnt;
+    const double m2 = D2 - D1 * mu;
+    const double m3 = D3 - 3.0 * mu * D2 + 2.0 * mu * mu * D1;
+    const float Pc = (float)((3.0 * m2 + (mag ? l3m : 0.0)) / cnt);
+    const float Qc = (float)((l3m * (mag ? (c + mu) : 1.0) - m3) / cnt);
+    const float third = Pc * (1.0f / 3.0f);
+    const float R = sqrtf(0.25f * Qc * Qc + third * third * third);
+    const float big = -copysignf(cbrtf(0.5f * fabsf(Qc) + R), Qc);
+    const float w = (big != 0.0f) ? big - third / big : 0.0f;
+    const double u0 = mu + (double)w;
+    if (isfinite(u0)) u = u0;
+  }
   bool ok = false;
 #pragma unroll 1
   for (int it = 0; it < 64; ++it) {

@@ -15,11 +15,12 @@ namespace tk {
 
 namespace {
 
-template <int G>
+template <int G, int EPL>
 __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
   constexpr int N = G * EPL;                  // padded row length
   constexpr int GROUPS = 128 / G;             // rows per thread block
-  constexpr int STRIDE = N + (N >> 3) + 1;    // padded slots per array per row
+  constexpr int STRIDE = N + N / EPL + 1;     // padded slots per array per row
+  auto pad8 = [](int i) -> int { return pad_e<EPL>(i); };
   __shared__ float sm[GROUPS][4][STRIDE];     // [0] keys / staging, [1..3] prefix sums of d, d^2, d^3
   __shared__ float sm2[GROUPS][STRIDE];       // second staging buffer (VJP)
 
@@ -40,9 +41,9 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
   const float* x_row = P.theta + row * (long long)n;
   unsigned long long r[EPL];
   bool bad = false;
-  group_load_pack(P, x_row, lig, mag, r, bad);
+  group_load_pack_e<EPL>(P, x_row, lig, mag, r, bad);
 
-  group_sort<G>(r, lig, mask);                // lane `lig` now holds sorted ranks [8 lig, 8 lig + 8)
+  group_sort_e<G, EPL>(r, lig, mask);         // lane `lig` now holds sorted ranks [EPL lig, EPL lig + EPL)
 
   if (P.perm_out) {
     int32_t* pr = P.perm_out + row * (long long)n;
@@ -75,7 +76,6 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
   if (has_block) {
     const float W_hi = (piv == c) ? M.width(c) : c + M.width(c);
     const float W_lo = vtop_c - piv;
-    float e1[EPL], e2[EPL], e3[EPL];
     int c_hi = 0, c_lo = 0;
     float s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
@@ -85,23 +85,22 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
       const bool ge_hi = valid && (di >= W_hi);
       const bool gt_lo = valid && (di > W_lo);
       c_hi += ge_hi; c_lo += gt_lo;
-      e1[i] = s1; e2[i] = s2; e3[i] = s3;          // exclusive within the lane
       if (gt_lo && !ge_hi) { s1 += di; float d2 = di * di; s2 += d2; s3 += d2 * di; }
     }
     const int wl = group_sum<G, int>(c_hi, mask);
     const int wh = group_sum<G, int>(c_lo, mask);
     {
-      const float o1 = group_excl<G>(s1, lig, mask);
+      // exclusive prefix sums of the window terms: lane offsets by shuffles, then a second pass
+      float o1 = group_excl<G>(s1, lig, mask), o2 = 0.f, o3 = 0.f;
+      if (M.q4) { o2 = group_excl<G>(s2, lig, mask); o3 = group_excl<G>(s3, lig, mask); }
 #pragma unroll
-      for (int i = 0; i < EPL; ++i) p1[pad8(EPL * lig + i)] = o1 + e1[i];
-      if (lig == G - 1) p1[pad8(N)] = o1 + s1;
-      if (M.q4) {
-        const float o2 = group_excl<G>(s2, lig, mask);
-        const float o3 = group_excl<G>(s3, lig, mask);
-#pragma unroll
-        for (int i = 0; i < EPL; ++i) { p2[pad8(EPL * lig + i)] = o2 + e2[i]; p3[pad8(EPL * lig + i)] = o3 + e3[i]; }
-        if (lig == G - 1) { p2[pad8(N)] = o2 + s2; p3[pad8(N)] = o3 + s3; }
+      for (int i = 0; i < EPL; ++i) {
+        const int rk = EPL * lig + i;
+        p1[pad8(rk)] = o1;
+        if (M.q4) { p2[pad8(rk)] = o2; p3[pad8(rk)] = o3; }
+        if (rk >= wl && rk < wh) { const float di = un_key(r[i]) - piv; o1 += di; const float d2 = di * di; o2 += d2; o3 += d2 * di; }
       }
+      if (lig == G - 1) { p1[pad8(N)] = o1; if (M.q4) { p2[pad8(N)] = o2; p3[pad8(N)] = o3; } }
     }
     __syncwarp(mask);
 
@@ -162,9 +161,10 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
       const int rk = EPL * lig + i;
       if (rk >= a0 && rk < b0) { const float di = un_key(r[i]) - piv; f1 += di; const float d2 = di * di; f2 += d2; f3 += d2 * di; }
     }
-    const double D1 = group_sum<G, double>((double)f1, mask);
+    // at most 512 well-scaled terms: fp32 tree sums are accurate to a few ulp
+    const double D1 = (double)group_sum<G, float>(f1, mask);
     double D2 = 0.0, D3 = 0.0;
-    if (M.q4) { D2 = group_sum<G, double>((double)f2, mask); D3 = group_sum<G, double>((double)f3, mask); }
+    if (M.q4) { D2 = (double)group_sum<G, float>(f2, mask); D3 = (double)group_sum<G, float>(f3, mask); }
     const double cnt = (double)(b0 - a0), m = (double)(k - a0);
     const double u_left = mag ? (double)W_lo : D1 / cnt - (double)P.lam * (double)cbrtf((float)(m / cnt)) * 1.000001;
     int nc = 0;
@@ -198,7 +198,7 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
     }
     __syncwarp(mask);
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
+    for (int h = 0; h < EPL / 4; ++h) {
       const int base = EPL * lig + 4 * h;
       if (P.vec4) {
         if (base < n) {
@@ -268,18 +268,24 @@ __global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
 
 cudaError_t launch_group(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
+  if (P.n > 256) {      // one warp per row, 16 elements per lane
+    P.N = 512;
+    const unsigned blocks = (unsigned)((P.rows + 3) / 4);
+    tk_group_kernel<32, 16><<<blocks, 128, 0, stream>>>(P);
+    return cudaGetLastError();
+  }
   int G = 1;
-  while (G * EPL < P.n) G <<= 1;
-  P.N = G * EPL;
+  while (G * 8 < P.n) G <<= 1;
+  P.N = G * 8;
   const long long groups = 128 / G;
   const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
   switch (G) {
-    case 1: tk_group_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
-    case 2: tk_group_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
-    case 4: tk_group_kernel<4><<<blocks, 128, 0, stream>>>(P); break;
-    case 8: tk_group_kernel<8><<<blocks, 128, 0, stream>>>(P); break;
-    case 16: tk_group_kernel<16><<<blocks, 128, 0, stream>>>(P); break;
-    default: tk_group_kernel<32><<<blocks, 128, 0, stream>>>(P); break;
+    case 1: tk_group_kernel<1, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 2: tk_group_kernel<2, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 4: tk_group_kernel<4, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 8: tk_group_kernel<8, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 16: tk_group_kernel<16, 8><<<blocks, 128, 0, stream>>>(P); break;
+    default: tk_group_kernel<32, 8><<<blocks, 128, 0, stream>>>(P); break;
   }
   return cudaGetLastError();
 }
