@@ -75,27 +75,48 @@ __global__ void __launch_bounds__(TPB) long_hist_kernel(const float* theta, cons
     hist[(row * RADIX + i) * (long long)tiles + tile] = h[i];
 }
 
-// exclusive scan of hist[row][digit][tile] in (digit, tile) order: one block per row
+// exclusive scan of hist[row][digit][tile] in (digit, tile) order: one block per row.  Each warp
+// owns digits w, w + 32, ..: it sums a digit's tiles with coalesced reads, the 256 digit totals
+// are scanned by the first warps, then each warp scans its digits' tiles 32 at a time.
 __global__ void __launch_bounds__(1024) long_scan_hist_kernel(uint32_t* hist, int tiles) {
-  __shared__ uint32_t part[1024];
+  __shared__ uint32_t dtot[RADIX];
   const long long row = blockIdx.x;
   uint32_t* h = hist + row * (long long)RADIX * tiles;
-  const int total = RADIX * tiles;
-  const int per = (total + 1023) / 1024;
-  const int lo = min(threadIdx.x * per, total), hi = min(lo + per, total);
-  uint32_t s = 0;
-  for (int i = lo; i < hi; ++i) s += h[i];
-  part[threadIdx.x] = s;
-  __syncthreads();
-  // inclusive scan of the 1024 partials (Hillis-Steele)
-  for (int o = 1; o < 1024; o <<= 1) {
-    uint32_t v = (threadIdx.x >= o) ? part[threadIdx.x - o] : 0;
-    __syncthreads();
-    part[threadIdx.x] += v;
-    __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int d = warp; d < RADIX; d += 32) {
+    const uint32_t* hd = h + (long long)d * tiles;
+    uint32_t s = 0;
+    for (int i = lane; i < tiles; i += 32) s += hd[i];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) dtot[d] = s;
   }
-  uint32_t run = part[threadIdx.x] - s;
-  for (int i = lo; i < hi; ++i) { uint32_t v = h[i]; h[i] = run; run += v; }
+  __syncthreads();
+  if (warp == 0) {      // exclusive scan of the 256 digit totals, 8 per lane
+    uint32_t v[8], s = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { v[i] = dtot[lane * 8 + i]; s += v[i]; }
+    uint32_t inc = s;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+    uint32_t run = inc - s;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { dtot[lane * 8 + i] = run; run += v[i]; }
+  }
+  __syncthreads();
+  for (int d = warp; d < RADIX; d += 32) {
+    uint32_t* hd = h + (long long)d * tiles;
+    uint32_t carry = dtot[d];
+    for (int i0 = 0; i0 < tiles; i0 += 32) {
+      const int i = i0 + lane;
+      const uint32_t v = (i < tiles) ? hd[i] : 0u;
+      uint32_t inc = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { uint32_t up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+      if (i < tiles) hd[i] = carry + inc - v;
+      carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+  }
 }
 
 template <bool FIRST>
