@@ -119,12 +119,19 @@ __global__ void __launch_bounds__(1024) long_scan_hist_kernel(uint32_t* hist, in
   }
 }
 
+// Stable scatter of one tile.  Elements are first ranked (warp by warp, in position order, so
+// equal digits keep their order), then the tile is reordered by digit in shared memory so that
+// the global writes are runs of consecutive addresses per digit.
 template <bool FIRST>
 __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, const uint32_t* keys_in,
                                                            const int32_t* idx_in, uint32_t* keys_out,
                                                            int32_t* idx_out, const uint32_t* hist, int n,
                                                            int tiles, int shift, int mag) {
-  __shared__ uint32_t cnt[WARPS][RADIX];     // running per-warp digit counts, then warp bases
+  __shared__ uint32_t cnt[WARPS][RADIX];     // running per-warp digit counts, then warp offsets inside the digit
+  __shared__ uint32_t tstart[RADIX];         // first tile-local position of every digit
+  __shared__ uint32_t gbase[RADIX];          // first global position of this tile's run of every digit
+  __shared__ uint32_t skey[TILE];
+  __shared__ int32_t sidx[TILE];
   const int tile = blockIdx.x;
   const long long row = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -153,11 +160,25 @@ __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, c
     __syncwarp();
   }
   __syncthreads();
-  // per digit: exclusive prefix over the warps, plus the tile's global base
+  // per digit: offsets of the warps inside the digit, the digit's size in this tile, its global base
   for (int d = threadIdx.x; d < RADIX; d += TPB) {
-    uint32_t run = hist[(row * RADIX + d) * (long long)tiles + tile];
+    uint32_t run = 0;
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) { uint32_t v = cnt[w][d]; cnt[w][d] = run; run += v; }
+    tstart[d] = run;
+    gbase[d] = hist[(row * RADIX + d) * (long long)tiles + tile];
+  }
+  __syncthreads();
+  if (warp == 0) {      // exclusive scan of the 256 digit sizes, 8 per lane
+    uint32_t v[8], sum = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { v[i] = tstart[lane * 8 + i]; sum += v[i]; }
+    uint32_t inc = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+    uint32_t run = inc - sum;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) { tstart[lane * 8 + i] = run; run += v[i]; }
   }
   __syncthreads();
 #pragma unroll
@@ -165,10 +186,19 @@ __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, c
     const int pos = wstart + i * 32 + lane;
     if (pos < n) {
       const uint32_t digit = (key[i] >> shift) & 0xFF;
-      const uint32_t dst = cnt[warp][digit] + lrank[i];
-      keys_out[base + dst] = key[i];
-      idx_out[base + dst] = FIRST ? pos : idx_in[base + pos];
+      const uint32_t lp = tstart[digit] + cnt[warp][digit] + lrank[i];
+      skey[lp] = key[i];
+      sidx[lp] = FIRST ? pos : idx_in[base + pos];
     }
+  }
+  __syncthreads();
+  const int count = min(TILE, n - tile * TILE);
+  for (int j = threadIdx.x; j < count; j += TPB) {
+    const uint32_t kk = skey[j];
+    const uint32_t digit = (kk >> shift) & 0xFF;
+    const uint32_t dst = gbase[digit] + ((uint32_t)j - tstart[digit]);
+    keys_out[base + dst] = kk;
+    idx_out[base + dst] = sidx[j];
   }
 }
 
