@@ -32,6 +32,7 @@ struct LongWs {
   uint32_t* keyA; uint32_t* keyB;
   int32_t* idxA; int32_t* idxB;
   uint32_t* hist;        // [rows][RADIX][tiles]
+  uint32_t* dtot;        // [rows][RADIX] digit totals (rows with many tiles)
   float* pin1; float* pin2; float* pin3;   // in-tile exclusive prefix of d, d^2, d^3 (window only)
   double* tsum;          // [rows][3][tiles] tile totals, turned into exclusive offsets
   tk_rowstate* state;    // [rows] when the caller passes none
@@ -116,6 +117,57 @@ __global__ void __launch_bounds__(1024) long_scan_hist_kernel(uint32_t* hist, in
       if (i < tiles) hd[i] = carry + inc - v;
       carry += __shfl_sync(0xffffffffu, inc, 31);
     }
+  }
+}
+
+// The same scan for rows with many tiles, spread over 256 blocks per row: digit totals first,
+// then every block derives its digit's base from the totals and scans its own tiles.
+__global__ void __launch_bounds__(256) long_digit_total_kernel(const uint32_t* hist, uint32_t* dtot, int tiles) {
+  __shared__ uint32_t red[8];
+  const int d = blockIdx.x;
+  const long long row = blockIdx.y;
+  const uint32_t* hd = hist + (row * RADIX + d) * (long long)tiles;
+  uint32_t s = 0;
+  for (int i = threadIdx.x; i < tiles; i += 256) s += hd[i];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t tot = 0;
+    for (int w = 0; w < 8; ++w) tot += red[w];
+    dtot[row * RADIX + d] = tot;
+  }
+}
+
+__global__ void __launch_bounds__(256) long_digit_scan_kernel(uint32_t* hist, const uint32_t* dtot, int tiles) {
+  __shared__ uint32_t red[8];
+  __shared__ uint32_t wsum[8];
+  const int d = blockIdx.x;
+  const long long row = blockIdx.y;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // base of this digit: sum of the totals of the smaller digits
+  uint32_t b = (threadIdx.x < d) ? dtot[row * RADIX + threadIdx.x] : 0u;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) b += __shfl_xor_sync(0xffffffffu, b, o);
+  if (lane == 0) red[warp] = b;
+  __syncthreads();
+  uint32_t carry = 0;
+  for (int w = 0; w < 8; ++w) carry += red[w];
+  uint32_t* hd = hist + (row * RADIX + d) * (long long)tiles;
+  for (int i0 = 0; i0 < tiles; i0 += 256) {
+    const int i = i0 + threadIdx.x;
+    const uint32_t v = (i < tiles) ? hd[i] : 0u;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { uint32_t up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+    __syncthreads();                       // wsum of the previous chunk has been read
+    if (lane == 31) wsum[warp] = inc;
+    __syncthreads();
+    uint32_t woff = 0, tot = 0;
+    for (int w = 0; w < 8; ++w) { if (w < warp) woff += wsum[w]; tot += wsum[w]; }
+    if (i < tiles) hd[i] = carry + woff + inc - v;
+    carry += tot;
   }
 }
 
@@ -307,11 +359,20 @@ __global__ void __launch_bounds__(1024) long_solve_kernel(const Problem P, LongW
   float u = 0.0f;
   if (S.has_block) {        // uniform over the block
     double* ts = ws.tsum + row * 3ll * tiles;
-    // exclusive scan of the tile totals (tiles is small: n / 4096)
-    if (t < 3) {
-      double run = 0.0;
-      double* a = ts + (long long)t * tiles;
-      for (int i = 0; i < tiles; ++i) { double v = a[i]; a[i] = run; run += v; }
+    // exclusive scan of the tile totals: warps 0..2 take one moment each, 32 tiles at a time
+    if (t < 96) {
+      const int lane = t & 31;
+      double* a = ts + (long long)(t >> 5) * tiles;
+      double carry = 0.0;
+      for (int i0 = 0; i0 < tiles; i0 += 32) {
+        const int i = i0 + lane;
+        const double v = (i < tiles) ? a[i] : 0.0;
+        double inc = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) { double up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+        if (i < tiles) a[i] = carry + inc - v;
+        carry += __shfl_sync(0xffffffffu, inc, 31);
+      }
     }
     __syncthreads();
     const float* pin1 = ws.pin1 + row * (long long)n;
@@ -481,6 +542,7 @@ LongWs carve(void* workspace, long long rows, int n, int tiles, size_t* total) {
   o = take(el * 4); w.idxA = reinterpret_cast<int32_t*>(b + o);
   o = take(el * 4); w.idxB = reinterpret_cast<int32_t*>(b + o);
   o = take((size_t)rows * RADIX * tiles * 4); w.hist = reinterpret_cast<uint32_t*>(b + o);
+  o = take((size_t)rows * RADIX * 4); w.dtot = reinterpret_cast<uint32_t*>(b + o);
   o = take(el * 4); w.pin1 = reinterpret_cast<float*>(b + o);
   o = take(el * 4); w.pin2 = reinterpret_cast<float*>(b + o);
   o = take(el * 4); w.pin3 = reinterpret_cast<float*>(b + o);
@@ -509,7 +571,13 @@ static cudaError_t long_sort(const Problem& P, const LongWs& ws, int tiles, cuda
     const int shift = 8 * pass;
     if (pass == 0) long_hist_kernel<true><<<grid, TPB, 0, stream>>>(P.theta, nullptr, ws.hist, P.n, tiles, shift, mag, P.status);
     else long_hist_kernel<false><<<grid, TPB, 0, stream>>>(nullptr, kin, ws.hist, P.n, tiles, shift, mag, nullptr);
-    long_scan_hist_kernel<<<(unsigned)P.rows, 1024, 0, stream>>>(ws.hist, tiles);
+    if (tiles > 64) {
+      const dim3 dgrid(RADIX, (unsigned)P.rows);
+      long_digit_total_kernel<<<dgrid, 256, 0, stream>>>(ws.hist, ws.dtot, tiles);
+      long_digit_scan_kernel<<<dgrid, 256, 0, stream>>>(ws.hist, ws.dtot, tiles);
+    } else {
+      long_scan_hist_kernel<<<(unsigned)P.rows, 1024, 0, stream>>>(ws.hist, tiles);
+    }
     if (pass == 0) long_scatter_kernel<true><<<grid, TPB, 0, stream>>>(P.theta, nullptr, nullptr, kout, iout, ws.hist, P.n, tiles, shift, mag);
     else long_scatter_kernel<false><<<grid, TPB, 0, stream>>>(nullptr, kin, iin, kout, iout, ws.hist, P.n, tiles, shift, mag);
     kin = kout; iin = iout;
