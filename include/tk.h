@@ -47,8 +47,11 @@ typedef enum {
 typedef enum {
   TK_SOLVER_AUTO = 0,
   TK_SOLVER_PAV = 1,      /* exact pooling of adjacent violators (Sec. 5, App. B.2)          */
-  TK_SOLVER_DYKSTRA = 2   /* alternating projections on odd/even pairs (Algorithm 1; for
+  TK_SOLVER_DYKSTRA = 2,  /* alternating projections on odd/even pairs (Algorithm 1; for
                              p != 2 the dual block coordinate ascent of App. A.8)            */
+  TK_SOLVER_THRESHOLD = 3 /* the same exact result as TK_SOLVER_PAV without sorting: root of
+                             the capped-simplex threshold function (Sec. 3, P(1_k)); rows of
+                             up to 16384 elements; no permutation output                     */
 } tk_solver;
 
 typedef enum {

@@ -10,6 +10,8 @@ cudaError_t launch_cta(const Problem& P, cudaStream_t stream);
 int cta_padded_length(int n);
 // sub-warp row kernels for n <= 256 (tk_group.cu)
 cudaError_t launch_group(const Problem& P, cudaStream_t stream);
+// exact forward pass without a sort (tk_thr.cu)
+cudaError_t launch_thr(const Problem& P, cudaStream_t stream);
 // alternating-projection solver path (tk_dykstra.cu)
 cudaError_t launch_dykstra(const Problem& P, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
@@ -106,13 +108,19 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
   if (rows == 0) return TK_OK;
   if (out == nullptr) return TK_ERR_INVALID_ARG;
   int solver = opts ? opts->solver : TK_SOLVER_AUTO;
-  if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_DYKSTRA) return TK_ERR_INVALID_ARG;
+  if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_THRESHOLD) return TK_ERR_INVALID_ARG;
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, lambda, mode);
   P.out = out;
   P.what = tk::W_FWD;
   if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
+  if (solver == TK_SOLVER_THRESHOLD) {
+    // no sort, hence no permutation to return; rows held on chip only
+    if (n > tk::kMaxOnChipN || (opts && opts->perm_out)) return TK_ERR_UNSUPPORTED;
+    cudaError_t et = tk::launch_thr(P, (cudaStream_t)stream);
+    return et == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+  }
   if (solver == TK_SOLVER_DYKSTRA) {
     // Forward pass only: rows held on chip; no row state (the iterate of a fixed number of
     // sweeps has no exact block structure to save); phi even with p = 4/3 has no closed-form pair step.

@@ -181,8 +181,12 @@ __device__ __forceinline__ double solve_block_u(bool q4, bool mag, double lam, d
     const float Qc = (float)((l3m * (mag ? (c + mu) : 1.0) - m3) / cnt);
     const float third = Pc * (1.0f / 3.0f);
     const float R = sqrtf(0.25f * Qc * Qc + third * third * third);
-    const float big = -copysignf(cbrtf(0.5f * fabsf(Qc) + R), Qc);
-    const float w = (big != 0.0f) ? big - third / big : 0.0f;
+    // w = A + B with A = -sign(Q) cbrt(|Q|/2 + R), A B = -P/3 and A^3 + B^3 = -Q; written as
+    // -Q / (A^2 - A B + B^2) it has no cancellation when the linear term dominates
+    const float A = cbrtf(0.5f * fabsf(Qc) + R);
+    const float B = (A != 0.0f) ? third / A : 0.0f;
+    const float den = A * A + third + B * B;
+    const float w = (den > 0.0f) ? -Qc / den : 0.0f;
     const double u0 = mu + (double)w;
     if (isfinite(u0)) u = u0;
   }
@@ -194,7 +198,10 @@ __device__ __forceinline__ double solve_block_u(bool q4, bool mag, double lam, d
     if (!(gp < 0.0)) { ok = true; break; }
     double du = -g / gp;
     u += du;
-    if (fabs(du) <= 1e-13 * (fabs(u) + lam)) { ok = true; break; }
+    // phi = x: gamma enters through differences only, whose scale is lambda.  phi even: the
+    // equation and the cap width depend on gamma = c + u itself, which can be far smaller.
+    const double scale = mag ? fabs(c + u) : fabs(u) + lam;
+    if (fabs(du) <= 1e-13 * scale + 1e-300) { ok = true; break; }
   }
   if (!ok && not_converged) *not_converged = 1;
   return u;

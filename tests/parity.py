@@ -70,7 +70,7 @@ def disputed_rows_ok(theta, k, p, lam, mode, det, gpu_ab, ref_ab):
 
 
 def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.ndarray | None = None,
-             check_perm: bool = True, label: str = ""):
+             check_perm: bool = True, label: str = "", solver: int = 0):
     """Runs forward (+ argsort, + both VJP paths) on the GPU and compares with the oracle.
     Returns a dict of measured errors."""
     theta = np.ascontiguousarray(theta, np.float32)
@@ -83,13 +83,14 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ws_bytes = tk.tk_workspace_bytes(rows, n, k, p, mode)
     ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device=dev) if ws_bytes else None
-    tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, perm_out=perm, state_out=state, workspace=ws,
-                 status_out=status)
+    sorts = solver != tk.TK_SOLVER_THRESHOLD          # the sort-free solver has no permutation to give
+    tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, perm_out=perm if sorts else None, state_out=state,
+                 workspace=ws, status_out=status, solver=solver)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, f"{label}: status {int(status.item())}"
     ref, det = tko.fwd(theta, k, p, lam, mode, details=True)
     res = {}
-    if check_perm:
+    if check_perm and sorts:
         assert np.array_equal(perm.cpu().numpy(), det["perm"]), f"{label}: permutation differs"
     gout = out.cpu().numpy()
     assert np.isfinite(gout).all(), f"{label}: non-finite output"
@@ -97,7 +98,7 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
     res["fwd_max_abs"] = float(np.abs(gout - ref).max())
     assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
     # plain entry point gives the same bits
-    if ws_bytes == 0:
+    if ws_bytes == 0 and sorts:
         out2 = torch.empty_like(out)
         tk.tk_fwd(th, rows, n, k, p, lam, mode, out2)
         assert torch.equal(out, out2), f"{label}: tk_fwd differs from tk_fwd_ex"
@@ -114,7 +115,7 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         keep = np.ones(rows, bool)
         keep[bad] = False
         for name, kwargs in (("vjp_state", {"state": state}), ("vjp_recompute", {})):
-            if name == "vjp_recompute" and ws_bytes:
+            if name == "vjp_recompute" and (ws_bytes or not sorts):
                 continue
             grad = torch.full((rows, n), float("nan"), device=dev)
             tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, workspace=ws, **kwargs)

@@ -224,3 +224,53 @@ def test_dykstra_default_sweeps_and_limits():
         tk.tk_fwd_ex(th, 16, 64, 2, 2.0, 0.3, tk.TK_MASK, out, solver=tk.TK_SOLVER_DYKSTRA,
                      state_out=tk.new_state(16))
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_sort_free_solver_matches_oracle(mode, p):
+    """TK_SOLVER_THRESHOLD: same values, same pooled block, and a row state the VJP accepts."""
+    from parity import run_case
+    shapes = [(1, 1, 1.0, 1), (2, 1, 0.5, 2), (5, 5, 1.0, 4), (33, 7, 0.3, 6), (64, 2, 0.1, 7), (64, 8, 1.0, 7),
+              (257, 40, 0.05, 11), (1000, 5, 0.5, 21), (1500, 150, 1.0, 22), (4096, 512, 1.0, 23),
+              (5000, 77, 0.2, 24), (10007, 1000, 1.0, 25), (16384, 2048, 1.0, 26), (4096, 400, 1e-3, 27)]
+    for n, k, lam, seed in shapes:
+        rows = 4 if n > 4096 else 11
+        x = rows_of(n, rows, seed, 0.02 if lam == 1e-3 else 1.0)
+        g = wl.cotangent_like(x, seed)
+        run_case(x, k, p, lam, mode, g, solver=tk.TK_SOLVER_THRESHOLD,
+                 label=f"sort-free n={n} k={k} lam={lam} mode={mode} p={p}")
+
+
+def test_sort_free_solver_ties_outliers_and_limits():
+    from parity import run_case
+    x = wl.class_logit_rows(64, 1000, seed=2, scale=3.0)
+    run_case(x, 5, P43, 0.5, tk.TK_TOPK, wl.cotangent_like(x, 2), solver=tk.TK_SOLVER_THRESHOLD, label="ties")
+    y = rows_of(200, 16, 31)
+    y[:, 10:20] = 0.0
+    y[:, 20:25] = -0.0
+    y[:, 30:60] = y[:, 90:120]
+    y[:, 130:150] = -y[:, 150:170]
+    for mode in (tk.TK_MASK, tk.TK_TOPKMAG):
+        for p in (2.0, P43):
+            run_case(y, 40, p, 0.7, mode, None, solver=tk.TK_SOLVER_THRESHOLD, label=f"ties mode={mode} p={p}")
+    const = np.full((4, 77), 1.25, np.float32)
+    run_case(const, 7, 2.0, 1.0, tk.TK_MASK, None, solver=tk.TK_SOLVER_THRESHOLD, label="constant row")
+    w = rows_of(96, 20, 41)
+    for p in (2.0, P43):
+        run_case(w, 9, p, 1e-6, tk.TK_MASK, None, solver=tk.TK_SOLVER_THRESHOLD, label=f"lam=1e-6 p={p}")
+        run_case(w, 9, p, 1e-6, tk.TK_TOPKMAG, None, solver=tk.TK_SOLVER_THRESHOLD, label=f"mag lam=1e-6 p={p}")
+    z = rows_of(300, 10, 42)
+    z[:, 0] = 1e6
+    z[:, 1] = -1e6
+    # (lambda = 1e-6 next to keys of 1e6 is left out: there the fp64 oracle's own rho(s - (s - lambda))
+    # is off by eps |s| / lambda = 2e-4, more than the tolerance; the kernels return exactly 1)
+    for lam in (1e-3, 1.0, 50.0, 1e4):
+        for p in (2.0, P43):
+            run_case(z, 30, p, lam, tk.TK_MASK, None, solver=tk.TK_SOLVER_THRESHOLD, label=f"outliers lam={lam}")
+            run_case(z, 30, p, lam, tk.TK_TOPKMAG, None, solver=tk.TK_SOLVER_THRESHOLD, label=f"mag lam={lam}")
+    th = torch.from_numpy(z).cuda()
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 10, 300, 30, 2.0, 1.0, tk.TK_MASK, torch.empty_like(th), solver=tk.TK_SOLVER_THRESHOLD,
+                     perm_out=torch.empty((10, 300), dtype=torch.int32, device="cuda"))
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
