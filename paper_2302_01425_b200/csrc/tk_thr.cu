@@ -50,16 +50,49 @@ __device__ __forceinline__ Sums block_reduce(Sums v, float* red, bool q4) {
   return r;
 }
 
-template <int E, int MAXT>
+// Step du that solves the candidate set's cubic (App. A.6) with the sums taken about the current
+// gamma:  sum (t_i - du)^3 = lam^3 m [(gamma + du) for phi even].  Because the anchor is the
+// current iterate, du -> 0 as the outer iteration converges and fp32 is enough: an error of one
+// ulp of S3 moves du by about 1e-7 of the block's width, and the next pass re-anchors.
+__device__ __forceinline__ float solve_piece_cubic(bool mag, float lam3, float gam, float cnt, float m,
+                                                   float S1, float S2, float S3) {
+  const float l3m = lam3 * m;
+  const float mu = S1 / cnt;
+  const float m2 = fmaxf(S2 - S1 * mu, 0.0f);
+  const float m3 = S3 - 3.0f * mu * S2 + 2.0f * mu * mu * S1;
+  const float Pc = (3.0f * m2 + (mag ? l3m : 0.0f)) / cnt;
+  const float Qc = (l3m * (mag ? (gam + mu) : 1.0f) - m3) / cnt;
+  const float third = Pc * (1.0f / 3.0f);
+  const float R = sqrtf(0.25f * Qc * Qc + third * third * third);
+  const float A = cbrtf(0.5f * fabsf(Qc) + R);
+  const float B = (A != 0.0f) ? third / A : 0.0f;
+  const float den = A * A + third + B * B;
+  float u = mu + ((den > 0.0f) ? -Qc / den : 0.0f);
+  if (!isfinite(u)) u = 0.0f;
+#pragma unroll 1
+  for (int it = 0; it < 12; ++it) {
+    const float g = ((-cnt * u + 3.0f * S1) * u - 3.0f * S2) * u + S3 - (mag ? l3m * (gam + u) : l3m);
+    const float gp = -3.0f * ((cnt * u - 2.0f * S1) * u + S2) - (mag ? l3m : 0.0f);
+    if (!(gp < 0.0f)) break;
+    const float du = -g / gp;
+    u += du;
+    if (fabsf(du) <= 2e-7f * (fabsf(u) + (mag ? gam : 0.0f)) + 1e-37f) break;
+  }
+  return u;
+}
+
+template <int E, int MAXT, bool Q4, bool MAG>
 __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
+  __shared__ int whist[MAXT / 32][256];   // per-warp digit counts (no contention between warps)
   __shared__ int hist[256];
   __shared__ float red[160];
   __shared__ int sh_digit, sh_kk, sh_eq;
   const int T = blockDim.x, t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const int n = P.n, k = P.k;
   const long long row = blockIdx.x;
-  const Math M = make_math(P);
-  const bool mag = M.mag;
+  Math M = make_math(P);
+  M.q4 = Q4; M.mag = MAG;                       // compile-time constants from here on
+  constexpr bool mag = MAG;
   const float* x_row = P.theta + row * (long long)n;
   float x[E];
   bool bad = false;
@@ -78,25 +111,39 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
     for (int i = 0; i < E; ++i) { const int idx = i * T + t; x[i] = (idx < n) ? __ldg(x_row + idx) : 0.0f; }
   }
   auto index_of = [&](int i) -> int { return P.vec4 ? 4 * ((i >> 2) * T + t) + (i & 3) : i * T + t; };
+  // keys once; slots past the end of the row become NaN, which fails every comparison below
+  float key[E];
+  unsigned valid = 0;
 #pragma unroll
-  for (int i = 0; i < E; ++i) if (index_of(i) < n && !isfinite(x[i])) bad = true;
+  for (int i = 0; i < E; ++i) {
+    const bool in = index_of(i) < n;
+    if (in && !isfinite(x[i])) bad = true;
+    valid |= in ? (1u << i) : 0u;
+    key[i] = in ? sort_key(x[i], mag) : __int_as_float(0x7fc00000);
+  }
 
   // ---- 1. the k-th largest key, exactly: MSB-first radix select on the integer keys
   uint32_t prefix = 0, pmask = 0;
   int kk = k;                                   // rank wanted among the keys matching the prefix
 #pragma unroll 1
   for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = t; i < 256; i += T) hist[i] = 0;
-    __syncthreads();
+    for (int i = lane; i < 256; i += 32) whist[warp][i] = 0;
+    __syncwarp();
 #pragma unroll
     for (int i = 0; i < E; ++i) {
-      const uint32_t u = f2key(sort_key(x[i], mag));
-      const bool take = index_of(i) < n && (u & pmask) == prefix;
-      // warp-aggregated: lanes with the same digit send one atomic (the leading byte of real
-      // data falls into a handful of bins)
+      const uint32_t u = f2key(key[i]);
+      const bool take = ((valid >> i) & 1u) && (u & pmask) == prefix;
+      // lanes with the same digit are counted by their first lane, in the warp's own histogram
       const unsigned digit = take ? ((u >> shift) & 255u) : 256u;
       const unsigned peers = __match_any_sync(0xffffffffu, digit);
-      if (take && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+      if (take && lane == __ffs(peers) - 1) whist[warp][digit] += __popc(peers);
+      __syncwarp();
+    }
+    __syncthreads();
+    for (int i = t; i < 256; i += T) {
+      int s = 0;
+      for (int w2 = 0; w2 < (T >> 5); ++w2) s += whist[w2][i];
+      hist[i] = s;
     }
     __syncthreads();
     if (warp == 0) {                            // lane l owns digits 255 - 8 l - j, j = 0..7 (descending)
@@ -131,8 +178,7 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
     float m = -INFINITY;
 #pragma unroll
     for (int i = 0; i < E; ++i) {
-      const float key = sort_key(x[i], mag);
-      if (index_of(i) < n && key < c) m = fmaxf(m, key);
+      if (key[i] < c) m = fmaxf(m, key[i]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
@@ -165,10 +211,9 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
       Sums acc{0, 0, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int i = 0; i < E; ++i) {
-        const float tt = (sort_key(x[i], mag) - piv) - off;
-        const bool valid = index_of(i) < n;
-        const bool top = valid && tt >= w;
-        const bool mid = valid && tt > 0.0f && !top;
+        const float tt = (key[i] - piv) - off;      // NaN for slots past the row: neither top nor mid
+        const bool top = tt >= w;
+        const bool mid = tt > 0.0f && !top;
         acc.ct += top; acc.cm += mid;
         if (mid) { acc.s1 += tt; if (M.q4) { const float t2 = tt * tt; acc.s2 += t2; acc.s3 += t2 * tt; } }
       }
@@ -184,10 +229,12 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
       float du = 0.0f;
       bool have_cand = false;
       if (S.cm > 0 && m >= 1) {
-        int nc = 0;
-        du = (float)solve_block_u(M.q4, mag, (double)P.lam, (double)gam, (double)S.cm, (double)m, (double)S.s1,
-                                  (double)S.s2, (double)S.s3,
-                                  (double)(S.s1 / S.cm - P.lam * 1.01f * cbrtf((float)m / (float)S.cm)), &nc);
+        if (M.q4) {
+          du = solve_piece_cubic(mag, P.lam3, gam, (float)S.cm, (float)m, S.s1, S.s2, S.s3);
+        } else {
+          const float fm = (float)m, fc = (float)S.cm;
+          du = mag ? (S.s1 - P.lam * fm * gam) / (fc + P.lam * fm) : (S.s1 - P.lam * fm) / fc;
+        }
         have_cand = true;
         // Exact root: this point was the solution of the previous set, it sees the same set, and
         // it already solves it (the remaining step is rounding-sized, so applying it cannot move
@@ -227,15 +274,15 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
   float y[E];
 #pragma unroll
   for (int i = 0; i < E; ++i) {
-    const float key = sort_key(x[i], mag);
+    const float kx = key[i];
     float v;
     if (block) {
-      const float tt = (key - piv) - off;
-      if (tt >= wid) v = mag ? M.vtop(key) : 1.0f;
+      const float tt = (kx - piv) - off;
+      if (tt >= wid) v = mag ? M.vtop(kx) : 1.0f;
       else if (tt > 0.0f) v = M.rho(tt);
       else v = 0.0f;
     } else {
-      v = (key >= c) ? (mag ? M.vtop(key) : 1.0f) : 0.0f;
+      v = (kx >= c) ? (mag ? M.vtop(kx) : 1.0f) : 0.0f;
     }
     if (mag) v = signbit(x[i]) ? -v : v;
     if (P.mode == TK_TOPK) v *= x[i];
@@ -264,14 +311,23 @@ cudaError_t launch_thr(const Problem& P0, cudaStream_t stream) {
   while (N < P.n) N <<= 1;
   P.N = N;
   // threads: 32..1024, a multiple of 32; items per thread 4, 8 or 16
-  const int E = N >= 8192 ? 16 : (N >= 2048 ? 8 : 4);
+  const int E = N >= 4096 ? 16 : (N >= 1024 ? 8 : 4);
   const int T = N / E;
   const dim3 grid((unsigned)P.rows);
+  const bool q4 = P.q4 != 0, mag = P.mode == TK_TOPKMAG;
+#define TK_THR_LAUNCH(EE, MT)                                                        \
+  do {                                                                               \
+    if (q4 && mag) tk_thr_kernel<EE, MT, true, true><<<grid, T, 0, stream>>>(P);      \
+    else if (q4) tk_thr_kernel<EE, MT, true, false><<<grid, T, 0, stream>>>(P);       \
+    else if (mag) tk_thr_kernel<EE, MT, false, true><<<grid, T, 0, stream>>>(P);      \
+    else tk_thr_kernel<EE, MT, false, false><<<grid, T, 0, stream>>>(P);              \
+  } while (0)
   switch (E) {
-    case 4: tk_thr_kernel<4, 512><<<grid, T, 0, stream>>>(P); break;
-    case 8: tk_thr_kernel<8, 1024><<<grid, T, 0, stream>>>(P); break;
-    default: tk_thr_kernel<16, 1024><<<grid, T, 0, stream>>>(P); break;
+    case 4: TK_THR_LAUNCH(4, 128); break;
+    case 8: TK_THR_LAUNCH(8, 256); break;
+    default: TK_THR_LAUNCH(16, 1024); break;
   }
+#undef TK_THR_LAUNCH
   return cudaGetLastError();
 }
 
