@@ -311,7 +311,21 @@ def main():
                                  "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
                                  "kernels": r["kernels"], "config": r["config"]}
                         if name.startswith("sweep_n") and int(name[7:]) <= 4096:
-                            entry["dykstra_forward_100_sweeps"] = time_dykstra_forward(name, dev, tk, torch)
+                            entry["dykstra_forward_100_sweeps"] = time_solver_forward(
+                                name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
+                        ncase = workload_cases(name)[0].n
+                        if 512 <= ncase <= 16384:
+                            # the same exact result without the sort (solver = TK_SOLVER_THRESHOLD),
+                            # reported beside the sorted path, never instead of it
+                            sf = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_THRESHOLD)
+                            vj = {round(kx["p"], 6): kx for kx in sf}
+                            fwd_us = sum(x["avg_us"] for x in sf)
+                            vjp_us = r["kernels"][1]["avg_us"] * r["kernels"][1]["launches_per_step"]
+                            el = r["elements_per_step"]
+                            entry["sort_free"] = {
+                                "forward": sf,
+                                "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * el / ((fwd_us + vjp_us) * 1e-6) / 1e9 / peak,
+                                "note": "tk_fwd_ex(solver=TK_SOLVER_THRESHOLD, state saved) + tk_vjp(from state)"}
                         extra.append(entry)
                     except tk.TkError as e:
                         extra.append({"workload": name, "unavailable": str(e)})
@@ -322,14 +336,16 @@ def main():
         dist.destroy_process_group()
 
 
-def time_dykstra_forward(workload, dev, tk, torch, sweeps=100, launches=3):
-    """Forward pass through the alternating-projection solver (fixed sweeps), per variant."""
+def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3):
+    """Forward pass through another solver path (alternating projections with a fixed number of
+    sweeps, or the sort-free exact solver), per variant."""
     out = []
     for c in workload_cases(workload):
         th = torch.from_numpy(c.theta()).to(dev)
         y = torch.empty_like(th)
-        run = lambda: tk.tk_fwd_ex(th, c.rows, c.n, c.k, c.p, c.lam, c.mode, y,
-                                   solver=tk.TK_SOLVER_DYKSTRA, sweeps=sweeps)
+        st = tk.new_state(c.rows, dev) if solver == tk.TK_SOLVER_THRESHOLD else None
+        run = lambda: tk.tk_fwd_ex(th, c.rows, c.n, c.k, c.p, c.lam, c.mode, y, solver=solver, sweeps=sweeps,
+                                   state_out=st)
         run()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
