@@ -203,6 +203,24 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------ multi-rank helpers
+def max_over_ranks(value: float, device=None) -> float:
+    """Slowest rank's time: the job's time when every rank processes its own rows (weak scaling,
+    no collective on the data path).  Works on any initialised backend (nccl on GPUs, gloo on CPU)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(elements_per_rank_step: int, steps: int, world: int, ms_total_max: float) -> float:
+    """elements/s of the whole job: all ranks' elements over the slowest rank's time."""
+    return world * elements_per_rank_step * steps / (ms_total_max * 1e-3)
+
+
 # ------------------------------------------------------------------ GPU arm
 def main():
     ap = argparse.ArgumentParser()
@@ -256,18 +274,14 @@ def main():
         res.update(e2e_ms_total=float("nan"), e2e_steps=0, h2d_bytes_per_step=0, d2h_bytes_per_step=0)
     ms_total = res["ms_total"]
     if world > 1:
-        tmax = torch.tensor([ms_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_total = float(tmax.item())
-        e2e_t = torch.tensor([res["e2e_ms_total"]], device=dev, dtype=torch.float64)
-        dist.all_reduce(e2e_t, op=dist.ReduceOp.MAX)
-        res["e2e_ms_total"] = float(e2e_t.item())
+        ms_total = max_over_ranks(ms_total, dev)
+        res["e2e_ms_total"] = max_over_ranks(res["e2e_ms_total"], dev)
 
     if rank == 0:
         peak, peak_kind = hbm_peak()
         steps = res["steps"]
         el_step = res["elements_per_step"]
-        value = world * el_step * steps / (ms_total * 1e-3)
+        value = whole_job_value(el_step, steps, world, ms_total)
         dom = res["dominant"]
         achieved = dom["alg_bytes_per_launch"] / (dom["avg_us"] * 1e-6) / 1e9
         line = {
