@@ -15,8 +15,10 @@ namespace tk {
 
 namespace {
 
+// 8 elements per lane: registers capped at 64 so that 8 blocks (32 warps) fit an SM and a 1024-block
+// grid (16384 rows of 64) is a single wave on 148 SMs.
 template <int G, int EPL>
-__global__ void __launch_bounds__(128) tk_group_kernel(const Problem P) {
+__global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const Problem P) {
   constexpr int N = G * EPL;                  // padded row length
   constexpr int GROUPS = 128 / G;             // rows per thread block
   constexpr int STRIDE = N + N / EPL + 1;     // padded slots per array per row

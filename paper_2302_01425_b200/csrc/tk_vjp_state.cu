@@ -69,8 +69,9 @@ __device__ __forceinline__ float finish(const Problem& P, const Math& M, const R
   return o;
 }
 
-// G lanes of a warp per row (G = 1..32, power of two), 32/G rows per warp
-template <int G>
+// G lanes of a warp per row (G = 1..32, power of two), 32/G rows per warp.  Every lane keeps its
+// CH float4 chunks of theta and g in registers, so the row is read from memory once (n <= 4 G CH).
+template <int G, int CH>
 __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
   const Math M = make_math(P);
   const int lane = threadIdx.x & 31;
@@ -80,23 +81,37 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
   constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
   const unsigned mask = kGroupBits << (lane / G * G);
   const int n = P.n;
-  const RowCtx c = load_ctx(P, M, row);
   const float* x_row = P.theta + row * (long long)n;
   const float* g_row = P.gout + row * (long long)n;
   float* o_row = P.out + row * (long long)n;
+  float x[CH][4], g[CH][4];
+  if (P.vec4) {
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      const int v = c * G + lig;
+      float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), gv = xv;
+      if (4 * v < n) { xv = __ldg(reinterpret_cast<const float4*>(x_row) + v); gv = __ldg(reinterpret_cast<const float4*>(g_row) + v); }
+      x[c][0] = xv.x; x[c][1] = xv.y; x[c][2] = xv.z; x[c][3] = xv.w;
+      g[c][0] = gv.x; g[c][1] = gv.y; g[c][2] = gv.z; g[c][3] = gv.w;
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < CH; ++c)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int i = 4 * (c * G + lig) + j;
+        x[c][j] = (i < n) ? __ldg(x_row + i) : 0.0f;
+        g[c][j] = (i < n) ? __ldg(g_row + i) : 0.0f;
+      }
+  }
+  const RowCtx c = load_ctx(P, M, row);
   float A = 0.f, D = 0.f;
   if (c.has_block) {
-    if (P.vec4) {
-      const float4* x4 = reinterpret_cast<const float4*>(x_row);
-      const float4* g4 = reinterpret_cast<const float4*>(g_row);
-      for (int v = lig; 4 * v < n; v += G) {
-        float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
-        accumulate(P, M, c, x.x, g.x, A, D); accumulate(P, M, c, x.y, g.y, A, D);
-        accumulate(P, M, c, x.z, g.z, A, D); accumulate(P, M, c, x.w, g.w, A, D);
-      }
-    } else {
-      for (int i = lig; i < n; i += G) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
-    }
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (4 * (ch * G + lig) + j < n) accumulate(P, M, c, x[ch][j], g[ch][j], A, D);
 #pragma unroll
     for (int o = G >> 1; o > 0; o >>= 1) {
       A += __shfl_xor_sync(mask, A, o);
@@ -105,18 +120,18 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
     if (M.mag) D += (float)c.m;
   }
   const float ratio = D > 0.0f ? A / D : 0.0f;
-  if (P.vec4) {
-    const float4* x4 = reinterpret_cast<const float4*>(x_row);
-    const float4* g4 = reinterpret_cast<const float4*>(g_row);
-    float4* o4 = reinterpret_cast<float4*>(o_row);
-    for (int v = lig; 4 * v < n; v += G) {
-      float4 x = __ldg(x4 + v), g = __ldg(g4 + v), o;
-      o.x = finish(P, M, c, x.x, g.x, ratio); o.y = finish(P, M, c, x.y, g.y, ratio);
-      o.z = finish(P, M, c, x.z, g.z, ratio); o.w = finish(P, M, c, x.w, g.w, ratio);
-      o4[v] = o;
+#pragma unroll
+  for (int ch = 0; ch < CH; ++ch) {
+    const int v = ch * G + lig;
+    float o[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o[j] = finish(P, M, c, x[ch][j], g[ch][j], ratio);
+    if (P.vec4) {
+      if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o[0], o[1], o[2], o[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) if (4 * v + j < n) o_row[4 * v + j] = o[j];
     }
-  } else {
-    for (int i = lig; i < n; i += G) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
   }
 }
 
@@ -236,18 +251,21 @@ cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t 
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
   if (P.n <= 512) {
-    // lanes per row: one float4 (or 4 scalars) per lane and pass where possible
+    // lanes per row: one float4 per lane up to 128 elements, then 2 or 4 chunks per lane
     int G = 1;
     while (G < 32 && G * 4 < P.n) G <<= 1;
+    const int CH = (P.n + 4 * G - 1) / (4 * G);     // 1, 2, 3 or 4
     const long long rows_per_block = 8 * (32 / G);
     const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
+    if (CH > 2) { tk_vjp_state_group<32, 4><<<blocks, 256, 0, stream>>>(P); return cudaGetLastError(); }
+    if (CH == 2) { tk_vjp_state_group<32, 2><<<blocks, 256, 0, stream>>>(P); return cudaGetLastError(); }
     switch (G) {
-      case 1: tk_vjp_state_group<1><<<blocks, 256, 0, stream>>>(P); break;
-      case 2: tk_vjp_state_group<2><<<blocks, 256, 0, stream>>>(P); break;
-      case 4: tk_vjp_state_group<4><<<blocks, 256, 0, stream>>>(P); break;
-      case 8: tk_vjp_state_group<8><<<blocks, 256, 0, stream>>>(P); break;
-      case 16: tk_vjp_state_group<16><<<blocks, 256, 0, stream>>>(P); break;
-      default: tk_vjp_state_group<32><<<blocks, 256, 0, stream>>>(P); break;
+      case 1: tk_vjp_state_group<1, 1><<<blocks, 256, 0, stream>>>(P); break;
+      case 2: tk_vjp_state_group<2, 1><<<blocks, 256, 0, stream>>>(P); break;
+      case 4: tk_vjp_state_group<4, 1><<<blocks, 256, 0, stream>>>(P); break;
+      case 8: tk_vjp_state_group<8, 1><<<blocks, 256, 0, stream>>>(P); break;
+      case 16: tk_vjp_state_group<16, 1><<<blocks, 256, 0, stream>>>(P); break;
+      default: tk_vjp_state_group<32, 1><<<blocks, 256, 0, stream>>>(P); break;
     }
   } else {
     tk_vjp_state_cta<<<(unsigned)P.rows, 256, 0, stream>>>(P);
