@@ -11,6 +11,8 @@ int cta_padded_length(int n);
 // sub-warp row kernels for n <= 512 (tk_group.cu); key-only sort, results by value (tk_groupv.cu)
 cudaError_t launch_group(const Problem& P, cudaStream_t stream);
 cudaError_t launch_groupv(const Problem& P, cudaStream_t stream);
+// block-per-row kernel with a key-only sort and results by value (tk_ctav.cu)
+cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
 // exact forward pass without a sort (tk_thr.cu)
 cudaError_t launch_thr(const Problem& P, cudaStream_t stream);
 // alternating-projection solver path (tk_dykstra.cu)
@@ -31,7 +33,7 @@ constexpr int kMaxGroupN = 512;      // longest row a single warp holds in regis
 inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   // Without a permutation to return, short rows sort their keys only and place results by value.
   const bool needs_perm = P.perm_out != nullptr || P.sorted_out != nullptr || P.what == W_ARGSORT;
-  if (P.n <= 256 && !needs_perm) return launch_groupv(P, stream);
+  if (!needs_perm) return P.n <= 256 ? launch_groupv(P, stream) : launch_ctav(P, stream);
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
 }
 }  // namespace tk
