@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(256) long_digit_scan_kernel(uint32_t* hist, co
 // Stable scatter of one tile.  Elements are first ranked (warp by warp, in position order, so
 // equal digits keep their order), then the tile is reordered by digit in shared memory so that
 // the global writes are runs of consecutive addresses per digit.
-template <bool FIRST>
+template <bool FIRST, bool WITH_IDX>
 __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, const uint32_t* keys_in,
                                                            const int32_t* idx_in, uint32_t* keys_out,
                                                            int32_t* idx_out, const uint32_t* hist, int n,
@@ -183,7 +183,7 @@ __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, c
   __shared__ uint32_t tstart[RADIX];         // first tile-local position of every digit
   __shared__ uint32_t gbase[RADIX];          // first global position of this tile's run of every digit
   __shared__ uint32_t skey[TILE];
-  __shared__ int32_t sidx[TILE];
+  __shared__ int32_t sidx[WITH_IDX ? TILE : 1];   // indices travel only when a permutation is wanted
   const int tile = blockIdx.x;
   const long long row = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, c
       const uint32_t digit = (key[i] >> shift) & 0xFF;
       const uint32_t lp = tstart[digit] + cnt[warp][digit] + lrank[i];
       skey[lp] = key[i];
-      sidx[lp] = FIRST ? pos : idx_in[base + pos];
+      if (WITH_IDX) sidx[lp] = FIRST ? pos : idx_in[base + pos];
     }
   }
   __syncthreads();
@@ -250,7 +250,7 @@ __global__ void __launch_bounds__(TPB) long_scatter_kernel(const float* theta, c
     const uint32_t digit = (kk >> shift) & 0xFF;
     const uint32_t dst = gbase[digit] + ((uint32_t)j - tstart[digit]);
     keys_out[base + dst] = kk;
-    idx_out[base + dst] = sidx[j];
+    if (WITH_IDX) idx_out[base + dst] = sidx[j];
   }
 }
 
@@ -530,6 +530,35 @@ __global__ void __launch_bounds__(256) long_map_kernel(const Problem P, LongWs w
   P.out[base + idx] = y;
 }
 
+// y placed by value, in the original order: the class of an element follows from its key, gamma
+// and the block's width, so neither the permutation nor a scatter is needed.
+__global__ void __launch_bounds__(256) long_map_value_kernel(const Problem P, const tk_rowstate* state) {
+  const long long row = blockIdx.y;
+  const int n = P.n;
+  const Math M = make_math(P);
+  const tk_rowstate st = state[row];
+  const bool has_block = st.b > st.a;
+  const float wid = has_block ? M.width(st.pivot + st.offset) : 0.0f;
+  const long long base = row * (long long)n;
+  const int start = blockIdx.x * kLongTile;
+#pragma unroll 4
+  for (int j = 0; j < kLongTile / 256; ++j) {
+    const int i = start + j * 256 + threadIdx.x;
+    if (i < n) {
+      const float x = __ldg(P.theta + base + i);
+      const float key = sort_key(x, M.mag);
+      const float d = key - st.pivot;
+      int cls; float tt = 0.0f;
+      if (!has_block) cls = d >= 0.0f ? 2 : 0;
+      else { const float t = d - st.offset; tt = fminf(fmaxf(t, 0.0f), wid); cls = t >= wid ? 2 : (t > 0.0f ? 1 : 0); }
+      float y = cls == 2 ? (M.mag ? M.vtop(key) : 1.0f) : (cls == 1 ? M.rho(tt) : 0.0f);
+      if (M.mag) y = signbit(x) ? -y : y;
+      if (P.mode == TK_TOPK) y *= x;
+      P.out[base + i] = y;
+    }
+  }
+}
+
 LongWs carve(void* workspace, long long rows, int n, int tiles, size_t* total) {
   LongWs w{};
   size_t off = 0;
@@ -561,8 +590,8 @@ size_t long_workspace_bytes(long long rows, int n) {
   return total;
 }
 
-// Sorts every row; the result is in ws.keyB / ws.idxB.
-static cudaError_t long_sort(const Problem& P, const LongWs& ws, int tiles, cudaStream_t stream) {
+// Sorts every row; the result is in ws.keyB (and ws.idxB when the indices travel too).
+static cudaError_t long_sort(const Problem& P, const LongWs& ws, int tiles, bool with_idx, cudaStream_t stream) {
   const dim3 grid((unsigned)tiles, (unsigned)P.rows);
   const int mag = P.mode == TK_TOPKMAG;
   const uint32_t* kin = nullptr; const int32_t* iin = nullptr;
@@ -578,8 +607,13 @@ static cudaError_t long_sort(const Problem& P, const LongWs& ws, int tiles, cuda
     } else {
       long_scan_hist_kernel<<<(unsigned)P.rows, 1024, 0, stream>>>(ws.hist, tiles);
     }
-    if (pass == 0) long_scatter_kernel<true><<<grid, TPB, 0, stream>>>(P.theta, nullptr, nullptr, kout, iout, ws.hist, P.n, tiles, shift, mag);
-    else long_scatter_kernel<false><<<grid, TPB, 0, stream>>>(nullptr, kin, iin, kout, iout, ws.hist, P.n, tiles, shift, mag);
+    if (pass == 0) {
+      if (with_idx) long_scatter_kernel<true, true><<<grid, TPB, 0, stream>>>(P.theta, nullptr, nullptr, kout, iout, ws.hist, P.n, tiles, shift, mag);
+      else long_scatter_kernel<true, false><<<grid, TPB, 0, stream>>>(P.theta, nullptr, nullptr, kout, iout, ws.hist, P.n, tiles, shift, mag);
+    } else {
+      if (with_idx) long_scatter_kernel<false, true><<<grid, TPB, 0, stream>>>(nullptr, kin, iin, kout, iout, ws.hist, P.n, tiles, shift, mag);
+      else long_scatter_kernel<false, false><<<grid, TPB, 0, stream>>>(nullptr, kin, iin, kout, iout, ws.hist, P.n, tiles, shift, mag);
+    }
     kin = kout; iin = iout;
     if (kout == ws.keyA) { kout = ws.keyB; iout = ws.idxB; } else { kout = ws.keyA; iout = ws.idxA; }
   }
@@ -592,7 +626,9 @@ cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_ds
   const int tiles = (P.n + TILE - 1) / TILE;
   size_t total = 0;
   LongWs ws = carve(workspace, P.rows, P.n, tiles, &total);
-  cudaError_t e = long_sort(P, ws, tiles, stream);
+  // the indices ride along only when the caller asks for the permutation
+  const bool with_idx = P.perm_out != nullptr || P.what == W_ARGSORT;
+  cudaError_t e = long_sort(P, ws, tiles, with_idx, stream);
   if (e != cudaSuccess) return e;
   const long long el = P.rows * (long long)P.n;
   if (P.perm_out || P.sorted_out)
@@ -604,8 +640,12 @@ cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_ds
   long_prefix_kernel<<<grid, TPB, 0, stream>>>(P, ws, tiles);
   long_solve_kernel<<<(unsigned)P.rows, 1024, 0, stream>>>(P, ws, tiles, state);
   if (!skip_map) {
-    const dim3 mgrid((unsigned)((P.n + 255) / 256), (unsigned)P.rows);
-    long_map_kernel<<<mgrid, 256, 0, stream>>>(P, ws, state);
+    if (with_idx) {
+      const dim3 mgrid((unsigned)((P.n + 255) / 256), (unsigned)P.rows);
+      long_map_kernel<<<mgrid, 256, 0, stream>>>(P, ws, state);      // un-permute: out[sigma_i] = y_i
+    } else {
+      long_map_value_kernel<<<grid, 256, 0, stream>>>(P, state);
+    }
   }
   return cudaGetLastError();
 }

@@ -99,12 +99,14 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
     assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
     # the call without a permutation output takes its own path for short rows (keys sorted alone,
     # results placed by value): same tolerance against the oracle, same pooled blocks
-    if ws_bytes == 0 and sorts:
+    if sorts:
         out2 = torch.full_like(out, float("nan"))
         state2 = tk.new_state(rows)
-        tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out2, state_out=state2, status_out=status)
-        out3 = torch.full_like(out, float("nan"))
-        tk.tk_fwd(th, rows, n, k, p, lam, mode, out3)
+        tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out2, state_out=state2, status_out=status, workspace=ws)
+        out3 = out2
+        if ws_bytes == 0:
+            out3 = torch.full_like(out, float("nan"))
+            tk.tk_fwd(th, rows, n, k, p, lam, mode, out3)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
         g2 = out2.cpu().numpy()
