@@ -33,7 +33,7 @@ constexpr int kMaxGroupN = 512;      // longest row a single warp holds in regis
 inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   // Without a permutation to return, short rows sort their keys only and place results by value.
   const bool needs_perm = P.perm_out != nullptr || P.sorted_out != nullptr || P.what == W_ARGSORT;
-  if (!needs_perm) return P.n <= 256 ? launch_groupv(P, stream) : launch_ctav(P, stream);
+  if (!needs_perm) return P.n <= 512 ? launch_groupv(P, stream) : launch_ctav(P, stream);
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
 }
 }  // namespace tk

@@ -1,4 +1,4 @@
-// tk_groupv.cu -- short rows (n <= 256), the default forward pass and VJP: sort of the KEYS only.
+// tk_groupv.cu -- short rows (n <= 512), the default forward pass and VJP: sort of the KEYS only.
 //
 // Given gamma and the edges of the pooled block, the output (and the VJP) of every element is a
 // function of its own key: key >= gamma + width -> capped, gamma < key < gamma + width -> pooled,
@@ -9,7 +9,8 @@
 // loaded them.  No index, no scatter, no staging buffer.  Equal keys get equal results, so the
 // stable order among ties is immaterial here; tk_argsort and perm_out use the (key, index) sort.
 //
-// Same G lanes x 8 elements layout, same solve (Sec. 5; App. A.6) as tk_group.cu.
+// Same layout (G lanes x 8 elements, or one warp x 16 elements for 256 < n <= 512) and the same
+// solve (Sec. 5; App. A.6) as tk_group.cu.
 #include "tk_common.cuh"
 #include "tk_group_sort.cuh"
 
@@ -35,40 +36,67 @@ __device__ __forceinline__ void merge8f(float (&r)[8]) {      // bitonic -> desc
   cef(r[0], r[2]); cef(r[1], r[3]); cef(r[4], r[6]); cef(r[5], r[7]);
   cef(r[0], r[1]); cef(r[2], r[3]); cef(r[4], r[5]); cef(r[6], r[7]);
 }
-template <int G>
-__device__ __forceinline__ void group_sort_keys(float (&r)[8], int lig, unsigned mask) {
-  sort8f(r);
+template <int E>
+__device__ __forceinline__ void lane_sort_f(float (&r)[E]);
+template <>
+__device__ __forceinline__ void lane_sort_f<8>(float (&r)[8]) { sort8f(r); }
+template <int E>
+__device__ __forceinline__ void lane_merge_f(float (&r)[E]) {   // bitonic -> descending
+#pragma unroll
+  for (int stride = E >> 1; stride > 0; stride >>= 1) {
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      const int j = i ^ stride;
+      if (j > i) cef(r[i], r[j]);
+    }
+  }
+}
+template <>
+__device__ __forceinline__ void lane_sort_f<16>(float (&r)[16]) {
+  float hi[8], lo[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { hi[i] = r[i]; lo[i] = r[i + 8]; }
+  sort8f(hi); sort8f(lo);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) cef(hi[i], lo[7 - i]);      // element against its mirror: two bitonic halves
+  merge8f(hi); merge8f(lo);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) { r[i] = hi[i]; r[i + 8] = lo[i]; }
+}
+
+template <int G, int E>
+__device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned mask) {
+  lane_sort_f<E>(r);
 #pragma unroll
   for (int size = 2; size <= G; size <<= 1) {
     {
       const bool keepmax = (lig & (size >> 1)) == 0;
-      float o[8];
+      float o[E];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) o[i] = __shfl_xor_sync(mask, r[7 - i], size - 1);
+      for (int i = 0; i < E; ++i) o[i] = __shfl_xor_sync(mask, r[E - 1 - i], size - 1);
 #pragma unroll
-      for (int i = 0; i < 8; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
+      for (int i = 0; i < E; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
     }
 #pragma unroll
     for (int st = size >> 2; st >= 1; st >>= 1) {
       const bool keepmax = (lig & st) == 0;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < E; ++i) {
         const float o = __shfl_xor_sync(mask, r[i], st);
         r[i] = keepmax ? fmaxf(r[i], o) : fminf(r[i], o);
       }
     }
-    merge8f(r);
+    lane_merge_f<E>(r);
   }
 }
 
-template <int G>
-__global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
-  constexpr int EPL = 8;
+template <int G, int EPL>
+__global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const Problem P) {
   constexpr int N = G * EPL;
   constexpr int GROUPS = 128 / G;
   constexpr int STRIDE = N + N / EPL + 1;
   __shared__ float sm[GROUPS][4][STRIDE];     // sorted keys, prefix sums of d, d^2, d^3
-  auto pad8 = [](int i) -> int { return i + (i >> 3); };
+  auto pad8 = [](int i) -> int { return i + i / EPL; };
 
   const int tid = threadIdx.x;
   const int grp = tid / G, lig = tid % G;
@@ -89,7 +117,7 @@ __global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
   float x[EPL], s[EPL];
   bool bad = false;
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
+  for (int h = 0; h < EPL / 4; ++h) {
     const int base = EPL * lig + 4 * h;
     if (P.vec4) {
       float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -106,7 +134,7 @@ __global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
     if (in && !isfinite(x[i])) bad = true;
     s[i] = in ? sort_key(x[i], mag) : -INFINITY;        // slots past the row sort last
   }
-  group_sort_keys<G>(s, lig, mask);           // lane `lig` holds sorted ranks [8 lig, 8 lig + 8)
+  group_sort_keys<G, EPL>(s, lig, mask);      // lane `lig` holds sorted ranks [EPL lig, EPL lig + EPL)
   int flags = bad ? TK_FLAG_NONFINITE : 0;
 
 #pragma unroll
@@ -252,7 +280,7 @@ __global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
     const float* g_row = P.gout + row * (long long)n;
     float g[EPL];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
+    for (int h = 0; h < EPL / 4; ++h) {
       const int base = EPL * lig + 4 * h;
       if (P.vec4) {
         float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -296,7 +324,7 @@ __global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
   }
   float* o_row = P.out + row * (long long)n;
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
+  for (int h = 0; h < EPL / 4; ++h) {
     const int base = EPL * lig + 4 * h;
     if (P.vec4) {
       if (base < n) reinterpret_cast<float4*>(o_row)[base >> 2] = make_float4(o[4 * h], o[4 * h + 1], o[4 * h + 2], o[4 * h + 3]);
@@ -310,21 +338,26 @@ __global__ void __launch_bounds__(128, 8) tk_groupv_kernel(const Problem P) {
 
 }  // namespace
 
-// Forward pass or recomputing VJP for rows of up to 256 elements when no permutation is asked for.
+// Forward pass or recomputing VJP for rows of up to 512 elements when no permutation is asked for.
 cudaError_t launch_groupv(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
+  if (P.n > 256) {                           // one warp per row, 16 elements per lane
+    P.N = 512;
+    tk_groupv_kernel<32, 16><<<(unsigned)((P.rows + 3) / 4), 128, 0, stream>>>(P);
+    return cudaGetLastError();
+  }
   int G = 1;
   while (G * 8 < P.n) G <<= 1;
   P.N = G * 8;
   const long long groups = 128 / G;
   const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
   switch (G) {
-    case 1: tk_groupv_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
-    case 2: tk_groupv_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
-    case 4: tk_groupv_kernel<4><<<blocks, 128, 0, stream>>>(P); break;
-    case 8: tk_groupv_kernel<8><<<blocks, 128, 0, stream>>>(P); break;
-    case 16: tk_groupv_kernel<16><<<blocks, 128, 0, stream>>>(P); break;
-    default: tk_groupv_kernel<32><<<blocks, 128, 0, stream>>>(P); break;
+    case 1: tk_groupv_kernel<1, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 2: tk_groupv_kernel<2, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 4: tk_groupv_kernel<4, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 8: tk_groupv_kernel<8, 8><<<blocks, 128, 0, stream>>>(P); break;
+    case 16: tk_groupv_kernel<16, 8><<<blocks, 128, 0, stream>>>(P); break;
+    default: tk_groupv_kernel<32, 8><<<blocks, 128, 0, stream>>>(P); break;
   }
   return cudaGetLastError();
 }
