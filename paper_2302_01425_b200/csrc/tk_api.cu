@@ -8,8 +8,10 @@ namespace tk {
 // on-chip row kernels (tk_cta.cu)
 cudaError_t launch_cta(const Problem& P, cudaStream_t stream);
 int cta_padded_length(int n);
-// sub-warp row kernels for n <= 512 (tk_group.cu); key-only sort, results by value (tk_groupv.cu)
+// sub-warp row kernels for n <= 512 with the permutation (tk_group.cu); key-only sort and results
+// by value: short rows (tk_rows.cu), up to 512 (tk_groupv.cu)
 cudaError_t launch_group(const Problem& P, cudaStream_t stream);
+cudaError_t launch_rows(const Problem& P, cudaStream_t stream);
 cudaError_t launch_groupv(const Problem& P, cudaStream_t stream);
 // block-per-row kernel with a key-only sort and results by value (tk_ctav.cu)
 cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
@@ -29,11 +31,15 @@ void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
 constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers
+constexpr int kMaxWalkN = 256;       // longest row whose solve is one thread's walk (tk_rows.cu)
 
 inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   // Without a permutation to return, short rows sort their keys only and place results by value.
   const bool needs_perm = P.perm_out != nullptr || P.sorted_out != nullptr || P.what == W_ARGSORT;
-  if (!needs_perm) return P.n <= 512 ? launch_groupv(P, stream) : launch_ctav(P, stream);
+  if (!needs_perm) {
+    if (P.n <= kMaxWalkN) return launch_rows(P, stream);
+    return P.n <= kMaxGroupN ? launch_groupv(P, stream) : launch_ctav(P, stream);
+  }
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
 }
 }  // namespace tk

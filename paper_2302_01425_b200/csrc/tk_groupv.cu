@@ -13,82 +13,11 @@
 // solve (Sec. 5; App. A.6) as tk_group.cu.
 #include "tk_common.cuh"
 #include "tk_group_sort.cuh"
+#include "tk_key_sort.cuh"
 
 namespace tk {
 
 namespace {
-
-__device__ __forceinline__ void cef(float& a, float& b) {   // a >= b after
-  const float hi = fmaxf(a, b), lo = fminf(a, b);
-  a = hi; b = lo;
-}
-__device__ __forceinline__ void sort8f(float (&r)[8]) {       // the 19-comparator network, descending
-  cef(r[0], r[1]); cef(r[2], r[3]); cef(r[4], r[5]); cef(r[6], r[7]);
-  cef(r[0], r[2]); cef(r[1], r[3]); cef(r[4], r[6]); cef(r[5], r[7]);
-  cef(r[1], r[2]); cef(r[5], r[6]); cef(r[0], r[4]); cef(r[3], r[7]);
-  cef(r[1], r[5]); cef(r[2], r[6]);
-  cef(r[1], r[4]); cef(r[3], r[6]);
-  cef(r[2], r[4]); cef(r[3], r[5]);
-  cef(r[3], r[4]);
-}
-__device__ __forceinline__ void merge8f(float (&r)[8]) {      // bitonic -> descending
-  cef(r[0], r[4]); cef(r[1], r[5]); cef(r[2], r[6]); cef(r[3], r[7]);
-  cef(r[0], r[2]); cef(r[1], r[3]); cef(r[4], r[6]); cef(r[5], r[7]);
-  cef(r[0], r[1]); cef(r[2], r[3]); cef(r[4], r[5]); cef(r[6], r[7]);
-}
-template <int E>
-__device__ __forceinline__ void lane_sort_f(float (&r)[E]);
-template <>
-__device__ __forceinline__ void lane_sort_f<8>(float (&r)[8]) { sort8f(r); }
-template <int E>
-__device__ __forceinline__ void lane_merge_f(float (&r)[E]) {   // bitonic -> descending
-#pragma unroll
-  for (int stride = E >> 1; stride > 0; stride >>= 1) {
-#pragma unroll
-    for (int i = 0; i < E; ++i) {
-      const int j = i ^ stride;
-      if (j > i) cef(r[i], r[j]);
-    }
-  }
-}
-template <>
-__device__ __forceinline__ void lane_sort_f<16>(float (&r)[16]) {
-  float hi[8], lo[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) { hi[i] = r[i]; lo[i] = r[i + 8]; }
-  sort8f(hi); sort8f(lo);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) cef(hi[i], lo[7 - i]);      // element against its mirror: two bitonic halves
-  merge8f(hi); merge8f(lo);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) { r[i] = hi[i]; r[i + 8] = lo[i]; }
-}
-
-template <int G, int E>
-__device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned mask) {
-  lane_sort_f<E>(r);
-#pragma unroll
-  for (int size = 2; size <= G; size <<= 1) {
-    {
-      const bool keepmax = (lig & (size >> 1)) == 0;
-      float o[E];
-#pragma unroll
-      for (int i = 0; i < E; ++i) o[i] = __shfl_xor_sync(mask, r[E - 1 - i], size - 1);
-#pragma unroll
-      for (int i = 0; i < E; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
-    }
-#pragma unroll
-    for (int st = size >> 2; st >= 1; st >>= 1) {
-      const bool keepmax = (lig & st) == 0;
-#pragma unroll
-      for (int i = 0; i < E; ++i) {
-        const float o = __shfl_xor_sync(mask, r[i], st);
-        r[i] = keepmax ? fmaxf(r[i], o) : fminf(r[i], o);
-      }
-    }
-    lane_merge_f<E>(r);
-  }
-}
 
 template <int G, int EPL>
 __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const Problem P) {
@@ -338,7 +267,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const 
 
 }  // namespace
 
-// Forward pass or recomputing VJP for rows of up to 512 elements when no permutation is asked for.
+// Forward pass or recomputing VJP for rows of 129..512 elements when no permutation is asked for.
 cudaError_t launch_groupv(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
   if (P.n > 256) {                           // one warp per row, 16 elements per lane
@@ -346,19 +275,8 @@ cudaError_t launch_groupv(const Problem& P0, cudaStream_t stream) {
     tk_groupv_kernel<32, 16><<<(unsigned)((P.rows + 3) / 4), 128, 0, stream>>>(P);
     return cudaGetLastError();
   }
-  int G = 1;
-  while (G * 8 < P.n) G <<= 1;
-  P.N = G * 8;
-  const long long groups = 128 / G;
-  const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
-  switch (G) {
-    case 1: tk_groupv_kernel<1, 8><<<blocks, 128, 0, stream>>>(P); break;
-    case 2: tk_groupv_kernel<2, 8><<<blocks, 128, 0, stream>>>(P); break;
-    case 4: tk_groupv_kernel<4, 8><<<blocks, 128, 0, stream>>>(P); break;
-    case 8: tk_groupv_kernel<8, 8><<<blocks, 128, 0, stream>>>(P); break;
-    case 16: tk_groupv_kernel<16, 8><<<blocks, 128, 0, stream>>>(P); break;
-    default: tk_groupv_kernel<32, 8><<<blocks, 128, 0, stream>>>(P); break;
-  }
+  P.N = 256;                                 // 128 < n <= 256: one warp per row, 8 elements per lane
+  tk_groupv_kernel<32, 8><<<(unsigned)((P.rows + 3) / 4), 128, 0, stream>>>(P);
   return cudaGetLastError();
 }
 
