@@ -16,7 +16,7 @@ LIB = os.path.join(_PKG, "libtk.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared",
+    "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared", "--threads", "0",
 ]
 
 

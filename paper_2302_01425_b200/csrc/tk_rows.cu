@@ -1,6 +1,6 @@
 // tk_rows.cu -- rows of up to 256 elements, the default forward pass and VJP.
 //
-// Every warp works alone on 32 rows (16 when n > 64, 8 when n > 128), in three phases:
+// Every warp works alone on up to 32 rows (16 when n > 64, 8 when n > 128), in three phases:
 //   1. in batches of 32/G rows (G lanes x 8 elements per row): load, sort the 32-bit KEYS by the
 //      shuffle network, leave the sorted row in the warp's shared memory;
 //   2. lane r solves row r: the isotonic problem of Sec. 5 has at most one pooled block [a0, b0)
@@ -167,19 +167,21 @@ __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, co
 
 constexpr int kRowsThreads = 128;
 
-template <int G>
+// B batches of 32/G rows per warp.  The most batches (32 rows per warp, 16 for n > 64, 8 for
+// n > 128) cost the fewest instructions per row; fewer batches give a small problem enough warps
+// to fill the machine.
+template <int G, int B>
 struct RowsGeom {
   static constexpr int N = 8 * G;                          // padded row length
   static constexpr int RPB = 32 / G;                       // rows per batch
-  static constexpr int R = (G <= 8) ? 32 : 256 / G;        // rows per warp
-  static constexpr int BATCHES = R / RPB;
+  static constexpr int R = RPB * B;                        // rows per warp
   static constexpr int STRIDE = (N + G - 1) | 1;           // odd: lane r walking row r meets no bank conflict
 };
 
-template <int G, bool Q4, bool MAG>
+template <int G, int B, bool Q4, bool MAG>
 __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem P) {
-  constexpr int RPB = RowsGeom<G>::RPB, R = RowsGeom<G>::R, BATCHES = RowsGeom<G>::BATCHES;
-  constexpr int STRIDE = RowsGeom<G>::STRIDE;
+  constexpr int RPB = RowsGeom<G, B>::RPB, R = RowsGeom<G, B>::R, BATCHES = B;
+  constexpr int STRIDE = RowsGeom<G, B>::STRIDE;
   constexpr int WARPS = kRowsThreads / 32;
   __shared__ float sm[WARPS][R][STRIDE];
 
@@ -326,19 +328,30 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
   if (flags && P.status) atomicOr(P.status, flags);
 }
 
-template <int G>
-cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
-  const long long per_block = (long long)(kRowsThreads / 32) * RowsGeom<G>::R;
+template <int G, int B>
+cudaError_t launch_rows_gb(const Problem& P, cudaStream_t stream) {
+  const long long per_block = (long long)(kRowsThreads / 32) * RowsGeom<G, B>::R;
   const unsigned blocks = (unsigned)((P.rows + per_block - 1) / per_block);
   const bool mag = P.mode == TK_TOPKMAG;
   if (P.q4) {
-    if (mag) tk_rows_kernel<G, true, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, true, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, B, true, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, B, true, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   } else {
-    if (mag) tk_rows_kernel<G, false, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, false, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, B, false, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, B, false, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   }
   return cudaGetLastError();
+}
+
+constexpr long long kWarpsToFill = 148 * 24;   // warps below which a launch leaves SMs short of work
+
+// The most batches per warp that still leave kWarpsToFill warps, out of {1, 2, BMAX}.
+template <int G, int BMAX>
+cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
+  constexpr int RPB = 32 / G;
+  if (BMAX > 2 && P.rows / (RPB * BMAX) >= kWarpsToFill) return launch_rows_gb<G, BMAX>(P, stream);
+  if (BMAX >= 2 && P.rows / (RPB * 2) >= kWarpsToFill) return launch_rows_gb<G, (BMAX >= 2 ? 2 : 1)>(P, stream);
+  return launch_rows_gb<G, 1>(P, stream);
 }
 
 }  // namespace
@@ -350,12 +363,12 @@ cudaError_t launch_rows(const Problem& P0, cudaStream_t stream) {
   while (G * 8 < P.n) G <<= 1;
   P.N = G * 8;
   switch (G) {
-    case 1: return launch_rows_g<1>(P, stream);
-    case 2: return launch_rows_g<2>(P, stream);
-    case 4: return launch_rows_g<4>(P, stream);
-    case 8: return launch_rows_g<8>(P, stream);
-    case 16: return launch_rows_g<16>(P, stream);
-    default: return launch_rows_g<32>(P, stream);
+    case 1: return launch_rows_g<1, 1>(P, stream);
+    case 2: return launch_rows_g<2, 2>(P, stream);
+    case 4: return launch_rows_g<4, 4>(P, stream);
+    case 8: return launch_rows_g<8, 8>(P, stream);
+    case 16: return launch_rows_g<16, 8>(P, stream);
+    default: return launch_rows_g<32, 8>(P, stream);
   }
 }
 
