@@ -153,6 +153,31 @@ __device__ __forceinline__ Math make_math(const Problem& P) {
   return m;
 }
 
+// Every later use of a row's solution classifies an element by its key alone:
+// t = (key - pivot) - u, capped if t >= width(pivot + u), pooled if t > 0, else zero.  The solved
+// u is rounded to fp32, and an element that sits a few 1e-9 inside the cap (a pooled rank whose
+// rho is 1 - 1e-7) can then read as capped: harmless for the forward value, but the VJP of a
+// capped element is a different formula.  This moves u by single ulps until the block's own edge
+// ranks read as what the solve decided: a0-1 capped, a0 and b0-1 pooled, b0 zero.  A conflict
+// (two edge keys closer than the arithmetic resolves) leaves u as it is.  key_at(i): sorted key of
+// rank i, 0 <= i < n.
+template <class KeyAt>
+__device__ __forceinline__ float settle_offset(const Math& M, float piv, float u, int a0, int b0, int n,
+                                               KeyAt key_at) {
+  const float k_am1 = a0 > 0 ? key_at(a0 - 1) : INFINITY;
+  const float k_a = key_at(a0), k_bm1 = key_at(b0 - 1);
+  const float k_b = b0 < n ? key_at(b0) : -INFINITY;
+#pragma unroll 1
+  for (int it = 0; it < 8; ++it) {
+    const float wid = M.width(piv + u);
+    const bool up = ((k_a - piv) - u >= wid) || ((k_b - piv) - u > 0.0f);
+    const bool down = !((k_bm1 - piv) - u > 0.0f) || ((k_am1 - piv) - u < wid);
+    if (up == down) break;
+    u = nextafterf(u, up ? INFINITY : -INFINITY);
+  }
+  return u;
+}
+
 // Root u of the pooled block's stationarity equation, from the block's power
 // sums D_m = sum_B d_i^m (cnt members, m of them with w = 1), pivot c:
 //   q = 2, phi = x   : sum (d_i - u)/lam = m            -> closed form

@@ -208,7 +208,7 @@ tk_cta_kernel(const Problem P) {
       double u_left = mag ? (double)W_lo : D1 / cnt - (double)P.lam * cbrt(m / cnt);
       int nc = 0;
       double uu = solve_block_u(M.q4, mag, (double)P.lam, (double)piv, cnt, m, D1, D2, D3, u_left, &nc);
-      sol.u = (float)uu;
+      sol.u = settle_offset(M, piv, (float)uu, a0, b0, n, [&](int i) -> float { return un_key(keys[pad(i)]); });
       if (nc) atomicOr(&row_flags, TK_FLAG_NOT_CONVERGED);
     }
     __syncthreads();

@@ -296,7 +296,7 @@ tk_ctav_kernel(const Problem P) {
       double u_left = mag ? (double)W_lo : D1 / cnt - (double)P.lam * cbrt(m / cnt);
       int nc = 0;
       double uu = solve_block_u(M.q4, mag, (double)P.lam, (double)piv, cnt, m, D1, D2, D3, u_left, &nc);
-      sol.u = (float)uu;
+      sol.u = settle_offset(M, piv, (float)uu, a0, b0, n, [&](int i) -> float { return keys[pad(i)]; });
       if (nc) atomicOr(&row_flags, TK_FLAG_NOT_CONVERGED);
     }
     __syncthreads();
@@ -361,6 +361,20 @@ tk_ctav_kernel(const Problem P) {
     float Db = block_sum<float>(D, reinterpret_cast<float*>(redd));
     if (mag) Db += (float)(k - a0);
     const float ratio = (Db > 0.0f) ? Ab / Db : 0.0f;
+    // second pass: residuals about the fp32 mean (one fma each, no cancellation) restore what the
+    // division rounded away; rho' can be 3/lambda, and an ulp of the mean times that shows
+    float A2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+      float tt;
+      if (((valid >> i) & 1u) && classify(sort_key(x[i], mag), tt) == 1) {
+        const float chi = mag ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
+        A2 += M.drho(tt) * fmaf(chi, g[i], -ratio);
+      }
+    }
+    float A2b = block_sum<float>(A2, reinterpret_cast<float*>(redd));
+    if (mag) A2b -= (float)(k - a0) * ratio;
+    const float delta = (Db > 0.0f) ? A2b / Db : 0.0f;
 #pragma unroll
     for (int i = 0; i < E; ++i) {
       float tt;
@@ -369,7 +383,7 @@ tk_ctav_kernel(const Problem P) {
       const float sgn = (mag && signbit(x[i])) ? -1.0f : 1.0f;
       const float chi = mag ? sgn : (P.mode == TK_TOPK ? x[i] : 1.0f);
       float v = 0.0f;
-      if (cls == 1) v = M.drho(tt) * (chi * g[i] - ratio);
+      if (cls == 1) v = M.drho(tt) * (fmaf(chi, g[i], -ratio) - delta);
       else if (cls == 2 && mag) v = chi * g[i] * M.top_slope(key);
       v *= sgn;
       if (P.mode == TK_TOPK) v += g[i] * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));

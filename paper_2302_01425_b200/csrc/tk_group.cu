@@ -171,6 +171,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const P
     const double u_left = mag ? (double)W_lo : D1 / cnt - (double)P.lam * (double)cbrtf((float)(m / cnt)) * 1.000001;
     int nc = 0;
     u = (float)solve_block_u(M.q4, mag, (double)P.lam, (double)piv, cnt, m, D1, D2, D3, u_left, &nc);
+    u = settle_offset(M, piv, u, a0, b0, n, [&](int i) -> float { return sk[pad8(i)]; });
     if (nc) flags |= TK_FLAG_NOT_CONVERGED;
   }
   if (P.state_out && lig == 0) {

@@ -174,6 +174,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const 
     const double u_left = mag ? (double)W_lo : D1 / cnt - (double)P.lam * (double)cbrtf((float)(m / cnt)) * 1.000001;
     int nc = 0;
     u = (float)solve_block_u(M.q4, mag, (double)P.lam, (double)piv, cnt, m, D1, D2, D3, u_left, &nc);
+    u = settle_offset(M, piv, u, a0, b0, n, [&](int i) -> float { return sk[pad8(i)]; });
     if (nc) flags |= TK_FLAG_NOT_CONVERGED;
   }
   if (P.state_out && lig == 0) {
@@ -236,6 +237,23 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const 
       if (mag) D += (float)(k - a0);
     }
     const float ratio = D > 0.0f ? A / D : 0.0f;
+    // second pass: residuals about the fp32 mean (one fma each, no cancellation) restore what the
+    // division rounded away; rho' can be 3/lambda, and an ulp of the mean times that shows
+    float delta = 0.0f;
+    if (has_block) {
+      float A2 = 0.f;
+#pragma unroll
+      for (int i = 0; i < EPL; ++i) {
+        float tt;
+        if (EPL * lig + i < n && classify(sort_key(x[i], mag), tt) == 1) {
+          const float chi = mag ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
+          A2 += M.drho(tt) * fmaf(chi, g[i], -ratio);
+        }
+      }
+      A2 = group_sum<G, float>(A2, mask);
+      if (mag) A2 -= (float)(k - a0) * ratio;
+      delta = D > 0.0f ? A2 / D : 0.0f;
+    }
 #pragma unroll
     for (int i = 0; i < EPL; ++i) {
       float tt;
@@ -244,7 +262,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 4) tk_groupv_kernel(const 
       const float sgn = (mag && signbit(x[i])) ? -1.0f : 1.0f;
       const float chi = mag ? sgn : (P.mode == TK_TOPK ? x[i] : 1.0f);
       float v = 0.0f;
-      if (cls == 1) v = M.drho(tt) * (chi * g[i] - ratio);
+      if (cls == 1) v = M.drho(tt) * (fmaf(chi, g[i], -ratio) - delta);
       else if (cls == 2 && mag) v = chi * g[i] * M.top_slope(key);
       v *= sgn;
       if (P.mode == TK_TOPK) v += g[i] * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));

@@ -492,6 +492,7 @@ __global__ void __launch_bounds__(1024) long_solve_kernel(const Problem P, LongW
       const double u_left = mag ? (double)S.W_lo : D1 / cnt - (double)P.lam * cbrt(m / cnt);
       int nc = 0;
       sh_u = (float)solve_block_u(M.q4, mag, (double)P.lam, (double)piv, cnt, m, D1, D2, D3, u_left, &nc);
+      sh_u = settle_offset(M, piv, sh_u, a0, b0, n, sval);
       if (nc && P.status) atomicOr(P.status, TK_FLAG_NOT_CONVERGED);
     }
     __syncthreads();
@@ -656,7 +657,8 @@ tk_rowstate* long_workspace_state(void* workspace, long long rows, int n) {
   return carve(workspace, rows, n, tiles, &total).state;
 }
 
-// rows * tiles * 8 bytes of scratch for the VJP's per-tile partial sums (dead after the solve)
+// rows * tiles * 16 bytes of scratch for the VJP's per-tile partial sums (the 24 bytes per tile of
+// the solve's tile totals, dead by then)
 void* long_workspace_partials(void* workspace, long long rows, int n) {
   const int tiles = (n + TILE - 1) / TILE;
   size_t total = 0;

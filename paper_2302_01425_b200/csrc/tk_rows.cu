@@ -161,6 +161,7 @@ __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, co
       }
     }
     u = block_value<Q4, MAG>(P.lam, P.lam3, piv, cnt, m, mu, M2, M3);
+    u = settle_offset(M, piv, u, a0, b0, n, key);
   }
   R.piv = piv; R.u = u; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = has_block ? 1 : 0;
 }
@@ -298,6 +299,20 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
       D = group_sum<G, float>(D, mask);
       if (MAG && has_block) D += (float)(k - a0);
       const float ratio = D > 0.0f ? A / D : 0.0f;
+      // second pass: residuals about the fp32 mean (one fma each, no cancellation) restore what
+      // the division rounded away; rho' can be 3/lambda, and an ulp of the mean times that shows
+      float A2 = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        float tt;
+        if (has_block && 8 * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
+          const float chi = MAG ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
+          A2 += M.drho(tt) * fmaf(chi, g[i], -ratio);
+        }
+      }
+      A2 = group_sum<G, float>(A2, mask);
+      if (MAG && has_block) A2 -= (float)(k - a0) * ratio;
+      const float delta = D > 0.0f ? A2 / D : 0.0f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         float tt;
@@ -306,7 +321,7 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
         const float sgn = (MAG && signbit(x[i])) ? -1.0f : 1.0f;
         const float chi = MAG ? sgn : (P.mode == TK_TOPK ? x[i] : 1.0f);
         float v = 0.0f;
-        if (cls == 1) v = M.drho(tt) * (chi * g[i] - ratio);
+        if (cls == 1) v = M.drho(tt) * (fmaf(chi, g[i], -ratio) - delta);
         else if (cls == 2 && MAG) v = chi * g[i] * M.top_slope(key);
         v *= sgn;
         if (P.mode == TK_TOPK) v += g[i] * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));

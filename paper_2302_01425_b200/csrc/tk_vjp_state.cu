@@ -51,15 +51,45 @@ __device__ __forceinline__ void accumulate(const Problem& P, const Math& M, cons
   }
 }
 
+// The mean A/D is needed to a relative accuracy of its DISTANCE from chi g, not of itself: rho' can
+// be 3/lambda, and one ulp of A/D times that is above 1e-5.  Two ways to get it:
+//  * rows held in registers: a second pass sums the residuals rho' (chi g - r0) about the fp32 mean
+//    r0 of the first pass; each residual is one fma (no cancellation), and the correction
+//    delta = (sum - m r0)/D restores what the division rounded away;
+//  * rows streamed from memory: A and D are accumulated in fp64 (products of floats are exact
+//    there), the mean is split into r0 = fl(mean) and delta = mean - r0.
+// Either way the result is rho' ((chi g - r0) - delta).
+__device__ __forceinline__ void accumulate_residual(const Problem& P, const Math& M, const RowCtx& c, float x,
+                                                    float g, float r0, float& A2) {
+  float tt;
+  float key = sort_key(x, M.mag);
+  if (classify(c, key, tt) == 1) {
+    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
+    A2 += M.drho(tt) * fmaf(chi, g, -r0);
+  }
+}
+
+__device__ __forceinline__ void accumulate_f64(const Problem& P, const Math& M, const RowCtx& c, float x,
+                                               float g, double& A, double& D) {
+  float tt;
+  float key = sort_key(x, M.mag);
+  if (classify(c, key, tt) == 1) {
+    double dr = (double)M.drho(tt);
+    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
+    D += dr;
+    A += dr * ((double)chi * (double)g);
+  }
+}
+
 __device__ __forceinline__ float finish(const Problem& P, const Math& M, const RowCtx& c, float x,
-                                        float g, float ratio) {
+                                        float g, float ratio, float delta) {
   float tt;
   float key = sort_key(x, M.mag);
   int cls = classify(c, key, tt);
   float sgn = (M.mag && signbit(x)) ? -1.0f : 1.0f;
   float chi = M.mag ? sgn : (P.mode == TK_TOPK ? x : 1.0f);
   float o = 0.0f;
-  if (cls == 1) o = M.drho(tt) * (chi * g - ratio);
+  if (cls == 1) o = M.drho(tt) * (fmaf(chi, g, -ratio) - delta);
   else if (cls == 2 && M.mag) o = chi * g * M.top_slope(key);
   o *= sgn;
   if (P.mode == TK_TOPK) {
@@ -120,12 +150,25 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
     if (M.mag) D += (float)c.m;
   }
   const float ratio = D > 0.0f ? A / D : 0.0f;
+  float delta = 0.0f;
+  if (c.has_block) {
+    float A2 = 0.f;
+#pragma unroll
+    for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (4 * (ch * G + lig) + j < n) accumulate_residual(P, M, c, x[ch][j], g[ch][j], ratio, A2);
+#pragma unroll
+    for (int o = G >> 1; o > 0; o >>= 1) A2 += __shfl_xor_sync(mask, A2, o);
+    if (M.mag) A2 -= (float)c.m * ratio;
+    delta = D > 0.0f ? A2 / D : 0.0f;
+  }
 #pragma unroll
   for (int ch = 0; ch < CH; ++ch) {
     const int v = ch * G + lig;
     float o[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) o[j] = finish(P, M, c, x[ch][j], g[ch][j], ratio);
+    for (int j = 0; j < 4; ++j) o[j] = finish(P, M, c, x[ch][j], g[ch][j], ratio, delta);
     if (P.vec4) {
       if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o[0], o[1], o[2], o[3]);
     } else {
@@ -137,7 +180,7 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
 
 // one thread block per row
 __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
-  __shared__ float red[2][8];
+  __shared__ double red[2][8];
   const Math M = make_math(P);
   const int t = threadIdx.x, T = blockDim.x, lane = t & 31, warp = t >> 5;
   const long long row = blockIdx.x;
@@ -146,51 +189,52 @@ __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
   const float* x_row = P.theta + row * (long long)n;
   const float* g_row = P.gout + row * (long long)n;
   float* o_row = P.out + row * (long long)n;
-  float A = 0.f, D = 0.f;
+  double A = 0.0, D = 0.0;
   if (c.has_block) {           // uniform per row
     if (P.vec4) {
       const float4* x4 = reinterpret_cast<const float4*>(x_row);
       const float4* g4 = reinterpret_cast<const float4*>(g_row);
       for (int v = t; 4 * v < n; v += T) {
         float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
-        accumulate(P, M, c, x.x, g.x, A, D); accumulate(P, M, c, x.y, g.y, A, D);
-        accumulate(P, M, c, x.z, g.z, A, D); accumulate(P, M, c, x.w, g.w, A, D);
+        accumulate_f64(P, M, c, x.x, g.x, A, D); accumulate_f64(P, M, c, x.y, g.y, A, D);
+        accumulate_f64(P, M, c, x.z, g.z, A, D); accumulate_f64(P, M, c, x.w, g.w, A, D);
       }
     } else {
-      for (int i = t; i < n; i += T) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+      for (int i = t; i < n; i += T) accumulate_f64(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
     }
     A = warp_sum(A); D = warp_sum(D);
     if (lane == 0) { red[0][warp] = A; red[1][warp] = D; }
     __syncthreads();
-    A = 0.f; D = 0.f;
+    A = 0.0; D = 0.0;
     for (int w = 0; w < (T >> 5); ++w) { A += red[0][w]; D += red[1][w]; }
-    if (M.mag) D += (float)c.m;
+    if (M.mag) D += (double)c.m;
   }
-  const float ratio = D > 0.0f ? A / D : 0.0f;
+  const double mean = D > 0.0 ? A / D : 0.0;
+  const float ratio = (float)mean, delta = (float)(mean - (double)ratio);
   if (P.vec4) {
     const float4* x4 = reinterpret_cast<const float4*>(x_row);
     const float4* g4 = reinterpret_cast<const float4*>(g_row);
     float4* o4 = reinterpret_cast<float4*>(o_row);
     for (int v = t; 4 * v < n; v += T) {
       float4 x = __ldg(x4 + v), g = __ldg(g4 + v), o;
-      o.x = finish(P, M, c, x.x, g.x, ratio); o.y = finish(P, M, c, x.y, g.y, ratio);
-      o.z = finish(P, M, c, x.z, g.z, ratio); o.w = finish(P, M, c, x.w, g.w, ratio);
+      o.x = finish(P, M, c, x.x, g.x, ratio, delta); o.y = finish(P, M, c, x.y, g.y, ratio, delta);
+      o.z = finish(P, M, c, x.z, g.z, ratio, delta); o.w = finish(P, M, c, x.w, g.w, ratio, delta);
       o4[v] = o;
     }
   } else {
-    for (int i = t; i < n; i += T) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+    for (int i = t; i < n; i += T) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio, delta);
   }
 }
 
 // Rows held in global memory: per-tile partial sums, then every block re-reduces them
 // (no atomics, so results do not depend on scheduling) and finishes its own tile.
-__global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, float2* partial, int tiles) {
-  __shared__ float red[2][8];
+__global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, double2* partial, int tiles) {
+  __shared__ double red[2][8];
   const Math M = make_math(P);
   const long long row = blockIdx.y;
   const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
   const RowCtx c = load_ctx(P, M, row);
-  float A = 0.f, D = 0.f;
+  double A = 0.0, D = 0.0;
   if (c.has_block) {
     const float* x_row = P.theta + row * (long long)n;
     const float* g_row = P.gout + row * (long long)n;
@@ -198,34 +242,35 @@ __global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, floa
 #pragma unroll 4
     for (int j = 0; j < kLongTile / 256; ++j) {
       const int i = start + j * 256 + t;
-      if (i < n) accumulate(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+      if (i < n) accumulate_f64(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
     }
   }
   A = warp_sum(A); D = warp_sum(D);
   if ((t & 31) == 0) { red[0][t >> 5] = A; red[1][t >> 5] = D; }
   __syncthreads();
   if (t == 0) {
-    float a = 0.f, d = 0.f;
+    double a = 0.0, d = 0.0;
     for (int w = 0; w < 8; ++w) { a += red[0][w]; d += red[1][w]; }
-    partial[row * (long long)tiles + tile] = make_float2(a, d);
+    partial[row * (long long)tiles + tile] = make_double2(a, d);
   }
 }
 
-__global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const float2* partial, int tiles) {
+__global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const double2* partial, int tiles) {
   __shared__ double red[2][8];
   const Math M = make_math(P);
   const long long row = blockIdx.y;
   const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
   const RowCtx c = load_ctx(P, M, row);
   double A = 0.0, D = 0.0;
-  for (int i = t; i < tiles; i += 256) { float2 v = partial[row * (long long)tiles + i]; A += v.x; D += v.y; }
+  for (int i = t; i < tiles; i += 256) { double2 v = partial[row * (long long)tiles + i]; A += v.x; D += v.y; }
   A = warp_sum(A); D = warp_sum(D);
   if ((t & 31) == 0) { red[0][t >> 5] = A; red[1][t >> 5] = D; }
   __syncthreads();
   A = 0.0; D = 0.0;
   for (int w = 0; w < 8; ++w) { A += red[0][w]; D += red[1][w]; }
   if (M.mag && c.has_block) D += (double)c.m;
-  const float ratio = D > 0.0 ? (float)(A / D) : 0.0f;
+  const double mean = D > 0.0 ? A / D : 0.0;
+  const float ratio = (float)mean, delta = (float)(mean - (double)ratio);
   const float* x_row = P.theta + row * (long long)n;
   const float* g_row = P.gout + row * (long long)n;
   float* o_row = P.out + row * (long long)n;
@@ -233,17 +278,17 @@ __global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const
 #pragma unroll 4
   for (int j = 0; j < kLongTile / 256; ++j) {
     const int i = start + j * 256 + t;
-    if (i < n) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio);
+    if (i < n) o_row[i] = finish(P, M, c, __ldg(x_row + i), __ldg(g_row + i), ratio, delta);
   }
 }
 
 }  // namespace
 
-// scratch: rows * ceil(n / kLongTile) * 8 bytes
+// scratch: rows * ceil(n / kLongTile) * 16 bytes
 cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream) {
   const int tiles = (P.n + kLongTile - 1) / kLongTile;
   const dim3 grid((unsigned)tiles, (unsigned)P.rows);
-  float2* partial = static_cast<float2*>(scratch);
+  double2* partial = static_cast<double2*>(scratch);
   tk_vjp_long_partial<<<grid, 256, 0, stream>>>(P, partial, tiles);
   tk_vjp_long_finish<<<grid, 256, 0, stream>>>(P, partial, tiles);
   return cudaGetLastError();

@@ -97,6 +97,7 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
     res["fwd_max_rel"] = float(rel_err(gout, ref).max())
     res["fwd_max_abs"] = float(np.abs(gout - ref).max())
     assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
+    bad_noperm = np.zeros(0, np.int64)
     # the call without a permutation output takes its own path for short rows (keys sorted alone,
     # results placed by value): same tolerance against the oracle, same pooled blocks
     if sorts:
@@ -116,7 +117,8 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         assert torch.equal(out2, out3), f"{label}: tk_fwd differs from tk_fwd_ex"
         st2 = read_state(state2, rows)
         ab2 = np.stack([st2["a"], st2["b"]], axis=1).astype(np.int64)
-        disputed_rows_ok(theta, k, p, lam, mode, det, ab2, oracle_blocks(det, k))
+        bad_noperm = disputed_rows_ok(theta, k, p, lam, mode, det, ab2, oracle_blocks(det, k))
+        res["rows_block_disputed_noperm"] = int(len(bad_noperm))
     st = read_state(state, rows)
     gpu_ab = np.stack([st["a"], st["b"]], axis=1).astype(np.int64)
     ref_ab = oracle_blocks(det, k)
@@ -126,11 +128,13 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         g = np.ascontiguousarray(g, np.float32)
         gt = torch.from_numpy(g).to(dev)
         gref = tko.vjp(theta, g, k, p, lam, mode)
-        keep = np.ones(rows, bool)
-        keep[bad] = False
         for name, kwargs in (("vjp_state", {"state": state}), ("vjp_recompute", {})):
             if name == "vjp_recompute" and (ws_bytes or not sorts):
                 continue
+            # rows left out: near-ties at a block edge in the solve this VJP rests on (the saved
+            # state of the first call; its own solve, the one of the second call, when it recomputes)
+            keep = np.ones(rows, bool)
+            keep[bad if name == "vjp_state" else bad_noperm] = False
             grad = torch.full((rows, n), float("nan"), device=dev)
             tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, workspace=ws, **kwargs)
             torch.cuda.synchronize()
@@ -140,4 +144,44 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
             res[name + "_max_rel"] = float(e[keep].max()) if keep.any() else 0.0
             res[name + "_max_abs"] = float(np.abs(gg - gref)[keep].max()) if keep.any() else 0.0
             assert res[name + "_max_rel"] <= TOL, f"{label}: {name} error {res}"
+    return res
+
+
+def run_sampled(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.ndarray,
+                sample: np.ndarray, label: str = ""):
+    """Full-size launch as the benchmark times it (default path: no permutation, row state saved,
+    VJP from state); the oracle checks the sampled rows only, element by element."""
+    theta = np.ascontiguousarray(theta, np.float32)
+    g = np.ascontiguousarray(g, np.float32)
+    rows, n = theta.shape
+    dev = torch.device("cuda")
+    th = torch.from_numpy(theta).to(dev)
+    gt = torch.from_numpy(g).to(dev)
+    out = torch.full((rows, n), float("nan"), device=dev)
+    grad = torch.full((rows, n), float("nan"), device=dev)
+    state = tk.new_state(rows)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_bytes = tk.tk_workspace_bytes(rows, n, k, p, mode)
+    ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device=dev) if ws_bytes else None
+    tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, state_out=state, workspace=ws, status_out=status)
+    tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, state=state, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, f"{label}: status {int(status.item())}"
+    assert bool(torch.isfinite(out).all()) and bool(torch.isfinite(grad).all()), f"{label}: non-finite result"
+    sample = np.asarray(sample, np.int64)
+    idx = torch.from_numpy(sample).to(dev)
+    sub = theta[sample]
+    ref, det = tko.fwd(sub, k, p, lam, mode, details=True)
+    res = {"fwd_max_rel": float(rel_err(out[idx].cpu().numpy(), ref).max())}
+    assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
+    st = read_state(state, rows)[sample]
+    gpu_ab = np.stack([st["a"], st["b"]], axis=1).astype(np.int64)
+    bad = disputed_rows_ok(sub, k, p, lam, mode, det, gpu_ab, oracle_blocks(det, k))
+    keep = np.ones(len(sample), bool)
+    keep[bad] = False
+    gref = tko.vjp(sub, g[sample], k, p, lam, mode)
+    e = rel_err(grad[idx].cpu().numpy(), gref)
+    res["vjp_max_rel"] = float(e[keep].max()) if keep.any() else 0.0
+    res["rows_block_disputed"] = int(len(bad))
+    assert res["vjp_max_rel"] <= TOL, f"{label}: VJP error {res}"
     return res

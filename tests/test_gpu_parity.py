@@ -167,6 +167,57 @@ def test_pruning_config_full_size():
     print("pruning", res)
 
 
+def test_moe_router_config_full_size():
+    """The benchmark's default workload, every variant, every element."""
+    from parity import run_case
+    for case in wl.moe_router_cases():
+        x = case.theta()
+        g = case.cotangent(x)
+        run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
+
+
+def test_class_logit_config_full_size():
+    from parity import run_case
+    case = wl.class_logit_case()
+    x = case.theta()
+    g = case.cotangent(x)
+    run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
+
+
+def test_sweep_configs_full_size_sampled_rows():
+    """2^26-element launches as the benchmark times them; the oracle checks a sample of rows."""
+    from parity import run_sampled
+    for case in wl.shape_sweep_cases():
+        if case.n > 4096:
+            continue
+        x = case.theta()
+        g = case.cotangent(x)
+        rng = np.random.Generator(np.random.PCG64(case.seed + 77))
+        count = max(32, min(4096, (1 << 18) // case.n))
+        sample = np.sort(rng.choice(case.rows, size=count, replace=False))
+        sample[0], sample[-1] = 0, case.rows - 1          # first and last row of the launch
+        res = run_sampled(x, case.k, case.p, case.lam, case.mode, g, sample, label=case.name)
+        print(case.name, res)
+        del x, g
+        torch.cuda.empty_cache()
+
+
+def test_short_row_kernel_every_batch_count():
+    """Rows of up to 256 elements run 1, 2 or the full number of row batches per warp, by row count:
+    one case per (lanes per row, batches) pair beyond the single-batch ones the small tests cover."""
+    from parity import run_case
+    modes = [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG]
+    cases = [(12, 120001), (24, 60001), (24, 120001), (50, 30001), (50, 120001),
+             (100, 15001), (100, 60001), (200, 7501), (200, 30001)]
+    for i, (n, rows) in enumerate(cases):
+        p = 2.0 if i % 2 == 0 else P43
+        lam = (0.1, 1.0, 3.0)[i % 3]
+        k = max(1, n // (3 + i % 4))
+        x = rows_of(n, rows, 300 + i)
+        g = wl.cotangent_like(x, 300 + i)
+        run_case(x, k, p, lam, modes[i % 3], g, label=f"n={n} rows={rows} k={k} lam={lam} p={p}")
+
+
 def test_sweep_n32768_sampled_rows():
     from parity import run_case
     for case in wl.shape_sweep_cases():
