@@ -4,8 +4,8 @@
 //   load row -> (key, index) packed in 64 bits -> block-wide merge sort in
 //   shared memory (stable: ties by ascending index) -> exact isotonic solve
 //   -> dual map y = rho(s - v) -> scatter through shared memory -> coalesced
-//   store.  The VJP variant (Prop. 7) continues from the solve with the
-//   cotangent staged in the same shared buffer.
+//   store.  Used when the caller wants the permutation (perm_out, tk_argsort);
+//   the default forward pass and every VJP sort the keys alone (tk_ctav.cu).
 //
 // Isotonic solve.  With w = 1_k the singleton minimisers are non-increasing on
 // ranks < k and on ranks >= k, so pooling adjacent violators can only ever grow
@@ -40,7 +40,6 @@ tk_cta_kernel(const Problem P) {
 
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);   // pad(N) slots
   float* stage = reinterpret_cast<float*>(smem_raw);                             // aliases keys, [N]
-  float* stage2 = stage + N;                                                     // second [N] in the same space
   const int key_slots = pad(N) + 1;
   double* cps = reinterpret_cast<double*>(keys + key_slots);                     // 3 x (T + 1)
   double* redd = cps + 3 * (T + 1);                                              // 40 doubles
@@ -231,7 +230,7 @@ tk_cta_kernel(const Problem P) {
   };
   __syncthreads();       // every read of keys[] is done; stage[] may overwrite it
 
-  if (P.what == W_FWD) {
+  {   // forward pass only: tk_vjp never asks for a permutation, so it never comes here
 #pragma unroll
     for (int i = 0; i < E; ++i) {
       int idx = un_idx(r[i]);
@@ -258,51 +257,6 @@ tk_cta_kernel(const Problem P) {
         o_row[i] = q;
       }
     }
-  } else {
-    // ---- VJP (Prop. 7 chained through the dual map).  In sorted coordinates, for the pooled
-    // block B: o_j = rho'_j (g_j - A/D), A = sum_B rho'_l g_l, D = sum_B rho'_l (+ m_B, phi even).
-    const float* g_row = P.gout + row * (long long)n;
-    for (int i = t; i < n; i += T) stage[i] = __ldg(g_row + i);
-    __syncthreads();
-    auto chi_in = [&](unsigned long long e, int idx) -> float {
-      if (mag) return un_neg(e) ? -1.0f : 1.0f;
-      if (P.mode == TK_TOPK) return __ldg(x_row + idx);
-      return 1.0f;
-    };
-    float A = 0.f, D = 0.f;
-#pragma unroll
-    for (int i = 0; i < E; ++i) {
-      int rk = t * E + i;
-      int idx = un_idx(r[i]);
-      if (rk < n && idx < n && rk >= a0 && rk < b0) {
-        float dr = M.drho(fminf(fmaxf(TK_D(i) - u, 0.0f), wid));
-        D += dr;
-        A += dr * chi_in(r[i], idx) * stage[idx];
-      }
-    }
-    float Ab = block_sum<float>(A, reinterpret_cast<float*>(redd));
-    float Db = block_sum<float>(D, reinterpret_cast<float*>(redd));
-    if (mag) Db += (float)(k - a0);
-    const float ratio = (Db > 0.0f) ? Ab / Db : 0.0f;
-#pragma unroll
-    for (int i = 0; i < E; ++i) {
-      int rk = t * E + i;
-      int idx = un_idx(r[i]);
-      if (rk < n && idx < n) {
-        float g = stage[idx];
-        float gsv = chi_in(r[i], idx) * g;
-        float o;
-        if (rk < a0) o = mag ? gsv * M.top_slope(un_key(r[i])) : 0.0f;
-        else if (rk < b0) o = M.drho(fminf(fmaxf(TK_D(i) - u, 0.0f), wid)) * (gsv - ratio);
-        else o = 0.0f;
-        if (mag && un_neg(r[i])) o = -o;
-        if (P.mode == TK_TOPK) o += g * y_of(rk, r[i]);     // product rule: g * mask
-        stage2[idx] = o;
-      }
-    }
-    __syncthreads();
-    float* o_row = P.out + row * (long long)n;
-    for (int i = t; i < n; i += T) o_row[i] = stage2[i];
   }
 #undef TK_D
   if (t == 0 && row_flags && P.status) atomicOr(P.status, row_flags);

@@ -7,7 +7,8 @@
 //   bitonic merges across lanes by shuffles) -> exact single-block isotonic
 //   solve (G-ary search on the monotone predicates, O(1) probes through prefix
 //   sums staged in shared memory) -> dual map -> scatter through shared memory
-//   -> coalesced store; optionally the VJP of Prop. 7 in the same pass.
+//   -> coalesced store.  Used when the caller wants the permutation (perm_out, tk_argsort);
+//   the default forward pass and every VJP sort the keys alone (tk_rows.cu, tk_groupv.cu).
 #include "tk_common.cuh"
 #include "tk_group_sort.cuh"
 
@@ -24,7 +25,6 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const P
   constexpr int STRIDE = N + N / EPL + 1;     // padded slots per array per row
   auto pad8 = [](int i) -> int { return pad_e<EPL>(i); };
   __shared__ float sm[GROUPS][4][STRIDE];     // [0] keys / staging, [1..3] prefix sums of d, d^2, d^3
-  __shared__ float sm2[GROUPS][STRIDE];       // second staging buffer (VJP)
 
   const int tid = threadIdx.x;
   const int grp = tid / G, lig = tid % G;
@@ -190,7 +190,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const P
   float* stage = sk;
   float* o_row = P.out + row * (long long)n;
 
-  if (P.what == W_FWD) {
+  {   // forward pass only: tk_vjp never asks for a permutation, so it never comes here
 #pragma unroll
     for (int i = 0; i < EPL; ++i) {
       const int idx = un_idx(r[i]);
@@ -220,49 +220,6 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const P
         }
       }
     }
-  } else {
-    // ---- VJP (Prop. 7): o_j = rho'_j (g_j - A/D) on the pooled block
-    const float* g_row = P.gout + row * (long long)n;
-    float* stage2 = sm2[grp];
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) { const int idx = EPL * lig + i; if (idx < n) stage[pad8(idx)] = __ldg(g_row + idx); }
-    __syncwarp(mask);
-    auto chi_in = [&](unsigned long long e, int idx) -> float {
-      if (mag) return un_neg(e) ? -1.0f : 1.0f;
-      if (P.mode == TK_TOPK) return __ldg(x_row + idx);
-      return 1.0f;
-    };
-    float A = 0.f, D = 0.f;
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) {
-      const int rk = EPL * lig + i, idx = un_idx(r[i]);
-      if (rk < n && idx < n && rk >= a0 && rk < b0) {
-        const float dr = M.drho(fminf(fmaxf((un_key(r[i]) - piv) - u, 0.0f), wid));
-        D += dr; A += dr * chi_in(r[i], idx) * stage[pad8(idx)];
-      }
-    }
-    A = group_sum<G, float>(A, mask);
-    D = group_sum<G, float>(D, mask);
-    if (mag) D += (float)(k - a0);
-    const float ratio = D > 0.0f ? A / D : 0.0f;
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) {
-      const int rk = EPL * lig + i, idx = un_idx(r[i]);
-      if (rk < n && idx < n) {
-        const float g = stage[pad8(idx)];
-        const float gsv = chi_in(r[i], idx) * g;
-        float o;
-        if (rk < a0) o = mag ? gsv * M.top_slope(un_key(r[i])) : 0.0f;
-        else if (rk < b0) o = M.drho(fminf(fmaxf((un_key(r[i]) - piv) - u, 0.0f), wid)) * (gsv - ratio);
-        else o = 0.0f;
-        if (mag && un_neg(r[i])) o = -o;
-        if (P.mode == TK_TOPK) o += g * y_of(rk, r[i]);
-        stage2[pad8(idx)] = o;
-      }
-    }
-    __syncwarp(mask);
-#pragma unroll
-    for (int i = 0; i < EPL; ++i) { const int idx = EPL * lig + i; if (idx < n) o_row[idx] = stage2[pad8(idx)]; }
   }
   if (flags && P.status) atomicOr(P.status, flags);
 }

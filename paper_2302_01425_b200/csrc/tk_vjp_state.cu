@@ -39,36 +39,14 @@ __device__ __forceinline__ int classify(const RowCtx& c, float key, float& tt) {
   return t > 0.0f ? 1 : 0;
 }
 
-__device__ __forceinline__ void accumulate(const Problem& P, const Math& M, const RowCtx& c, float x,
-                                           float g, float& A, float& D) {
-  float tt;
-  float key = sort_key(x, M.mag);
-  if (classify(c, key, tt) == 1) {
-    float dr = M.drho(tt);
-    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
-    D += dr;
-    A += dr * chi * g;
-  }
-}
-
 // The mean A/D is needed to a relative accuracy of its DISTANCE from chi g, not of itself: rho' can
 // be 3/lambda, and one ulp of A/D times that is above 1e-5.  Two ways to get it:
-//  * rows held in registers: a second pass sums the residuals rho' (chi g - r0) about the fp32 mean
-//    r0 of the first pass; each residual is one fma (no cancellation), and the correction
-//    delta = (sum - m r0)/D restores what the division rounded away;
+//  * rows held in registers: a second pass over the registers sums the residuals rho' (chi g - r0)
+//    about the fp32 mean r0 of the first pass; each residual is one fma (no cancellation), and
+//    the correction delta = (sum - m r0)/D restores what the division rounded away;
 //  * rows streamed from memory: A and D are accumulated in fp64 (products of floats are exact
 //    there), the mean is split into r0 = fl(mean) and delta = mean - r0.
 // Either way the result is rho' ((chi g - r0) - delta).
-__device__ __forceinline__ void accumulate_residual(const Problem& P, const Math& M, const RowCtx& c, float x,
-                                                    float g, float r0, float& A2) {
-  float tt;
-  float key = sort_key(x, M.mag);
-  if (classify(c, key, tt) == 1) {
-    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
-    A2 += M.drho(tt) * fmaf(chi, g, -r0);
-  }
-}
-
 __device__ __forceinline__ void accumulate_f64(const Problem& P, const Math& M, const RowCtx& c, float x,
                                                float g, double& A, double& D) {
   float tt;
@@ -135,29 +113,48 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
       }
   }
   const RowCtx c = load_ctx(P, M, row);
+  // One classification per element: w = sign * rho' on the pooled block (else 0) and the part of
+  // the result that does not depend on the block mean; then
+  //   o = w ((chi g - r0) - delta) + fixed,   r0 = fl(A / D),   delta = (sum w' (chi g - r0) - m r0) / D.
+  auto chi_of = [&](float xv) -> float {
+    return M.mag ? (signbit(xv) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? xv : 1.0f);
+  };
+  float w[CH][4], fixed[CH][4];
   float A = 0.f, D = 0.f;
+#pragma unroll
+  for (int ch = 0; ch < CH; ++ch)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float xv = x[ch][j], gv = g[ch][j];
+      const bool in = 4 * (ch * G + lig) + j < n;
+      float tt = 0.0f;
+      const float key = sort_key(xv, M.mag);
+      const int cls = in ? classify(c, key, tt) : 0;
+      const float sgn = (M.mag && signbit(xv)) ? -1.0f : 1.0f;
+      const float chi = chi_of(xv);
+      const float dr = cls == 1 ? M.drho(tt) : 0.0f;
+      float f = (cls == 2 && M.mag) ? gv * M.top_slope(key) : 0.0f;          // sgn chi = 1 there
+      if (P.mode == TK_TOPK) f += gv * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));
+      w[ch][j] = sgn * dr;
+      fixed[ch][j] = f;
+      D += dr;
+      A += dr * chi * gv;
+    }
+  float ratio = 0.0f, delta = 0.0f;
   if (c.has_block) {
-#pragma unroll
-    for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        if (4 * (ch * G + lig) + j < n) accumulate(P, M, c, x[ch][j], g[ch][j], A, D);
 #pragma unroll
     for (int o = G >> 1; o > 0; o >>= 1) {
       A += __shfl_xor_sync(mask, A, o);
       D += __shfl_xor_sync(mask, D, o);
     }
     if (M.mag) D += (float)c.m;
-  }
-  const float ratio = D > 0.0f ? A / D : 0.0f;
-  float delta = 0.0f;
-  if (c.has_block) {
+    ratio = D > 0.0f ? A / D : 0.0f;
     float A2 = 0.f;
 #pragma unroll
     for (int ch = 0; ch < CH; ++ch)
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (4 * (ch * G + lig) + j < n) accumulate_residual(P, M, c, x[ch][j], g[ch][j], ratio, A2);
+        A2 = fmaf(fabsf(w[ch][j]), fmaf(chi_of(x[ch][j]), g[ch][j], -ratio), A2);   // |w| = rho'
 #pragma unroll
     for (int o = G >> 1; o > 0; o >>= 1) A2 += __shfl_xor_sync(mask, A2, o);
     if (M.mag) A2 -= (float)c.m * ratio;
@@ -168,7 +165,9 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
     const int v = ch * G + lig;
     float o[4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) o[j] = finish(P, M, c, x[ch][j], g[ch][j], ratio, delta);
+    for (int j = 0; j < 4; ++j) {
+      o[j] = fmaf(w[ch][j], fmaf(chi_of(x[ch][j]), g[ch][j], -ratio) - delta, fixed[ch][j]);
+    }
     if (P.vec4) {
       if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o[0], o[1], o[2], o[3]);
     } else {
