@@ -295,21 +295,26 @@ cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t 
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
   if (P.n <= 512) {
-    // lanes per row: one float4 per lane up to 128 elements, then 2 or 4 chunks per lane
+    // lanes per row: two float4 per lane (one for n <= 4), four for 256 < n <= 512
+    if (P.n > 256) {
+      const unsigned blocks = (unsigned)((P.rows + 7) / 8);
+      tk_vjp_state_group<32, 4><<<blocks, 256, 0, stream>>>(P);
+      return cudaGetLastError();
+    }
     int G = 1;
-    while (G < 32 && G * 4 < P.n) G <<= 1;
-    const int CH = (P.n + 4 * G - 1) / (4 * G);     // 1, 2, 3 or 4
+    while (G < 32 && G * 8 < P.n) G <<= 1;
     const long long rows_per_block = 8 * (32 / G);
     const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
-    if (CH > 2) { tk_vjp_state_group<32, 4><<<blocks, 256, 0, stream>>>(P); return cudaGetLastError(); }
-    if (CH == 2) { tk_vjp_state_group<32, 2><<<blocks, 256, 0, stream>>>(P); return cudaGetLastError(); }
     switch (G) {
-      case 1: tk_vjp_state_group<1, 1><<<blocks, 256, 0, stream>>>(P); break;
-      case 2: tk_vjp_state_group<2, 1><<<blocks, 256, 0, stream>>>(P); break;
-      case 4: tk_vjp_state_group<4, 1><<<blocks, 256, 0, stream>>>(P); break;
-      case 8: tk_vjp_state_group<8, 1><<<blocks, 256, 0, stream>>>(P); break;
-      case 16: tk_vjp_state_group<16, 1><<<blocks, 256, 0, stream>>>(P); break;
-      default: tk_vjp_state_group<32, 1><<<blocks, 256, 0, stream>>>(P); break;
+      case 1:
+        if (P.n <= 4) tk_vjp_state_group<1, 1><<<blocks, 256, 0, stream>>>(P);
+        else tk_vjp_state_group<1, 2><<<blocks, 256, 0, stream>>>(P);
+        break;
+      case 2: tk_vjp_state_group<2, 2><<<blocks, 256, 0, stream>>>(P); break;
+      case 4: tk_vjp_state_group<4, 2><<<blocks, 256, 0, stream>>>(P); break;
+      case 8: tk_vjp_state_group<8, 2><<<blocks, 256, 0, stream>>>(P); break;
+      case 16: tk_vjp_state_group<16, 2><<<blocks, 256, 0, stream>>>(P); break;
+      default: tk_vjp_state_group<32, 2><<<blocks, 256, 0, stream>>>(P); break;
     }
   } else {
     tk_vjp_state_cta<<<(unsigned)P.rows, 256, 0, stream>>>(P);
