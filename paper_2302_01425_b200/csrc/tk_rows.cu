@@ -4,10 +4,10 @@
 //   1. in batches of 32/G rows (G lanes x 8 elements per row): load, sort the 32-bit KEYS by the
 //      shuffle network, leave the sorted row in the warp's shared memory;
 //   2. lane r solves row r: the isotonic problem of Sec. 5 has at most one pooled block [a0, b0)
-//      around ranks k-1 and k, and both edges are found by WALKING outwards from k with running
-//      power sums of d = key - pivot (see solve_row_walk).  Up to 32 rows walk side by side, so
-//      the solve costs a warp a few instructions per block member instead of a search replicated
-//      over the G lanes of every row;
+//      around ranks k-1 and k, and it is grown from that pair one rank at a time, pooling a
+//      neighbour while it violates the order, on running power sums of d = key - pivot (see
+//      solve_row_walk).  Up to 32 rows walk side by side, so the solve costs a warp a few
+//      instructions per block member instead of a search replicated over the G lanes of every row;
 //   3. in the same batches: the results by value (given gamma and the cap width, the output and
 //      the VJP of an element depend on its own key alone), stored where they were loaded.
 // No index travels through the sort and nothing is scattered; the phases are separated by warp
@@ -52,15 +52,22 @@ __device__ __forceinline__ float block_value(float lam, float lam3, float piv, f
 }
 
 // The isotonic solve of one row by ONE thread, on the row's sorted keys in shared memory (rank i at
-// sk[i + i/8]).  F(tau) = #{capped at tau} - k + sum over the ranks strictly between the caps of
-// rho(s_i - tau) / phi'(tau) is the monotone threshold function whose root is gamma.  Rank j > k
-// joins the block while F(s_j) < 0; rank j < k-1 joins while F(vtop(s_j)) > 0.  Each edge is one
-// flat loop: a step either moves the far end of the summed range (which only moves one way as j
-// does) or tests j and moves on, so 32 lanes with different rows stay in one instruction stream.
+// sk[i]).  With w = 1_k every rank is its own minimiser (vtop(s_i) for i < k, s_i for i >= k) and
+// both runs are non-increasing, so pooling adjacent violators only ever grows ONE block from the
+// pair (k-1, k) (Sec. 5).  The block [a, b) with m = k - a weighted members has the value gamma
+// that solves  H(tau) = sum_{i in block} rho(s_i - tau) - m phi'(tau) = 0,  H decreasing, and
+//   rank b   violates (gamma < s_b)          <=>  H(s_b) < 0          -> pool it,
+//   rank a-1 violates (vtop(s_{a-1}) < gamma) <=>  H(vtop(s_{a-1})) > 0 -> pool it.
+// rho is an odd polynomial of degree q - 1, so H is a polynomial in tau whose coefficients are the
+// block's power sums of d = key - pivot: a test is a handful of fmas and pooling a rank is one add
+// per sum.  The loop is flat (one candidate per step, the side changes when a test fails, two
+// failures in a row end it), so 32 lanes with different rows stay in one instruction stream, and
+// it runs for (block size + a few) steps.  The sums only ever grow; fp64 copies of them give the
+// block mean and central moments for the block value.
 template <bool Q4, bool MAG>
 __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, const Math& M, const Problem& P,
                                                RowSol& R) {
-  auto key = [&](int i) -> float { return sk[i + (i >> 3)]; };
+  auto key = [&](int i) -> float { return sk[i]; };
   const float c = key(k - 1);
   const float vtop_c = M.vtop(c);
   const bool has_block = (k < n) && (vtop_c < key(k));
@@ -71,96 +78,54 @@ __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, co
   int a0 = k, b0 = k;
   float u = 0.0f;
   if (has_block) {
-    const float W_hi = (piv == c) ? M.width(c) : c + M.width(c);
-    const float W_lo = vtop_c - piv;
     const float il3 = P.inv_lam * P.inv_lam * P.inv_lam;
     float D1 = 0.f, D2 = 0.f, D3 = 0.f;
-    auto add = [&](float d) { D1 += d; if (Q4) { const float d2 = d * d; D2 += d2; D3 = fmaf(d2, d, D3); } };
-    auto sub = [&](float d) { D1 -= d; if (Q4) { const float d2 = d * d; D2 -= d2; D3 = fmaf(-d2, d, D3); } };
-    // F at gamma = pivot + uu, ranks [r_hi, r_lo) between the caps with power sums E1..E3
-    auto Fval = [&](float uu, int r_hi, int r_lo, float E1, float E2, float E3) -> float {
-      const float cnt = (float)(r_lo - r_hi);
-      float S;
-      if (Q4) S = (((-cnt * uu + 3.0f * E1) * uu - 3.0f * E2) * uu + E3) * il3;
-      else S = (E1 - cnt * uu) * P.inv_lam;
-      if (MAG) S = S / (piv + uu);
-      return (float)(r_hi - k) + S;
+    double E1 = 0.0, E2 = 0.0, E3 = 0.0;
+    auto pool = [&](float d) {
+      D1 += d;
+      const double dd = (double)d;
+      E1 += dd;
+      if (Q4) {
+        const float d2 = d * d;
+        D2 += d2; D3 = fmaf(d2, d, D3);
+        const double dd2 = dd * dd;
+        E2 += dd2; E3 = fma(dd2, dd, E3);
+      }
     };
-    // ---- upper edge.  r_hi(j) = #{i < k : d_i >= d_j + width(s_j)} only grows with j: start it at
-    // its least value (the window's upper end) and advance.
-    {
-      int r_hi = k;
-      while (r_hi > 0) { const float d = key(r_hi - 1) - piv; if (d >= W_hi) break; add(d); --r_hi; }
-      add(key(k) - piv);
-      int j = k + 1;
-      b0 = k + 1;
-      float uu = 0.f, thr = 0.f;
-      bool in_window = false;
-      auto prep = [&]() {
-        const float tau = key(min(j, n - 1));
-        uu = tau - piv;
-        in_window = (j < n) && (uu > W_lo) && !(MAG && !(tau > 0.0f));   // else at or below vtop(c)
-        thr = uu + M.width(tau);
-      };
-      prep();
-      while (in_window) {
-        const float dr = key(min(r_hi, k - 1)) - piv;
-        if (r_hi < k && dr >= thr) { sub(dr); ++r_hi; }
-        else {
-          if (!(Fval(uu, r_hi, j, D1, D2, D3) < 0.0f)) break;
-          add(uu); ++j; b0 = j;
-          prep();
-        }
+    // H at tau = pivot + uu for the block [a, b)
+    auto H = [&](float uu, int a, int b) -> float {
+      const float cnt = (float)(b - a), m = (float)(k - a);
+      float S;
+      if (Q4) S = (((-cnt * uu + 3.0f * D1) * uu - 3.0f * D2) * uu + D3) * il3;
+      else S = (D1 - cnt * uu) * P.inv_lam;
+      return S - (MAG ? m * (piv + uu) : m);
+    };
+    a0 = k - 1; b0 = k + 1;
+    pool(c - piv);
+    pool(key(k) - piv);
+    int below = 1, fails = 0;          // which neighbour is tried next: rank b0 (below) or rank a0 - 1
+    while (fails < 2) {
+      bool joins = false;
+      float d = 0.0f;
+      if (below) {
+        if (b0 < n) { d = key(b0) - piv; joins = H(d, a0, b0) < 0.0f; }
+        b0 += joins ? 1 : 0;
+      } else {
+        if (a0 > 0) { const float s = key(a0 - 1); d = s - piv; joins = H(M.vtop(s) - piv, a0, b0) > 0.0f; }
+        a0 -= joins ? 1 : 0;
       }
+      if (joins) { pool(d); fails = 0; }
+      else { ++fails; below ^= 1; }
     }
-    // ---- lower edge.  r_lo(j) = k + #{i >= k : d_i > vtop(s_j) - pivot} only shrinks as j falls:
-    // start it at its greatest value (the window's lower end) and retreat.
-    a0 = k - 1;
-    if (k >= 2) {
-      D1 = 0.f; D2 = 0.f; D3 = 0.f;
-      int r_lo = k;
-      while (r_lo < n) { const float d = key(r_lo) - piv; if (!(d > W_lo)) break; add(d); ++r_lo; }
-      add(key(k - 1) - piv);
-      int j = k - 2;
-      float dj = 0.f, uu = 0.f;
-      bool open = false, valid = false;
-      auto prep = [&]() {
-        const float sj = key(max(j, 0));
-        dj = sj - piv;
-        open = (j >= 0) && !(dj >= W_hi);               // else capped whatever gamma is
-        const float tau = M.vtop(sj);
-        uu = tau - piv;
-        valid = !(MAG && !(tau > 0.0f));
-      };
-      prep();
-      while (open) {
-        const float dl = key(max(r_lo - 1, k)) - piv;
-        if (valid && r_lo > k && !(dl > uu)) { sub(dl); --r_lo; }
-        else {
-          if (valid) {
-            const float dj2 = dj * dj;
-            // F <= 0: rank j stays a top singleton, and so do all ranks above it
-            if (Fval(uu, j, r_lo, D1 + dj, D2 + dj2, fmaf(dj2, dj, D3)) <= 0.0f) break;
-          }
-          a0 = j; add(dj); --j;
-          prep();
-        }
-      }
-    }
-    // ---- block mean and central sums over [a0, b0), then the block value
-    double s1 = 0.0;
-    for (int i = a0; i < b0; ++i) s1 += (double)(key(i) - piv);
-    const float cnt = (float)(b0 - a0), m = (float)(k - a0);
-    const float mu = (float)(s1 / (double)cnt);
+    // ---- block value from the mean and the central moments
+    const double cntd = (double)(b0 - a0);
+    const double mud = E1 / cntd;
     float M2 = 0.f, M3 = 0.f;
     if (Q4) {
-      for (int i = a0; i < b0; ++i) {
-        const float e = (key(i) - piv) - mu;
-        const float e2 = e * e;
-        M2 += e2; M3 = fmaf(e2, e, M3);
-      }
+      M2 = (float)(E2 - E1 * mud);
+      M3 = (float)(E3 - 3.0 * mud * E2 + 2.0 * mud * mud * E1);
     }
-    u = block_value<Q4, MAG>(P.lam, P.lam3, piv, cnt, m, mu, M2, M3);
+    u = block_value<Q4, MAG>(P.lam, P.lam3, piv, (float)cntd, (float)(k - a0), (float)mud, M2, M3);
     u = settle_offset(M, piv, u, a0, b0, n, key);
   }
   R.piv = piv; R.u = u; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = has_block ? 1 : 0;
@@ -176,7 +141,7 @@ struct RowsGeom {
   static constexpr int N = 8 * G;                          // padded row length
   static constexpr int RPB = 32 / G;                       // rows per batch
   static constexpr int R = RPB * B;                        // rows per warp
-  static constexpr int STRIDE = (N + G - 1) | 1;           // odd: lane r walking row r meets no bank conflict
+  static constexpr int STRIDE = N | 1;                     // odd: lane r walking row r meets no bank conflict
 };
 
 template <int G, int B, bool Q4, bool MAG>
@@ -231,7 +196,7 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
     group_sort_keys<G, 8>(s, lig, mask);
     float* sk = sm[warp][rr];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sk[9 * lig + i] = s[i];   // rank 8 lig + i, one spare slot per 8
+    for (int i = 0; i < 8; ++i) sk[8 * lig + i] = s[i];   // rank 8 lig + i
   }
   __syncwarp();
 
