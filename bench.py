@@ -56,6 +56,8 @@ def _workload_cases(name: str):
         return wl.moe_router_cases()
     if name == "class_logit":
         return [wl.class_logit_case()]
+    if name == "expert_choice":
+        return [wl.expert_choice_case()]
     if name == "pruning":
         return [wl.pruning_case()]
     if name == "tiny":
@@ -312,7 +314,7 @@ def main():
         if world == 1:
             if not args.no_extra:
                 extra = []
-                names = ["class_logit", "pruning"] + [f"sweep_n{n}" for n in (8, 64, 512, 4096, 32768)]
+                names = ["class_logit", "expert_choice", "pruning"] + [f"sweep_n{n}" for n in (8, 64, 512, 4096, 32768)]
                 for name in names:
                     if name == args.workload:
                         continue
@@ -327,6 +329,9 @@ def main():
                         if name.startswith("sweep_n") and int(name[7:]) <= 4096:
                             entry["dykstra_forward_100_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
+                        if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
+                            entry["dykstra_forward_10_sweeps"] = time_solver_forward(
+                                name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
                         ncase = workload_cases(name)[0].n
                         if 512 <= ncase <= 16384:
                             # the same exact result without the sort (solver = TK_SOLVER_THRESHOLD),

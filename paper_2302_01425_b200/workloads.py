@@ -129,6 +129,13 @@ def class_logit_case() -> Case:
                 kind="class_logit", scale=3.0)
 
 
+def expert_choice_case() -> Case:
+    """Expert-choice routing: every expert picks k = 28 of n = 400 tokens (32 experts x 1024 groups
+    of tokens = 32768 rows), p = 2.  The regularisation strength of that experiment is not stated;
+    lambda = 1 here."""
+    return Case("expert_choice", 32 * 1024, 400, 28, 2.0, 1.0, MODE_MASK, seed=4)
+
+
 def pruning_case() -> Case:
     n = 2048 * 2048
     return Case("pruning", 1, n, n // 10, 2.0, 1e-3, MODE_TOPKMAG, seed=3, scale=0.02)
@@ -146,5 +153,5 @@ def shape_sweep_cases(total_log2: int = 26) -> List[Case]:
 
 
 def all_cases() -> List[Case]:
-    return (tiny_cases() + moe_router_cases() + [class_logit_case(), pruning_case()]
+    return (tiny_cases() + moe_router_cases() + [class_logit_case(), expert_choice_case(), pruning_case()]
             + shape_sweep_cases())

@@ -184,6 +184,24 @@ def test_class_logit_config_full_size():
     run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
 
 
+def test_expert_choice_config_full_size():
+    """32768 x 400, k = 28: the exact path on every element, and 10 Dykstra sweeps against the
+    oracle's iteration at the same count."""
+    from oracle import tko
+    from parity import run_case, TOL
+    case = wl.expert_choice_case()
+    x = case.theta()
+    g = case.cotangent(x)
+    run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
+    th = torch.from_numpy(x).cuda()
+    out = torch.full_like(th, float("nan"))
+    tk.tk_fwd_ex(th, case.rows, case.n, case.k, case.p, case.lam, case.mode, out,
+                 solver=tk.TK_SOLVER_DYKSTRA, sweeps=10)
+    torch.cuda.synchronize()
+    ref = tko.dykstra(x, case.k, case.p, case.lam, case.mode, sweeps=10)
+    assert float(np.max(np.abs(out.cpu().numpy() - ref))) <= TOL
+
+
 def test_sweep_configs_full_size_sampled_rows():
     """2^26-element launches as the benchmark times them; the oracle checks a sample of rows."""
     from parity import run_sampled
