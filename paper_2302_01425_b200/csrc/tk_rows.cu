@@ -178,6 +178,7 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
   };
 
   // ---- phase 1: sort the keys of every row, batch by batch
+  float xkeep[8];                                 // a single batch keeps its row for phase 3
 #pragma unroll 1
   for (int b = 0; b < BATCHES; ++b) {
     const int rr = b * RPB + gw;
@@ -185,6 +186,10 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
     const bool live = row < P.rows;
     float x[8], s[8];
     load8(P.theta + (live ? row : 0) * (long long)n, live, x);
+    if (BATCHES == 1) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) xkeep[i] = x[i];
+    }
     bool bad = false;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
@@ -225,7 +230,12 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
     const float c = __shfl_sync(0xffffffffu, mine.c, rr);
     const int a0 = __shfl_sync(0xffffffffu, mine.a0, rr);
     float x[8];
-    load8(P.theta + (live ? row : 0) * (long long)n, live, x);
+    if (BATCHES == 1) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) x[i] = xkeep[i];
+    } else {
+      load8(P.theta + (live ? row : 0) * (long long)n, live, x);   // second read: L1 / L2
+    }
     const float wid = has_block ? M.width(piv + u) : 0.0f;
     // class of a key: 2 capped (top singleton), 1 pooled, 0 zero; tt = key - gamma, clamped
     auto classify = [&](float key, float& tt) -> int {
