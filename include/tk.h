@@ -92,8 +92,11 @@ typedef struct {
   int32_t *status_out;     /* one device word, OR of TK_FLAG_*; the caller zeroes it          */
 } tk_opts;
 
-/* Scratch bytes tk_fwd_ex / tk_vjp / tk_argsort need for this shape (0 when the
- * row is solved on chip).  solver as in tk_opts.                               */
+/* Scratch bytes tk_fwd_ex / tk_vjp / tk_argsort need for this shape: 0 for rows
+ * of up to 16384 elements.  Rows of 16385..32768 elements need it only when a
+ * permutation is returned (perm_out, tk_argsort) or tk_vjp has no saved row
+ * state; the plain forward pass and the VJP from state run without.  solver as
+ * in tk_opts.                                                                  */
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver);
 
 /* Forward pass (Prop. 2 with Prop. 5 / Prop. 6): out[r, :] = operator(theta[r, :]).

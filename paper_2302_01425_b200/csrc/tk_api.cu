@@ -30,6 +30,7 @@ tk_rowstate* long_workspace_state(void* workspace, long long rows, int n);
 void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
+constexpr int kMaxKeyOnlyN = 32768;  // longest row the key-only forward pass holds on chip (no workspace)
 constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers
 constexpr int kMaxWalkN = 256;       // longest row whose solve is one thread's walk (tk_rows.cu)
 
@@ -142,7 +143,10 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
     cudaError_t ed = tk::launch_dykstra(P, (cudaStream_t)stream);
     return ed == cudaSuccess ? TK_OK : TK_ERR_CUDA;
   }
-  if (n > tk::kMaxOnChipN) {
+  // Without a permutation to return, rows of up to 32768 elements are sorted (keys only) on chip and
+  // need no workspace; one that is passed is left untouched.
+  const bool key_only_on_chip = n <= tk::kMaxKeyOnlyN && P.perm_out == nullptr;
+  if (n > tk::kMaxOnChipN && !key_only_on_chip) {
     s = check_workspace(opts, rows, n);
     if (s != TK_OK) return s;
     cudaError_t el = tk::launch_long(P, opts->workspace, opts->state_out, false, (cudaStream_t)stream);
@@ -173,7 +177,11 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (opts) P.status = opts->status_out;
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(grad_out) && aligned16(grad_theta);
   cudaError_t e;
-  if (n > tk::kMaxOnChipN) {
+  if (n > tk::kMaxOnChipN && n <= tk::kMaxKeyOnlyN && opts && opts->state_out) {
+    // from saved state a row of this length is streamed by one thread block: no scratch
+    P.state_in = opts->state_out;
+    e = tk::launch_vjp_state(P, (cudaStream_t)stream);
+  } else if (n > tk::kMaxOnChipN) {
     s = check_workspace(opts, rows, n);
     if (s != TK_OK) return s;
     P.state_in = opts->state_out;

@@ -1,5 +1,8 @@
-// tk_ctav.cu -- rows of 257..16384 elements, the default forward pass and VJP: one thread block
-// per row, merge sort of the 32-bit KEYS only, results placed by value.
+// tk_ctav.cu -- rows of 513..16384 elements, the default forward pass and VJP, and the forward
+// pass of rows of up to 32768: one thread block per row, merge sort of the 32-bit KEYS only,
+// results placed by value.  With 32 keys per thread (rows above 16384) the row itself is not
+// kept in registers: the results pass reads it again (it is in L2), and the VJP is left to the
+// streaming kernel that works from the saved row state.
 //
 // Same reasoning as tk_groupv.cu: with gamma and the block edges known, the result of an element
 // depends on its key alone, so no index travels through the sort (a shared-memory slot is 4 bytes,
@@ -41,11 +44,13 @@ __device__ __forceinline__ void warp_sort_keys(float (&r)[E], int lane) {
   for (int size = 2; size <= 32; size <<= 1) {
     {
       const bool keepmax = (lane & (size >> 1)) == 0;
-      float o[E];
 #pragma unroll
-      for (int i = 0; i < E; ++i) o[i] = __shfl_xor_sync(0xffffffffu, r[E - 1 - i], size - 1);
-#pragma unroll
-      for (int i = 0; i < E; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
+      for (int i = 0; i < E / 2; ++i) {            // slot i meets the partner's slot E-1-i and vice versa
+        const float oa = __shfl_xor_sync(0xffffffffu, r[E - 1 - i], size - 1);
+        const float ob = __shfl_xor_sync(0xffffffffu, r[i], size - 1);
+        r[i] = keepmax ? fmaxf(r[i], oa) : fminf(r[i], oa);
+        r[E - 1 - i] = keepmax ? fmaxf(r[E - 1 - i], ob) : fminf(r[E - 1 - i], ob);
+      }
     }
 #pragma unroll
     for (int st = size >> 2; st >= 1; st >>= 1) {
@@ -70,6 +75,7 @@ __device__ __forceinline__ void warp_sort_keys(float (&r)[E], int lane) {
 template <int E, int MAXT>
 __global__ void __launch_bounds__(MAXT, MAXT == 512 ? 2 : 1)
 tk_ctav_kernel(const Problem P) {
+  constexpr bool KEEP = E <= 16;               // the row stays in registers for the results pass
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int T = blockDim.x;
   const int t = threadIdx.x;
@@ -89,29 +95,35 @@ tk_ctav_kernel(const Problem P) {
 
   // ---- load (striped, coalesced); x[] stays in registers for the epilogue
   const float* x_row = P.theta + row * (long long)n;
-  float x[E], s[E];
+  float x[KEEP ? E : 4], s[E];
   bool bad = false;
-  if (P.vec4) {
-    const float4* x4 = reinterpret_cast<const float4*>(x_row);
-#pragma unroll
-    for (int j = 0; j < E / 4; ++j) {
+  auto index_of = [&](int i) -> int { return P.vec4 ? 4 * ((i >> 2) * T + t) + (i & 3) : i * T + t; };
+  // the thread's elements 4 j .. 4 j + 3 (zeros past the row's end)
+  auto load4 = [&](const float* base, int j, float (&v4)[4]) {
+    if (P.vec4) {
       const int v = j * T + t;
       float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (4 * v < n) q = __ldg(x4 + v);
-      x[4 * j] = q.x; x[4 * j + 1] = q.y; x[4 * j + 2] = q.z; x[4 * j + 3] = q.w;
-    }
-  } else {
+      if (4 * v < n) q = __ldg(reinterpret_cast<const float4*>(base) + v);
+      v4[0] = q.x; v4[1] = q.y; v4[2] = q.z; v4[3] = q.w;
+    } else {
 #pragma unroll
-    for (int i = 0; i < E; ++i) { const int idx = i * T + t; x[i] = (idx < n) ? __ldg(x_row + idx) : 0.0f; }
-  }
-  auto index_of = [&](int i) -> int { return P.vec4 ? 4 * ((i >> 2) * T + t) + (i & 3) : i * T + t; };
+      for (int c4 = 0; c4 < 4; ++c4) { const int idx = (4 * j + c4) * T + t; v4[c4] = (idx < n) ? __ldg(base + idx) : 0.0f; }
+    }
+  };
   unsigned valid = 0;
 #pragma unroll
-  for (int i = 0; i < E; ++i) {
-    const bool in = index_of(i) < n;
-    valid |= in ? (1u << i) : 0u;
-    if (in && !isfinite(x[i])) bad = true;
-    s[i] = in ? sort_key(x[i], mag) : -INFINITY;          // slots past the row sort last
+  for (int j = 0; j < E / 4; ++j) {
+    float v4[4];
+    load4(x_row, j, v4);
+#pragma unroll
+    for (int c4 = 0; c4 < 4; ++c4) {
+      const int i = 4 * j + c4;
+      const bool in = index_of(i) < n;
+      valid |= in ? (1u << i) : 0u;
+      if (in && !isfinite(v4[c4])) bad = true;
+      s[i] = in ? sort_key(v4[c4], mag) : -INFINITY;      // slots past the row sort last
+      if (KEEP) x[i] = v4[c4];
+    }
   }
 
   // ---- sort of the keys: registers, the warp's 32 E keys through shuffles, then log2(T / 32)
@@ -319,6 +331,32 @@ tk_ctav_kernel(const Problem P) {
     tt = fminf(fmaxf(tq, 0.0f), wid);
     return tq >= wid ? 2 : (tq > 0.0f ? 1 : 0);
   };
+  float* o_row = P.out + row * (long long)n;
+  if constexpr (!KEEP) {
+    // forward pass only; the row is read again, four elements at a time, and stored at once
+#pragma unroll
+    for (int j = 0; j < E / 4; ++j) {
+      float v4[4], o4v[4];
+      load4(x_row, j, v4);
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float tt;
+        const float key = sort_key(v4[c4], mag);
+        const int cls = classify(key, tt);
+        float v = cls == 2 ? (mag ? M.vtop(key) : 1.0f) : (cls == 1 ? M.rho(tt) : 0.0f);
+        if (mag) v = signbit(v4[c4]) ? -v : v;
+        if (P.mode == TK_TOPK) v *= v4[c4];
+        o4v[c4] = v;
+      }
+      if (P.vec4) {
+        const int v = j * T + t;
+        if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o4v[0], o4v[1], o4v[2], o4v[3]);
+      } else {
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) { const int idx = (4 * j + c4) * T + t; if (idx < n) o_row[idx] = o4v[c4]; }
+      }
+    }
+  } else {
   float o[E];
   if (P.what == W_FWD) {
 #pragma unroll
@@ -390,7 +428,6 @@ tk_ctav_kernel(const Problem P) {
       o[i] = v;
     }
   }
-  float* o_row = P.out + row * (long long)n;
   if (P.vec4) {
     float4* o4 = reinterpret_cast<float4*>(o_row);
 #pragma unroll
@@ -402,6 +439,7 @@ tk_ctav_kernel(const Problem P) {
 #pragma unroll
     for (int i = 0; i < E; ++i) { const int idx = i * T + t; if (idx < n) o_row[idx] = o[i]; }
   }
+  }   // KEEP
   if (t == 0 && row_flags && P.status) atomicOr(P.status, row_flags);
 }
 
@@ -409,23 +447,27 @@ tk_ctav_kernel(const Problem P) {
 
 int cta_padded_length(int n);
 
+// rows of up to 16384: forward pass or recomputing VJP; up to 32768: forward pass only
 cudaError_t launch_ctav(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
   P.N = cta_padded_length(P.n);
   if (P.N < 512) P.N = 512;
-  const int E = 16;                         // one warp sorts 512 keys; T = N / 16 threads
+  const int E = P.N > 16384 ? 32 : 16;      // one warp sorts 32 E keys; T = N / E threads
+  if (E == 32 && P.what != W_FWD) return cudaErrorInvalidValue;
   const int T = P.N / E;
   const size_t smem = (size_t)(((P.N + (P.N >> PAD_SHIFT)) + 2) & ~1) * 4 + (size_t)3 * (T + 1) * 8 + 40 * 8 + 40 * 4 + 64;
   void (*kern)(const Problem) = nullptr;
   int slot;
-  if (T > 512) { kern = tk_ctav_kernel<16, 1024>; slot = 2; }
+  if (E == 32) { kern = tk_ctav_kernel<32, 1024>; slot = 0; }
+  else if (T > 512) { kern = tk_ctav_kernel<16, 1024>; slot = 2; }
   else { kern = tk_ctav_kernel<16, 512>; slot = 1; }
   static bool configured[3][64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
-    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 2) * 4 + 3 * 1025 * 8 + 40 * 8 + 40 * 4 + 64;
+    const int max_n = slot == 0 ? 32768 : 16384;
+    const int max_smem = (max_n + (max_n >> PAD_SHIFT) + 2) * 4 + 3 * 1025 * 8 + 40 * 8 + 40 * 4 + 64;
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (err != cudaSuccess) return err;
     if (dev >= 0 && dev < 64) configured[slot][dev] = true;

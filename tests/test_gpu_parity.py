@@ -134,7 +134,7 @@ def test_runs_are_bit_reproducible():
 @pytest.mark.parametrize("p", [2.0, P43])
 def test_rows_held_in_global_memory(mode, p):
     from parity import run_case
-    for n, k, lam, rows, seed in [(16385, 1638, 1.0, 3, 81), (20011, 77, 0.3, 2, 82), (40000, 4000, 1.0, 2, 83),
+    for n, k, lam, rows, seed in [(16385, 1638, 1.0, 3, 81), (20011, 77, 0.3, 2, 82), (32768, 9000, 2.0, 2, 85), (40000, 4000, 1.0, 2, 83),
                                   (70001, 35000, 0.05, 1, 84)]:
         x = rows_of(n, rows, seed)
         if seed == 82:
@@ -144,7 +144,7 @@ def test_rows_held_in_global_memory(mode, p):
 
 
 def test_long_rows_need_a_workspace():
-    n = 20000
+    n = 40000
     th = torch.zeros((1, n), device="cuda")
     out = torch.empty_like(th)
     with pytest.raises(tk.TkError) as e:
@@ -155,6 +155,22 @@ def test_long_rows_need_a_workspace():
     small = torch.empty(need - 256, dtype=torch.uint8, device="cuda")
     with pytest.raises(tk.TkError) as e:
         tk.tk_fwd_ex(th, 1, n, 10, 2.0, 1.0, tk.TK_MASK, out, workspace=small)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+    # 16384 < n <= 32768: the plain forward pass and the VJP from state run on chip without scratch;
+    # a permutation, or a VJP without saved state, still asks for it
+    n = 20000
+    th = torch.randn((2, n), device="cuda")
+    out = torch.empty_like(th)
+    st = tk.new_state(2)
+    tk.tk_fwd_ex(th, 2, n, 10, 2.0, 1.0, tk.TK_MASK, out, state_out=st)
+    tk.tk_vjp(th, th, 2, n, 10, 2.0, 1.0, tk.TK_MASK, out, state=st)
+    torch.cuda.synchronize()
+    perm = torch.empty((2, n), dtype=torch.int32, device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 2, n, 10, 2.0, 1.0, tk.TK_MASK, out, perm_out=perm)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_vjp(th, th, 2, n, 10, 2.0, 1.0, tk.TK_MASK, out)
     assert e.value.status == tk.TK_ERR_WORKSPACE
 
 
