@@ -1,7 +1,8 @@
 // tk_rows.cu -- rows of up to 256 elements, the default forward pass and VJP.
 //
 // Every warp works alone on up to 32 rows (16 when n > 64, 8 when n > 128), in three phases:
-//   1. in batches of 32/G rows (G lanes x 8 elements per row): load, sort the 32-bit KEYS by the
+//   1. in batches of 32/G rows (G lanes x 8 keys per row; one lane x 16 keys for 8 < n <= 16,
+//      where the whole network then runs in registers): load, sort the 32-bit KEYS by the
 //      shuffle network, leave the sorted row in the warp's shared memory;
 //   2. lane r solves row r: the isotonic problem of Sec. 5 has at most one pooled block [a0, b0)
 //      around ranks k-1 and k, and it is grown from that pair one rank at a time, pooling a
@@ -136,18 +137,18 @@ constexpr int kRowsThreads = 128;
 // B batches of 32/G rows per warp.  The most batches (32 rows per warp, 16 for n > 64, 8 for
 // n > 128) cost the fewest instructions per row; fewer batches give a small problem enough warps
 // to fill the machine.
-template <int G, int B>
+template <int G, int E, int B>
 struct RowsGeom {
-  static constexpr int N = 8 * G;                          // padded row length
+  static constexpr int N = E * G;                          // padded row length
   static constexpr int RPB = 32 / G;                       // rows per batch
   static constexpr int R = RPB * B;                        // rows per warp
   static constexpr int STRIDE = N | 1;                     // odd: lane r walking row r meets no bank conflict
 };
 
-template <int G, int B, bool Q4, bool MAG>
-__global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem P) {
-  constexpr int RPB = RowsGeom<G, B>::RPB, R = RowsGeom<G, B>::R, BATCHES = B;
-  constexpr int STRIDE = RowsGeom<G, B>::STRIDE;
+template <int G, int E, int B, bool Q4, bool MAG>
+__global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(const Problem P) {
+  constexpr int RPB = RowsGeom<G, E, B>::RPB, R = RowsGeom<G, E, B>::R, BATCHES = B;
+  constexpr int STRIDE = RowsGeom<G, E, B>::STRIDE;
   constexpr int WARPS = kRowsThreads / 32;
   __shared__ float sm[WARPS][R][STRIDE];
 
@@ -161,11 +162,11 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
   M.q4 = Q4; M.mag = MAG;
   int flags = 0;
 
-  // the lane's 8 consecutive elements of a row (zeros past the row's end)
-  auto load8 = [&](const float* base, bool live, float (&v)[8]) {
+  // the lane's E consecutive elements of a row (zeros past the row's end)
+  auto load8 = [&](const float* base, bool live, float (&v)[E]) {
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int e0 = 8 * lig + 4 * h;
+    for (int h = 0; h < E / 4; ++h) {
+      const int e0 = E * lig + 4 * h;
       if (P.vec4) {
         float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
         if (live && e0 < n) q = __ldg(reinterpret_cast<const float4*>(base) + (e0 >> 2));
@@ -178,30 +179,30 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
   };
 
   // ---- phase 1: sort the keys of every row, batch by batch
-  float xkeep[8];                                 // a single batch keeps its row for phase 3
+  float xkeep[E];                                 // a single batch keeps its row for phase 3
 #pragma unroll 1
   for (int b = 0; b < BATCHES; ++b) {
     const int rr = b * RPB + gw;
     const long long row = row0 + rr;
     const bool live = row < P.rows;
-    float x[8], s[8];
+    float x[E], s[E];
     load8(P.theta + (live ? row : 0) * (long long)n, live, x);
     if (BATCHES == 1) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) xkeep[i] = x[i];
+      for (int i = 0; i < E; ++i) xkeep[i] = x[i];
     }
     bool bad = false;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      const bool in = 8 * lig + i < n;
+    for (int i = 0; i < E; ++i) {
+      const bool in = E * lig + i < n;
       if (in && !isfinite(x[i])) bad = true;
       s[i] = in ? sort_key(x[i], MAG) : -INFINITY;       // slots past the row sort last
     }
     if (bad && live) flags |= TK_FLAG_NONFINITE;
-    group_sort_keys<G, 8>(s, lig, mask);
+    group_sort_keys<G, E>(s, lig, mask);
     float* sk = sm[warp][rr];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) sk[8 * lig + i] = s[i];   // rank 8 lig + i
+    for (int i = 0; i < E; ++i) sk[E * lig + i] = s[i];   // rank E lig + i
   }
   __syncwarp();
 
@@ -229,10 +230,10 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
     const float u = __shfl_sync(0xffffffffu, mine.u, rr);
     const float c = __shfl_sync(0xffffffffu, mine.c, rr);
     const int a0 = __shfl_sync(0xffffffffu, mine.a0, rr);
-    float x[8];
+    float x[E];
     if (BATCHES == 1) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) x[i] = xkeep[i];
+      for (int i = 0; i < E; ++i) x[i] = xkeep[i];
     } else {
       load8(P.theta + (live ? row : 0) * (long long)n, live, x);   // second read: L1 / L2
     }
@@ -244,10 +245,10 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
       tt = fminf(fmaxf(t, 0.0f), wid);
       return t >= wid ? 2 : (t > 0.0f ? 1 : 0);
     };
-    float o[8];
+    float o[E];
     if (P.what == W_FWD) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < E; ++i) {
         float tt;
         const float key = sort_key(x[i], MAG);
         const int cls = classify(key, tt);
@@ -258,13 +259,13 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
       }
     } else {
       // ---- VJP (Prop. 7): o_j = rho'_j (chi_j g_j - A/D) on the pooled block, by value
-      float g[8];
+      float g[E];
       load8(P.gout + (live ? row : 0) * (long long)n, live, g);
       float A = 0.f, D = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < E; ++i) {
         float tt;
-        if (has_block && 8 * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
+        if (has_block && E * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
           const float dr = M.drho(tt);
           const float chi = MAG ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
           D += dr; A += dr * chi * g[i];
@@ -278,9 +279,9 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
       // the division rounded away; rho' can be 3/lambda, and an ulp of the mean times that shows
       float A2 = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < E; ++i) {
         float tt;
-        if (has_block && 8 * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
+        if (has_block && E * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
           const float chi = MAG ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
           A2 += M.drho(tt) * fmaf(chi, g[i], -ratio);
         }
@@ -289,7 +290,7 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
       if (MAG && has_block) A2 -= (float)(k - a0) * ratio;
       const float delta = D > 0.0f ? A2 / D : 0.0f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < E; ++i) {
         float tt;
         const float key = sort_key(x[i], MAG);
         const int cls = classify(key, tt);
@@ -305,8 +306,8 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
     }
     float* o_row = P.out + (live ? row : 0) * (long long)n;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int e0 = 8 * lig + 4 * h;
+    for (int h = 0; h < E / 4; ++h) {
+      const int e0 = E * lig + 4 * h;
       if (P.vec4) {
         if (live && e0 < n) reinterpret_cast<float4*>(o_row)[e0 >> 2] = make_float4(o[4 * h], o[4 * h + 1], o[4 * h + 2], o[4 * h + 3]);
       } else {
@@ -318,30 +319,30 @@ __global__ void __launch_bounds__(kRowsThreads, 6) tk_rows_kernel(const Problem 
   if (flags && P.status) atomicOr(P.status, flags);
 }
 
-template <int G, int B>
+template <int G, int E, int B>
 cudaError_t launch_rows_gb(const Problem& P, cudaStream_t stream) {
-  const long long per_block = (long long)(kRowsThreads / 32) * RowsGeom<G, B>::R;
+  const long long per_block = (long long)(kRowsThreads / 32) * RowsGeom<G, E, B>::R;
   const unsigned blocks = (unsigned)((P.rows + per_block - 1) / per_block);
   const bool mag = P.mode == TK_TOPKMAG;
   if (P.q4) {
-    if (mag) tk_rows_kernel<G, B, true, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, B, true, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, E, B, true, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, E, B, true, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   } else {
-    if (mag) tk_rows_kernel<G, B, false, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, B, false, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, E, B, false, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, E, B, false, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   }
   return cudaGetLastError();
 }
 
 constexpr long long kWarpsToFill = 148 * 24;   // warps below which a launch leaves SMs short of work
 
-// The most batches per warp that still leave kWarpsToFill warps, out of {1, 2, BMAX}.
+// 8 keys per lane.  The most batches per warp that still leave kWarpsToFill warps, out of {1, 2, BMAX}.
 template <int G, int BMAX>
 cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
   constexpr int RPB = 32 / G;
-  if (BMAX > 2 && P.rows / (RPB * BMAX) >= kWarpsToFill) return launch_rows_gb<G, BMAX>(P, stream);
-  if (BMAX >= 2 && P.rows / (RPB * 2) >= kWarpsToFill) return launch_rows_gb<G, (BMAX >= 2 ? 2 : 1)>(P, stream);
-  return launch_rows_gb<G, 1>(P, stream);
+  if (BMAX > 2 && P.rows / (RPB * BMAX) >= kWarpsToFill) return launch_rows_gb<G, 8, BMAX>(P, stream);
+  if (BMAX >= 2 && P.rows / (RPB * 2) >= kWarpsToFill) return launch_rows_gb<G, 8, (BMAX >= 2 ? 2 : 1)>(P, stream);
+  return launch_rows_gb<G, 8, 1>(P, stream);
 }
 
 }  // namespace
@@ -349,12 +350,15 @@ cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
 // Forward pass or recomputing VJP for rows of up to 256 elements when no permutation is asked for.
 cudaError_t launch_rows(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
+  if (P.n > 8 && P.n <= 16) {                  // one lane per row, 16 keys: the whole sort in registers
+    P.N = 16;
+    return launch_rows_gb<1, 16, 1>(P, stream);
+  }
   int G = 1;
   while (G * 8 < P.n) G <<= 1;
   P.N = G * 8;
   switch (G) {
     case 1: return launch_rows_g<1, 1>(P, stream);
-    case 2: return launch_rows_g<2, 2>(P, stream);
     case 4: return launch_rows_g<4, 4>(P, stream);
     case 8: return launch_rows_g<8, 8>(P, stream);
     case 16: return launch_rows_g<16, 8>(P, stream);
