@@ -9,10 +9,9 @@ namespace tk {
 cudaError_t launch_cta(const Problem& P, cudaStream_t stream);
 int cta_padded_length(int n);
 // sub-warp row kernels for n <= 512 with the permutation (tk_group.cu); key-only sort and results
-// by value: short rows (tk_rows.cu), up to 512 (tk_groupv.cu)
+// by value for rows of up to 1024 elements (tk_rows.cu)
 cudaError_t launch_group(const Problem& P, cudaStream_t stream);
 cudaError_t launch_rows(const Problem& P, cudaStream_t stream);
-cudaError_t launch_groupv(const Problem& P, cudaStream_t stream);
 // block-per-row kernel with a key-only sort and results by value (tk_ctav.cu)
 cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
 // exact forward pass without a sort (tk_thr.cu)
@@ -31,15 +30,15 @@ void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
 constexpr int kMaxKeyOnlyN = 32768;  // longest row the key-only forward pass holds on chip (no workspace)
-constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers
-constexpr int kMaxWalkN = 256;       // longest row whose solve is one thread's walk (tk_rows.cu)
+constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers as (key, index) words
+constexpr int kMaxWalkN = 1024;      // longest row of the warp-autonomous kernel (tk_rows.cu)
 
 inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   // Without a permutation to return, short rows sort their keys only and place results by value.
   const bool needs_perm = P.perm_out != nullptr || P.sorted_out != nullptr || P.what == W_ARGSORT;
   if (!needs_perm) {
     if (P.n <= kMaxWalkN) return launch_rows(P, stream);
-    return P.n <= kMaxGroupN ? launch_groupv(P, stream) : launch_ctav(P, stream);
+    return launch_ctav(P, stream);
   }
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
 }

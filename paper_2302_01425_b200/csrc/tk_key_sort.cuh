@@ -54,6 +54,19 @@ __device__ __forceinline__ void lane_sort_f<16>(float (&r)[16]) {
   for (int i = 0; i < 8; ++i) { r[i] = hi[i]; r[i + 8] = lo[i]; }
 }
 
+template <>
+__device__ __forceinline__ void lane_sort_f<32>(float (&r)[32]) {
+  float hi[16], lo[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { hi[i] = r[i]; lo[i] = r[i + 16]; }
+  lane_sort_f<16>(hi); lane_sort_f<16>(lo);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) cef(hi[i], lo[15 - i]);     // element against its mirror: two bitonic halves
+  lane_merge_f<16>(hi); lane_merge_f<16>(lo);
+#pragma unroll
+  for (int i = 0; i < 16; ++i) { r[i] = hi[i]; r[i + 16] = lo[i]; }
+}
+
 template <int G, int E>
 __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned mask) {
   lane_sort_f<E>(r);
@@ -61,11 +74,21 @@ __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned
   for (int size = 2; size <= G; size <<= 1) {
     {
       const bool keepmax = (lig & (size >> 1)) == 0;
-      float o[E];
+      if (E <= 16) {
+        float o[E];
 #pragma unroll
-      for (int i = 0; i < E; ++i) o[i] = __shfl_xor_sync(mask, r[E - 1 - i], size - 1);
+        for (int i = 0; i < E; ++i) o[i] = __shfl_xor_sync(mask, r[E - 1 - i], size - 1);
 #pragma unroll
-      for (int i = 0; i < E; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
+        for (int i = 0; i < E; ++i) r[i] = keepmax ? fmaxf(r[i], o[i]) : fminf(r[i], o[i]);
+      } else {                                    // fewer live registers: slot i and its mirror together
+#pragma unroll
+        for (int i = 0; i < E / 2; ++i) {
+          const float oa = __shfl_xor_sync(mask, r[E - 1 - i], size - 1);
+          const float ob = __shfl_xor_sync(mask, r[i], size - 1);
+          r[i] = keepmax ? fmaxf(r[i], oa) : fminf(r[i], oa);
+          r[E - 1 - i] = keepmax ? fmaxf(r[E - 1 - i], ob) : fminf(r[E - 1 - i], ob);
+        }
+      }
     }
 #pragma unroll
     for (int st = size >> 2; st >= 1; st >>= 1) {

@@ -132,6 +132,105 @@ __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, co
   R.piv = piv; R.u = u; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = has_block ? 1 : 0;
 }
 
+// The same growth by a whole warp for one row (rows of more than 128 elements have a warp to
+// themselves): 32 candidates per step.  Lane i tests rank b + i (or a - 1 - i) against the block
+// with the i candidates before it already pooled -- its power sums are the block's plus an
+// exclusive prefix over the lanes -- which is exactly the test the one-at-a-time loop would make
+// when it got there, and the candidates that join are the leading run of passing lanes.  A side
+// is left at its first failing candidate, as in the serial loop, so the result is the same; a
+// block of m ranks costs about m/32 + 3 steps.  Block sums for the value are then taken in fp64
+// by the warp.
+template <bool Q4, bool MAG>
+__device__ __forceinline__ void solve_row_coop(const float* sk, int n, int k, const Math& M, const Problem& P,
+                                               int lane, RowSol& R) {
+  auto key = [&](int i) -> float { return sk[i]; };
+  const float c = key(k - 1);
+  const float vtop_c = M.vtop(c);
+  const bool has_block = (k < n) && (vtop_c < key(k));
+  const float piv = (MAG && vtop_c < 0.5f * c) ? 0.0f : c;   // as in solve_row_walk
+  int a0 = k, b0 = k;
+  float u = 0.0f;
+  if (has_block) {                                           // uniform over the warp
+    const float il3 = P.inv_lam * P.inv_lam * P.inv_lam;
+    const float dk = key(k) - piv, dc = c - piv;
+    float D1 = dc + dk, D2 = 0.f, D3 = 0.f;
+    if (Q4) { D2 = dc * dc + dk * dk; D3 = dc * dc * dc + dk * dk * dk; }
+    a0 = k - 1; b0 = k + 1;
+    auto excl = [&](float v) -> float {                      // exclusive prefix over the lanes
+      float inc = v;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) { const float up = __shfl_up_sync(0xffffffffu, inc, o); if (lane >= o) inc += up; }
+      return inc - v;
+    };
+    int below = 1, fails = 0;
+    while (fails < 2) {
+      const int j = below ? b0 + lane : a0 - 1 - lane;
+      const bool valid = below ? (j < n) : (j >= 0);
+      const float s = valid ? key(j) : 0.0f;
+      const float d = valid ? s - piv : 0.0f;
+      float d2 = 0.f, d3 = 0.f, x2 = 0.f, x3 = 0.f;
+      const float x1 = excl(d);
+      if (Q4) { d2 = d * d; d3 = d2 * d; x2 = excl(d2); x3 = excl(d3); }
+      // the block this candidate is tested against: the current one plus the candidates before it
+      const int a = below ? a0 : a0 - lane, b = below ? b0 + lane : b0;
+      const float cnt = (float)(b - a), m = (float)(k - a);
+      const float uu = below ? d : M.vtop(s) - piv;
+      const float S1 = D1 + x1, S2 = D2 + x2, S3 = D3 + x3;
+      float Sv;
+      if (Q4) Sv = (((-cnt * uu + 3.0f * S1) * uu - 3.0f * S2) * uu + S3) * il3;
+      else Sv = (S1 - cnt * uu) * P.inv_lam;
+      const float Hv = Sv - (MAG ? m * (piv + uu) : m);
+      const bool ok = valid && (below ? (Hv < 0.0f) : (Hv > 0.0f));
+      const unsigned bal = __ballot_sync(0xffffffffu, ok);
+      const int run = (bal == 0xffffffffu) ? 32 : __ffs(~bal) - 1;      // leading run of joining candidates
+      if (run > 0) {
+        // pool them: inclusive sums at lane run - 1
+        D1 += __shfl_sync(0xffffffffu, x1 + d, run - 1);
+        if (Q4) { D2 += __shfl_sync(0xffffffffu, x2 + d2, run - 1); D3 += __shfl_sync(0xffffffffu, x3 + d3, run - 1); }
+        if (below) b0 += run; else a0 -= run;
+        fails = 0;
+      }
+      if (run < 32) { ++fails; below ^= 1; }
+    }
+    // ---- block sums in fp64, then the block value (every lane computes the same)
+    double E1 = 0.0, E2 = 0.0, E3 = 0.0;
+    for (int i = a0 + lane; i < b0; i += 32) {
+      const double dd = (double)(key(i) - piv);
+      E1 += dd;
+      if (Q4) { const double dd2 = dd * dd; E2 += dd2; E3 = fma(dd2, dd, E3); }
+    }
+    E1 = warp_sum(E1);
+    if (Q4) { E2 = warp_sum(E2); E3 = warp_sum(E3); }
+    const double cntd = (double)(b0 - a0);
+    const double mud = E1 / cntd;
+    float M2 = 0.f, M3 = 0.f;
+    if (Q4) {
+      M2 = (float)(E2 - E1 * mud);
+      M3 = (float)(E3 - 3.0 * mud * E2 + 2.0 * mud * mud * E1);
+    }
+    u = block_value<Q4, MAG>(P.lam, P.lam3, piv, (float)cntd, (float)(k - a0), (float)mud, M2, M3);
+    u = settle_offset(M, piv, u, a0, b0, n, key);
+  }
+  R.piv = piv; R.u = u; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = has_block ? 1 : 0;
+}
+
+// Ranks that can be pooled at all: keys strictly between vtop(c) and c + width(c), c the k-th
+// largest key (two binary searches on the sorted row).  An upper bound of the block's size, used
+// to choose between the one-lane growth (cheap per member, serial) and the warp's (32 at a time).
+__device__ __forceinline__ int window_ranks(const float* sk, int n, int k, const Math& M) {
+  const float c = sk[k - 1];
+  const float lo_key = M.vtop(c), hi_key = c + M.width(c);
+  if (!(k < n) || !(lo_key < sk[k])) return 0;
+  int l = 0, r = k;                              // first rank with key < hi_key
+  while (l < r) { const int mid = (l + r) >> 1; if (sk[mid] >= hi_key) l = mid + 1; else r = mid; }
+  const int wl = l;
+  l = k; r = n;                                  // first rank with key <= lo_key
+  while (l < r) { const int mid = (l + r) >> 1; if (sk[mid] > lo_key) l = mid + 1; else r = mid; }
+  return l - wl;
+}
+
+constexpr int kSerialGrowthMax = 224;   // window above which a warp per row grows the block cooperatively
+
 constexpr int kRowsThreads = 128;
 
 // B batches of 32/G rows per warp.  The most batches (32 rows per warp, 16 for n > 64, 8 for
@@ -146,7 +245,7 @@ struct RowsGeom {
 };
 
 template <int G, int E, int B, bool Q4, bool MAG>
-__global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(const Problem P) {
+__global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) tk_rows_kernel(const Problem P) {
   constexpr int RPB = RowsGeom<G, E, B>::RPB, R = RowsGeom<G, E, B>::R, BATCHES = B;
   constexpr int STRIDE = RowsGeom<G, E, B>::STRIDE;
   constexpr int WARPS = kRowsThreads / 32;
@@ -162,41 +261,41 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(c
   M.q4 = Q4; M.mag = MAG;
   int flags = 0;
 
-  // the lane's E consecutive elements of a row (zeros past the row's end)
-  auto load8 = [&](const float* base, bool live, float (&v)[E]) {
+  // elements 4 h .. 4 h + 3 of the lane's E consecutive elements of a row (zeros past the row's end)
+  auto load4 = [&](const float* base, bool live, int h, float (&v4)[4]) {
+    const int e0 = E * lig + 4 * h;
+    if (P.vec4) {
+      float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (live && e0 < n) q = __ldg(reinterpret_cast<const float4*>(base) + (e0 >> 2));
+      v4[0] = q.x; v4[1] = q.y; v4[2] = q.z; v4[3] = q.w;
+    } else {
 #pragma unroll
-    for (int h = 0; h < E / 4; ++h) {
-      const int e0 = E * lig + 4 * h;
-      if (P.vec4) {
-        float4 q = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (live && e0 < n) q = __ldg(reinterpret_cast<const float4*>(base) + (e0 >> 2));
-        v[4 * h] = q.x; v[4 * h + 1] = q.y; v[4 * h + 2] = q.z; v[4 * h + 3] = q.w;
-      } else {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) v[4 * h + c4] = (live && e0 + c4 < n) ? __ldg(base + e0 + c4) : 0.0f;
-      }
+      for (int c4 = 0; c4 < 4; ++c4) v4[c4] = (live && e0 + c4 < n) ? __ldg(base + e0 + c4) : 0.0f;
     }
   };
 
   // ---- phase 1: sort the keys of every row, batch by batch
-  float xkeep[E];                                 // a single batch keeps its row for phase 3
+  constexpr bool KEEPX = B == 1 && E <= 16;      // a single batch keeps its row in registers for phase 3
+  float xkeep[KEEPX ? E : 1];
 #pragma unroll 1
   for (int b = 0; b < BATCHES; ++b) {
     const int rr = b * RPB + gw;
     const long long row = row0 + rr;
     const bool live = row < P.rows;
-    float x[E], s[E];
-    load8(P.theta + (live ? row : 0) * (long long)n, live, x);
-    if (BATCHES == 1) {
-#pragma unroll
-      for (int i = 0; i < E; ++i) xkeep[i] = x[i];
-    }
+    float s[E];
     bool bad = false;
 #pragma unroll
-    for (int i = 0; i < E; ++i) {
-      const bool in = E * lig + i < n;
-      if (in && !isfinite(x[i])) bad = true;
-      s[i] = in ? sort_key(x[i], MAG) : -INFINITY;       // slots past the row sort last
+    for (int h = 0; h < E / 4; ++h) {
+      float x4[4];
+      load4(P.theta + (live ? row : 0) * (long long)n, live, h, x4);
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        const int i = 4 * h + c4;
+        const bool in = E * lig + i < n;
+        if (in && !isfinite(x4[c4])) bad = true;
+        s[i] = in ? sort_key(x4[c4], MAG) : -INFINITY;   // slots past the row sort last
+        if (KEEPX) xkeep[KEEPX ? i : 0] = x4[c4];
+      }
     }
     if (bad && live) flags |= TK_FLAG_NONFINITE;
     group_sort_keys<G, E>(s, lig, mask);
@@ -209,17 +308,35 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(c
   // ---- phase 2: lane r solves row r
   RowSol mine;
   mine.piv = 0.f; mine.u = 0.f; mine.c = 0.f; mine.a0 = k; mine.b0 = k; mine.has_block = 0;
-  if (lane < R && row0 + lane < P.rows) {
-    solve_row_walk<Q4, MAG>(sm[warp][lane % R], n, k, M, P, mine);
-    if (P.state_out) {
-      tk_rowstate st;
-      st.pivot = mine.has_block ? mine.piv : mine.c; st.offset = mine.u; st.a = mine.a0; st.b = mine.b0;
-      P.state_out[row0 + lane] = st;
+  bool coop = false;
+  if (G == 32 && E >= 16) {                      // rows of more than 256 elements: blocks can be large
+    int w = 0;
+    if (lane < R && row0 + lane < P.rows) w = window_ranks(sm[warp][lane % R], n, k, M);
+    coop = __any_sync(0xffffffffu, w > kSerialGrowthMax);
+  }
+  if (coop) {
+    // the warp grows its rows one after the other, 32 candidates at a time
+#pragma unroll 1
+    for (int r = 0; r < R; ++r) {
+      if (row0 + r < P.rows) {                   // uniform over the warp
+        RowSol sol;
+        solve_row_coop<Q4, MAG>(sm[warp][r], n, k, M, P, lane, sol);
+        if (lane == r) mine = sol;
+      }
     }
+  } else if (lane < R && row0 + lane < P.rows) {
+    solve_row_walk<Q4, MAG>(sm[warp][lane % R], n, k, M, P, mine);
+  }
+  if (lane < R && row0 + lane < P.rows && P.state_out) {
+    tk_rowstate st;
+    st.pivot = mine.has_block ? mine.piv : mine.c; st.offset = mine.u; st.a = mine.a0; st.b = mine.b0;
+    P.state_out[row0 + lane] = st;
   }
   __syncwarp();
 
-  // ---- phase 3: results by value, in the original order
+  // ---- phase 3: results by value, in the original order, four elements at a time.  A launch with
+  // a single batch of up to 16 keys per lane still has the row in registers; otherwise the row is
+  // read again (L1 / L2).
 #pragma unroll 1
   for (int b = 0; b < BATCHES; ++b) {
     const int rr = b * RPB + gw;
@@ -230,13 +347,8 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(c
     const float u = __shfl_sync(0xffffffffu, mine.u, rr);
     const float c = __shfl_sync(0xffffffffu, mine.c, rr);
     const int a0 = __shfl_sync(0xffffffffu, mine.a0, rr);
-    float x[E];
-    if (BATCHES == 1) {
-#pragma unroll
-      for (int i = 0; i < E; ++i) x[i] = xkeep[i];
-    } else {
-      load8(P.theta + (live ? row : 0) * (long long)n, live, x);   // second read: L1 / L2
-    }
+    const float* x_row = P.theta + (live ? row : 0) * (long long)n;
+    float* o_row = P.out + (live ? row : 0) * (long long)n;
     const float wid = has_block ? M.width(piv + u) : 0.0f;
     // class of a key: 2 capped (top singleton), 1 pooled, 0 zero; tt = key - gamma, clamped
     auto classify = [&](float key, float& tt) -> int {
@@ -245,30 +357,96 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(c
       tt = fminf(fmaxf(t, 0.0f), wid);
       return t >= wid ? 2 : (t > 0.0f ? 1 : 0);
     };
-    float o[E];
+    auto chi_of = [&](float xv) -> float {
+      return MAG ? (signbit(xv) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? xv : 1.0f);
+    };
+    // up to 16 keys per lane: the lane's part of the row (and of the cotangent) is loaded at once
+    // and held; with 32 it is fetched chunk by chunk in every pass
+    constexpr bool HOLD = E <= 16;
+    float xall[HOLD ? E : 1], gall[HOLD ? E : 1];
+    if (HOLD) {
+#pragma unroll
+      for (int h = 0; h < E / 4; ++h) {
+        float v4[4];
+        if (KEEPX) {
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) v4[c4] = xkeep[KEEPX ? 4 * h + c4 : 0];
+        } else {
+          load4(x_row, live, h, v4);
+        }
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) xall[HOLD ? 4 * h + c4 : 0] = v4[c4];
+      }
+      if (P.what != W_FWD) {
+#pragma unroll
+        for (int h = 0; h < E / 4; ++h) {
+          float v4[4];
+          load4(P.gout + (live ? row : 0) * (long long)n, live, h, v4);
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) gall[HOLD ? 4 * h + c4 : 0] = v4[c4];
+        }
+      }
+    }
+    auto x4_of = [&](int h, float (&v4)[4]) {
+      if (HOLD) {
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) v4[c4] = xall[HOLD ? 4 * h + c4 : 0];
+      } else {
+        load4(x_row, live, h, v4);
+      }
+    };
+    auto g4_of = [&](const float* g_row, int h, float (&v4)[4]) {
+      if (HOLD) {
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) v4[c4] = gall[HOLD ? 4 * h + c4 : 0];
+      } else {
+        load4(g_row, live, h, v4);
+      }
+    };
+    auto store4 = [&](int h, const float (&o4)[4]) {
+      const int e0 = E * lig + 4 * h;
+      if (P.vec4) {
+        if (live && e0 < n) reinterpret_cast<float4*>(o_row)[e0 >> 2] = make_float4(o4[0], o4[1], o4[2], o4[3]);
+      } else {
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) if (live && e0 + c4 < n) o_row[e0 + c4] = o4[c4];
+      }
+    };
     if (P.what == W_FWD) {
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        float tt;
-        const float key = sort_key(x[i], MAG);
-        const int cls = classify(key, tt);
-        float v = cls == 2 ? (MAG ? M.vtop(key) : 1.0f) : (cls == 1 ? M.rho(tt) : 0.0f);
-        if (MAG) v = signbit(x[i]) ? -v : v;
-        if (P.mode == TK_TOPK) v *= x[i];
-        o[i] = v;
+      for (int h = 0; h < E / 4; ++h) {
+        float x4[4], o4[4];
+        x4_of(h, x4);
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float tt;
+          const float key = sort_key(x4[c4], MAG);
+          const int cls = classify(key, tt);
+          float v = cls == 2 ? (MAG ? M.vtop(key) : 1.0f) : (cls == 1 ? M.rho(tt) : 0.0f);
+          if (MAG) v = signbit(x4[c4]) ? -v : v;
+          if (P.mode == TK_TOPK) v *= x4[c4];
+          o4[c4] = v;
+        }
+        store4(h, o4);
       }
     } else {
       // ---- VJP (Prop. 7): o_j = rho'_j (chi_j g_j - A/D) on the pooled block, by value
-      float g[E];
-      load8(P.gout + (live ? row : 0) * (long long)n, live, g);
+      const float* g_row = P.gout + (live ? row : 0) * (long long)n;
       float A = 0.f, D = 0.f;
+      if (has_block) {
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        float tt;
-        if (has_block && E * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
-          const float dr = M.drho(tt);
-          const float chi = MAG ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
-          D += dr; A += dr * chi * g[i];
+        for (int h = 0; h < E / 4; ++h) {
+          float x4[4], g4[4];
+          x4_of(h, x4);
+          g4_of(g_row, h, g4);
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            float tt;
+            if (E * lig + 4 * h + c4 < n && classify(sort_key(x4[c4], MAG), tt) == 1) {
+              const float dr = M.drho(tt);
+              D += dr; A += dr * chi_of(x4[c4]) * g4[c4];
+            }
+          }
         }
       }
       A = group_sum<G, float>(A, mask);
@@ -278,41 +456,43 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : 4) tk_rows_kernel(c
       // second pass: residuals about the fp32 mean (one fma each, no cancellation) restore what
       // the division rounded away; rho' can be 3/lambda, and an ulp of the mean times that shows
       float A2 = 0.f;
+      if (has_block) {
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        float tt;
-        if (has_block && E * lig + i < n && classify(sort_key(x[i], MAG), tt) == 1) {
-          const float chi = MAG ? (signbit(x[i]) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x[i] : 1.0f);
-          A2 += M.drho(tt) * fmaf(chi, g[i], -ratio);
+        for (int h = 0; h < E / 4; ++h) {
+          float x4[4], g4[4];
+          x4_of(h, x4);
+          g4_of(g_row, h, g4);
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            float tt;
+            if (E * lig + 4 * h + c4 < n && classify(sort_key(x4[c4], MAG), tt) == 1)
+              A2 += M.drho(tt) * fmaf(chi_of(x4[c4]), g4[c4], -ratio);
+          }
         }
       }
       A2 = group_sum<G, float>(A2, mask);
       if (MAG && has_block) A2 -= (float)(k - a0) * ratio;
       const float delta = D > 0.0f ? A2 / D : 0.0f;
 #pragma unroll
-      for (int i = 0; i < E; ++i) {
-        float tt;
-        const float key = sort_key(x[i], MAG);
-        const int cls = classify(key, tt);
-        const float sgn = (MAG && signbit(x[i])) ? -1.0f : 1.0f;
-        const float chi = MAG ? sgn : (P.mode == TK_TOPK ? x[i] : 1.0f);
-        float v = 0.0f;
-        if (cls == 1) v = M.drho(tt) * (fmaf(chi, g[i], -ratio) - delta);
-        else if (cls == 2 && MAG) v = chi * g[i] * M.top_slope(key);
-        v *= sgn;
-        if (P.mode == TK_TOPK) v += g[i] * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));
-        o[i] = v;
-      }
-    }
-    float* o_row = P.out + (live ? row : 0) * (long long)n;
+      for (int h = 0; h < E / 4; ++h) {
+        float x4[4], g4[4], o4[4];
+        x4_of(h, x4);
+        g4_of(g_row, h, g4);
 #pragma unroll
-    for (int h = 0; h < E / 4; ++h) {
-      const int e0 = E * lig + 4 * h;
-      if (P.vec4) {
-        if (live && e0 < n) reinterpret_cast<float4*>(o_row)[e0 >> 2] = make_float4(o[4 * h], o[4 * h + 1], o[4 * h + 2], o[4 * h + 3]);
-      } else {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) if (live && e0 + c4 < n) o_row[e0 + c4] = o[4 * h + c4];
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float tt;
+          const float key = sort_key(x4[c4], MAG);
+          const int cls = classify(key, tt);
+          const float sgn = (MAG && signbit(x4[c4])) ? -1.0f : 1.0f;
+          const float chi = chi_of(x4[c4]);
+          float v = 0.0f;
+          if (cls == 1) v = M.drho(tt) * (fmaf(chi, g4[c4], -ratio) - delta);
+          else if (cls == 2 && MAG) v = chi * g4[c4] * M.top_slope(key);
+          v *= sgn;
+          if (P.mode == TK_TOPK) v += g4[c4] * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));
+          o4[c4] = v;
+        }
+        store4(h, o4);
       }
     }
   }
@@ -347,12 +527,23 @@ cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
 
 }  // namespace
 
-// Forward pass or recomputing VJP for rows of up to 256 elements when no permutation is asked for.
+// Forward pass or recomputing VJP for rows of up to 1024 elements when no permutation is asked for.
 cudaError_t launch_rows(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
   if (P.n > 8 && P.n <= 16) {                  // one lane per row, 16 keys: the whole sort in registers
     P.N = 16;
     return launch_rows_gb<1, 16, 1>(P, stream);
+  }
+  if (P.n > 512) {                             // one warp per row, 32 keys per lane, up to 2 rows per warp
+    P.N = 1024;
+    if (P.rows / 2 >= kWarpsToFill) return launch_rows_gb<32, 32, 2>(P, stream);
+    return launch_rows_gb<32, 32, 1>(P, stream);
+  }
+  if (P.n > 256) {                             // one warp per row, 16 keys per lane, up to 4 rows per warp
+    P.N = 512;
+    if (P.rows / 4 >= kWarpsToFill) return launch_rows_gb<32, 16, 4>(P, stream);
+    if (P.rows / 2 >= kWarpsToFill) return launch_rows_gb<32, 16, 2>(P, stream);
+    return launch_rows_gb<32, 16, 1>(P, stream);
   }
   int G = 1;
   while (G * 8 < P.n) G <<= 1;
