@@ -1,10 +1,10 @@
-// tk_ctav.cu -- rows of 513..16384 elements, the default forward pass and VJP, and the forward
+// tk_ctav.cu -- rows of 1025..16384 elements, the default forward pass and VJP, and the forward
 // pass of rows of up to 32768: one thread block per row, merge sort of the 32-bit KEYS only,
 // results placed by value.  With 32 keys per thread (rows above 16384) the row itself is not
 // kept in registers: the results pass reads it again (it is in L2), and the VJP is left to the
 // streaming kernel that works from the saved row state.
 //
-// Same reasoning as tk_groupv.cu: with gamma and the block edges known, the result of an element
+// Same reasoning as tk_rows.cu: with gamma and the block edges known, the result of an element
 // depends on its key alone, so no index travels through the sort (a shared-memory slot is 4 bytes,
 // a comparison one instruction), nothing is scattered, and every thread stores where it loaded.
 // The isotonic solve on the sorted keys is the one of tk_cta.cu (Sec. 5, App. A.6).

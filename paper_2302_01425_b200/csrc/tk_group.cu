@@ -8,7 +8,7 @@
 //   solve (G-ary search on the monotone predicates, O(1) probes through prefix
 //   sums staged in shared memory) -> dual map -> scatter through shared memory
 //   -> coalesced store.  Used when the caller wants the permutation (perm_out, tk_argsort);
-//   the default forward pass and every VJP sort the keys alone (tk_rows.cu, tk_groupv.cu).
+//   the default forward pass and every VJP sort the keys alone (tk_rows.cu).
 #include "tk_common.cuh"
 #include "tk_group_sort.cuh"
 
