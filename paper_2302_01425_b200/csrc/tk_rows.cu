@@ -1,18 +1,21 @@
-// tk_rows.cu -- rows of up to 256 elements, the default forward pass and VJP.
+// tk_rows.cu -- rows of up to 1024 elements, the default forward pass and VJP.
 //
-// Every warp works alone on up to 32 rows (16 when n > 64, 8 when n > 128), in three phases:
-//   1. in batches of 32/G rows (G lanes x 8 keys per row; one lane x 16 keys for 8 < n <= 16,
-//      where the whole network then runs in registers): load, sort the 32-bit KEYS by the
-//      shuffle network, leave the sorted row in the warp's shared memory;
-//   2. lane r solves row r: the isotonic problem of Sec. 5 has at most one pooled block [a0, b0)
-//      around ranks k-1 and k, and it is grown from that pair one rank at a time, pooling a
-//      neighbour while it violates the order, on running power sums of d = key - pivot (see
-//      solve_row_walk).  Up to 32 rows walk side by side, so the solve costs a warp a few
-//      instructions per block member instead of a search replicated over the G lanes of every row;
+// Every warp works alone on its rows (up to 32 of them for n <= 64, one warp per row with 1 to 8
+// rows per warp for n > 128), in three phases:
+//   1. in batches of 32/G rows (G lanes per row with 8 keys each up to n = 256, a warp per row with
+//      16 or 32 keys per lane above; one lane with 16 keys for 8 < n <= 16, where the whole
+//      network runs in registers): load, sort the 32-bit KEYS by the shuffle network, leave the
+//      sorted row in the warp's shared memory;
+//   2. the isotonic problem of Sec. 5 has at most one pooled block [a0, b0) around ranks k-1 and
+//      k, and it is grown from that pair, pooling a neighbour while it violates the order, on
+//      running power sums of d = key - pivot.  Lane r grows row r one rank at a time
+//      (solve_row_walk): up to 32 rows side by side, a few instructions per block member, instead
+//      of a search replicated over the lanes of every row.  A warp that owns whole rows whose
+//      window is wide grows them together, 32 candidates per step (solve_row_coop);
 //   3. in the same batches: the results by value (given gamma and the cap width, the output and
 //      the VJP of an element depend on its own key alone), stored where they were loaded.
 // No index travels through the sort and nothing is scattered; the phases are separated by warp
-// barriers only, so the other warps of the SM fill the latency of a warp that is walking.
+// barriers only, so the other warps of the SM fill the latency of a warp that is growing a block.
 // The block value is solved in fp32 about the block mean (App. A.6 cubic in depressed form).
 #include "tk_common.cuh"
 #include "tk_group_sort.cuh"
