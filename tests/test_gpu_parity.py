@@ -250,6 +250,16 @@ def test_short_row_kernel_every_batch_count():
         x = rows_of(n, rows, 300 + i)
         g = wl.cotangent_like(x, 300 + i)
         run_case(x, k, p, lam, modes[i % 3], g, label=f"n={n} rows={rows} k={k} lam={lam} p={p}")
+    # a warp per row (16 or 32 keys per lane), 1, 2 or 4 rows per warp; narrow windows grow the block
+    # on one lane, wide ones (large lambda) on the whole warp
+    wide = [(300, 15001, 0.05), (400, 4001, 5.0), (512, 8001, 3.0), (512, 15001, 20.0),
+            (700, 3001, 4.0), (1024, 7201, 0.2), (1000, 7201, 10.0), (513, 3001, 1.0)]
+    for i, (n, rows, lam) in enumerate(wide):
+        p = 2.0 if i % 2 == 0 else P43
+        k = max(1, n // (2 + i % 5))
+        x = rows_of(n, rows, 400 + i)
+        g = wl.cotangent_like(x, 400 + i)
+        run_case(x, k, p, lam, modes[i % 3], g, label=f"n={n} rows={rows} k={k} lam={lam} p={p}")
 
 
 def test_sweep_n32768_sampled_rows():
