@@ -57,21 +57,28 @@ tk_status check_workspace(const tk_opts* opts, int64_t rows, int64_t n) {
   return TK_OK;
 }
 
-// q = p/(p-1) must be 2 or 4 (p = 2 or p = 4/3).
-tk_status classify_p(double p, int* q4) {
+// q = p/(p-1): 2 and 4 (p = 2, p = 4/3) have closed-form block solves and run everywhere.  Any
+// other 1 < p <= 1.5 (q >= 3) is *qm1 = q - 1 > 0: forward pass by the sort-free solver, VJP from
+// saved state.  Not supported: q < 2 (p > 2: rho' unbounded at 0) and 2 < q < 3 (rho'' unbounded at
+// 0: an fp32 key difference cannot carry the VJP of a barely pooled element to 1e-5).
+tk_status classify_p(double p, int* q4, double* qm1) {
+  *q4 = 0; *qm1 = 0.0;
   if (!(p > 1.0) || !isfinite(p)) return TK_ERR_INVALID_ARG;
   double q = p / (p - 1.0);
-  if (fabs(q - 2.0) <= 1e-6) { *q4 = 0; return TK_OK; }
+  if (fabs(q - 2.0) <= 1e-6) return TK_OK;
   if (fabs(q - 4.0) <= 1e-6) { *q4 = 1; return TK_OK; }
-  return TK_ERR_UNSUPPORTED;
+  if (!(q >= 3.0 - 1e-9) || q > 64.0) return TK_ERR_UNSUPPORTED;
+  *qm1 = q - 1.0;
+  return TK_OK;
 }
 
 tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, double p,
-                       double lambda, int mode, int* q4) {
+                       double lambda, int mode, int* q4, double* qm1) {
   if (rows < 0 || n < 1 || k < 1 || k > n) return TK_ERR_INVALID_ARG;
   if (mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
   if (!(lambda > 0.0) || !isfinite(lambda)) return TK_ERR_INVALID_ARG;
-  tk_status s = classify_p(p, q4);
+  tk_status s = classify_p(p, q4, qm1);
+  if (s == TK_OK && *qm1 > 0.0 && (mode == TK_TOPKMAG || n > tk::kMaxOnChipN)) s = TK_ERR_UNSUPPORTED;
   if (s != TK_OK) return s;
   if (rows > 0 && theta == nullptr) return TK_ERR_INVALID_ARG;
   if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
@@ -79,10 +86,10 @@ tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, do
 }
 
 void fill(tk::Problem& P, const float* theta, int64_t rows, int64_t n, int64_t k, int q4,
-          double lambda, int mode) {
+          double qm1, double lambda, int mode) {
   P = tk::Problem{};
   P.theta = theta;
-  P.rows = rows; P.n = (int)n; P.k = (int)k; P.q4 = q4; P.mode = mode;
+  P.rows = rows; P.n = (int)n; P.k = (int)k; P.q4 = q4; P.qm1 = (float)qm1; P.mode = mode;
   P.lam = (float)lambda;
   P.inv_lam = (float)(1.0 / lambda);
   P.lam3 = (float)(lambda * lambda * lambda);
@@ -115,14 +122,19 @@ size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode
 tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
                     double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
   int q4 = 0;
-  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4);
+  double qm1 = 0.0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4, &qm1);
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
   if (out == nullptr) return TK_ERR_INVALID_ARG;
   int solver = opts ? opts->solver : TK_SOLVER_AUTO;
   if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_THRESHOLD) return TK_ERR_INVALID_ARG;
+  if (qm1 > 0.0) {                 // general p: only the sort-free solver has no closed form to rely on
+    if (solver == TK_SOLVER_PAV || solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
+    solver = TK_SOLVER_THRESHOLD;
+  }
   tk::Problem P;
-  fill(P, theta, rows, n, k, q4, lambda, mode);
+  fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.out = out;
   P.what = tk::W_FWD;
   if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
@@ -164,12 +176,14 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
                  double p, double lambda, int mode, float* grad_theta, const tk_opts* opts,
                  tk_stream stream) {
   int q4 = 0;
-  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4);
+  double qm1 = 0.0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4, &qm1);
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
   if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
+  if (qm1 > 0.0 && !(opts && opts->state_out)) return TK_ERR_UNSUPPORTED;   // general p: from saved state only
   tk::Problem P;
-  fill(P, theta, rows, n, k, q4, lambda, mode);
+  fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.gout = grad_out;
   P.out = grad_theta;
   P.what = tk::W_VJP;
@@ -209,7 +223,7 @@ tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int3
   if (theta == nullptr || perm_out == nullptr) return TK_ERR_INVALID_ARG;
   if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
   tk::Problem P;
-  fill(P, theta, rows, n, 1, 0, 1.0, mode);
+  fill(P, theta, rows, n, 1, 0, 0.0, 1.0, mode);
   P.what = tk::W_ARGSORT;
   P.perm_out = perm_out;
   P.sorted_out = sorted_out;

@@ -31,6 +31,7 @@ struct Problem {
   int n, k;
   int N;                    // padded row length held on chip
   int q4;                   // 1: q = 4 (p = 4/3); 0: q = 2
+  float qm1;                // q - 1 for any other q > 2 (sort-free solver and VJP from state only), else 0
   int mode;                 // tk_mode
   int what;                 // What
   int vec4;                 // rows may be accessed as float4
@@ -96,14 +97,18 @@ __device__ __forceinline__ unsigned long long sel64(bool c, unsigned long long x
 // ---------------------------------------------------------------- scalar math
 struct Math {
   float lam, inv_lam, lam3;
+  float qm1;          // q - 1 when gen
   bool q4, mag;
+  bool gen;           // q is neither 2 nor 4: rho(t) = (t/lam)^(q-1) through powf (t >= 0 here)
 
   __device__ __forceinline__ float rho(float t) const {
     float a = t * inv_lam;
+    if (gen) return powf(a, qm1);
     return q4 ? a * a * a : a;
   }
   __device__ __forceinline__ float drho(float t) const {
     float a = t * inv_lam;
+    if (gen) return qm1 * powf(a, qm1 - 1.0f) * inv_lam;
     return q4 ? 3.0f * a * a * inv_lam : inv_lam;
   }
   // z >= 0 with z^3 + lam z = s (s >= 0): z = (s - v)/lam at the minimiser v of
@@ -150,6 +155,13 @@ __device__ __forceinline__ Math make_math(const Problem& P) {
   Math m;
   m.lam = P.lam; m.inv_lam = P.inv_lam; m.lam3 = P.lam3;
   m.q4 = P.q4 != 0; m.mag = P.mode == TK_TOPKMAG;
+  m.qm1 = P.qm1; m.gen = P.qm1 > 0.0f;
+  return m;
+}
+// for the kernels that only ever see q = 2 or q = 4: the general branch folds away
+__device__ __forceinline__ Math make_math_q24(const Problem& P) {
+  Math m = make_math(P);
+  m.gen = false;
   return m;
 }
 

@@ -35,7 +35,7 @@ tk_cta_kernel(const Problem P) {
   const int t = threadIdx.x;
   const int n = P.n, k = P.k, N = P.N;
   const long long row = blockIdx.x;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const bool mag = M.mag;
 
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);   // pad(N) slots

@@ -81,7 +81,7 @@ tk_ctav_kernel(const Problem P) {
   const int t = threadIdx.x;
   const int n = P.n, k = P.k, N = P.N;
   const long long row = blockIdx.x;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const bool mag = M.mag;
 
   float* keys = reinterpret_cast<float*>(smem_raw);                              // pad(N) + 1 sorted keys

@@ -159,7 +159,7 @@ __global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) 
   constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
   const unsigned mask = kGroupBits << ((tid & 31) / G * G);
   const int n = P.n;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const float* x_row = P.theta + row * (long long)n;
   unsigned long long r[EPL];
   bool bad = false;
@@ -200,7 +200,7 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int T = blockDim.x, t = threadIdx.x, n = P.n, N = P.N;
   const long long row = blockIdx.x;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
   float* stage = reinterpret_cast<float*>(smem_raw);
   float* xch = reinterpret_cast<float*>(keys + pad(N) + 1);   // T + 2 floats

@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(128, EPL == 8 ? 8 : 3) tk_group_kernel(const P
   constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
   const unsigned mask = kGroupBits << ((tid & 31) / G * G);
   const int n = P.n, k = P.k;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const bool mag = M.mag;
   float* sk = sm[grp][0];
   float* p1 = sm[grp][1];

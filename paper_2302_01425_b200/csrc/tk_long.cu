@@ -282,7 +282,7 @@ __global__ void __launch_bounds__(TPB) long_prefix_kernel(const Problem P, LongW
   const int tile = blockIdx.x;
   const long long row = blockIdx.y;
   const int n = P.n, k = P.k;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const uint32_t* skeys = ws.keyB + row * (long long)n;
   const RowSetup S = row_setup(M, skeys, n, k);
   if (!S.has_block) return;
@@ -350,7 +350,7 @@ __global__ void __launch_bounds__(1024) long_solve_kernel(const Problem P, LongW
   __shared__ float sh_u;
   const long long row = blockIdx.x;
   const int n = P.n, k = P.k, t = threadIdx.x, T = blockDim.x;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const bool mag = M.mag;
   const uint32_t* skeys = ws.keyB + row * (long long)n;
   const RowSetup S = row_setup(M, skeys, n, k);
@@ -511,7 +511,7 @@ __global__ void __launch_bounds__(256) long_map_kernel(const Problem P, LongWs w
   const int n = P.n;
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const tk_rowstate st = state[row];
   const bool has_block = st.b > st.a;
   const long long base = row * (long long)n;
@@ -536,7 +536,7 @@ __global__ void __launch_bounds__(256) long_map_kernel(const Problem P, LongWs w
 __global__ void __launch_bounds__(256) long_map_value_kernel(const Problem P, const tk_rowstate* state) {
   const long long row = blockIdx.y;
   const int n = P.n;
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const tk_rowstate st = state[row];
   const bool has_block = st.b > st.a;
   const float wid = has_block ? M.width(st.pivot + st.offset) : 0.0f;

@@ -260,7 +260,7 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) 
   const unsigned mask = kGroupBits << (gw * G);
   const long long row0 = ((long long)blockIdx.x * WARPS + warp) * R;
   const int n = P.n, k = P.k;
-  Math M = make_math(P);
+  Math M = make_math_q24(P);
   M.q4 = Q4; M.mag = MAG;
   int flags = 0;
 

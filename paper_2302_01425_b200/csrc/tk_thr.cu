@@ -26,6 +26,7 @@ namespace {
 struct Sums {
   int ct, cm;          // capped (top) and strictly-inside counts
   float s1, s2, s3;    // sums of t, t^2, t^3 over the inside keys, t = key - tau
+                       // (any other q: s1 = sum rho(t), s2 = sum rho'(t))
 };
 
 // block-wide sum of the five accumulators; result in every thread.  red: 5 x 32 floats
@@ -81,8 +82,11 @@ __device__ __forceinline__ float solve_piece_cubic(bool mag, float lam3, float g
   return u;
 }
 
-template <int E, int MAXT, bool Q4, bool MAG>
+// QM: 0 for q = 2, 1 for q = 4 (closed-form / cubic solve of every candidate set), 2 for any other
+// q > 2 (Sec. 7, sensitivity to p: one Newton step on the candidate set's equation per pass).
+template <int E, int MAXT, int QM, bool MAG>
 __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
+  constexpr bool Q4 = QM == 1, GEN = QM == 2;
   __shared__ int whist[MAXT / 32][256];   // per-warp digit counts (no contention between warps)
   __shared__ int hist[256];
   __shared__ float red[160];
@@ -91,7 +95,7 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
   const int n = P.n, k = P.k;
   const long long row = blockIdx.x;
   Math M = make_math(P);
-  M.q4 = Q4; M.mag = MAG;                       // compile-time constants from here on
+  M.q4 = Q4; M.mag = MAG; M.gen = GEN;          // compile-time constants from here on
   constexpr bool mag = MAG;
   const float* x_row = P.theta + row * (long long)n;
   float x[E];
@@ -215,21 +219,27 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
         const bool top = tt >= w;
         const bool mid = tt > 0.0f && !top;
         acc.ct += top; acc.cm += mid;
-        if (mid) { acc.s1 += tt; if (M.q4) { const float t2 = tt * tt; acc.s2 += t2; acc.s3 += t2 * tt; } }
+        if (mid) {
+          if (GEN) { acc.s1 += M.rho(tt); acc.s2 += M.drho(tt); }
+          else { acc.s1 += tt; if (M.q4) { const float t2 = tt * tt; acc.s2 += t2; acc.s3 += t2 * tt; } }
+        }
       }
-      const Sums S = block_reduce(acc, red, M.q4);
+      const Sums S = block_reduce(acc, red, Q4 || GEN);
       // every thread runs the same scalar logic on the same numbers
       const int m = k - S.ct;                  // inside keys that must carry weight
       float Fv;                                // sign of F(gamma)
       if (S.cm == 0) Fv = (float)(S.ct - k);
       else {
-        const float rs = M.q4 ? S.s3 * (P.inv_lam * P.inv_lam * P.inv_lam) : S.s1 * P.inv_lam;
+        const float rs = GEN ? S.s1 : (M.q4 ? S.s3 * (P.inv_lam * P.inv_lam * P.inv_lam) : S.s1 * P.inv_lam);
         Fv = (float)(S.ct - k) + (mag ? rs / gam : rs);
       }
       float du = 0.0f;
       bool have_cand = false;
       if (S.cm > 0 && m >= 1) {
-        if (M.q4) {
+        if (GEN) {
+          // Newton on sum rho(t_i - du) = m about du = 0 (the sums are taken at the current gamma)
+          du = S.s2 > 0.0f ? (S.s1 - (float)m) / S.s2 : 0.0f;
+        } else if (M.q4) {
           du = solve_piece_cubic(mag, P.lam3, gam, (float)S.cm, (float)m, S.s1, S.s2, S.s3);
         } else {
           const float fm = (float)m, fc = (float)S.cm;
@@ -259,6 +269,32 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
       }
     }
     if (!done) flags |= TK_FLAG_NOT_CONVERGED;
+    {
+      // The block is what the FINAL offset classifies as pooled: the row state then agrees, rank for
+      // rank, with the by-value classes of the results pass below and of the VJP from state.  The
+      // last step, however small, can carry an edge key across gamma or across the cap (a pooled key
+      // whose rho is 1 - 1e-7 sits a few 1e-9 inside the cap): when the classes at the final offset
+      // are not the set that was solved, the offset moves by single ulps towards it, a few times.
+      const int want_ct = a0, want_all = b0;
+#pragma unroll 1
+      for (int tries = 0; tries < 5; ++tries) {
+        const float w = M.width(piv + off);
+        int ct = 0, cm = 0;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+          const float tt = (key[i] - piv) - off;
+          const bool top = tt >= w;
+          ct += top; cm += (tt > 0.0f && !top);
+        }
+        Sums acc{ct, cm, 0.f, 0.f, 0.f};
+        const Sums S = block_reduce(acc, red, false);
+        a0 = S.ct; b0 = S.ct + S.cm;
+        const bool up = a0 > want_ct || b0 > want_all;        // a key too many reads capped / pooled
+        const bool down = a0 < want_ct || b0 < want_all;
+        if (up == down || tries == 4 || !done) break;
+        off = nextafterf(off, up ? INFINITY : -INFINITY);
+      }
+    }
     if (b0 <= a0) { a0 = k; b0 = k; }              // degenerate end of the bracket search: treat as no block
   }
   const bool block = b0 > a0;
@@ -314,13 +350,14 @@ cudaError_t launch_thr(const Problem& P0, cudaStream_t stream) {
   const int E = N >= 4096 ? 16 : (N >= 1024 ? 8 : 4);
   const int T = N / E;
   const dim3 grid((unsigned)P.rows);
-  const bool q4 = P.q4 != 0, mag = P.mode == TK_TOPKMAG;
+  const bool q4 = P.q4 != 0, mag = P.mode == TK_TOPKMAG, gen = P.qm1 > 0.0f;
 #define TK_THR_LAUNCH(EE, MT)                                                        \
   do {                                                                               \
-    if (q4 && mag) tk_thr_kernel<EE, MT, true, true><<<grid, T, 0, stream>>>(P);      \
-    else if (q4) tk_thr_kernel<EE, MT, true, false><<<grid, T, 0, stream>>>(P);       \
-    else if (mag) tk_thr_kernel<EE, MT, false, true><<<grid, T, 0, stream>>>(P);      \
-    else tk_thr_kernel<EE, MT, false, false><<<grid, T, 0, stream>>>(P);              \
+    if (gen) tk_thr_kernel<EE, MT, 2, false><<<grid, T, 0, stream>>>(P);              \
+    else if (q4 && mag) tk_thr_kernel<EE, MT, 1, true><<<grid, T, 0, stream>>>(P);    \
+    else if (q4) tk_thr_kernel<EE, MT, 1, false><<<grid, T, 0, stream>>>(P);          \
+    else if (mag) tk_thr_kernel<EE, MT, 0, true><<<grid, T, 0, stream>>>(P);          \
+    else tk_thr_kernel<EE, MT, 0, false><<<grid, T, 0, stream>>>(P);                  \
   } while (0)
   switch (E) {
     case 4: TK_THR_LAUNCH(4, 128); break;

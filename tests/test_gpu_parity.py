@@ -369,3 +369,36 @@ def test_sort_free_solver_ties_outliers_and_limits():
         tk.tk_fwd_ex(th, 10, 300, 30, 2.0, 1.0, tk.TK_MASK, torch.empty_like(th), solver=tk.TK_SOLVER_THRESHOLD,
                      perm_out=torch.empty((10, 300), dtype=torch.int32, device="cuda"))
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK])
+@pytest.mark.parametrize("p", [1.5, 1.2, 1.1])
+def test_general_p_matches_oracle(mode, p):
+    """p other than 2 and 4/3 (q = 3, 6, 11): forward pass by the sort-free solver, VJP from state."""
+    from parity import run_case
+    for n, k, lam, rows, seed in [(64, 2, 0.3, 1024, 501), (300, 40, 1.0, 32, 502), (1000, 5, 0.5, 16, 503),
+                                  (5000, 700, 2.0, 3, 504), (16384, 2048, 1.0, 2, 505)]:
+        x = rows_of(n, rows, seed)
+        g = wl.cotangent_like(x, seed)
+        res = run_case(x, k, p, lam, mode, g, label=f"p={p} n={n} k={k} lam={lam} mode={mode}",
+                       solver=tk.TK_SOLVER_THRESHOLD)
+        assert "vjp_state_max_rel" in res
+
+
+def test_general_p_limits():
+    th = torch.randn((4, 64), device="cuda")
+    out = torch.empty_like(th)
+    tk.tk_fwd(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out)                     # solver AUTO: routed to the sort-free solver
+    ref = torch.empty_like(th)
+    tk.tk_fwd_ex(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, ref, solver=tk.TK_SOLVER_THRESHOLD)
+    torch.cuda.synchronize()
+    assert torch.equal(out, ref)
+    for kwargs in ({"solver": tk.TK_SOLVER_PAV}, {"solver": tk.TK_SOLVER_DYKSTRA},
+                   {"perm_out": torch.empty((4, 64), dtype=torch.int32, device="cuda")}):
+        with pytest.raises(tk.TkError) as e:
+            tk.tk_fwd_ex(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out, **kwargs)
+        assert e.value.status == tk.TK_ERR_UNSUPPORTED
+    for p_bad in (3.0, 1.8):                                               # q < 2; 2 < q < 3
+        with pytest.raises(tk.TkError) as e:
+            tk.tk_fwd(th, 4, 64, 2, p_bad, 1.0, tk.TK_MASK, out)
+        assert e.value.status == tk.TK_ERR_UNSUPPORTED
