@@ -332,6 +332,10 @@ def main():
                         if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
                             entry["dykstra_forward_10_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
+                        if name in ("sweep_n64", "sweep_n4096"):
+                            # p = 1.5 (q = 3): no closed-form block solve, sort-free solver with Newton steps
+                            entry["general_p_1.5_forward"] = time_solver_forward(
+                                name, dev, tk, torch, tk.TK_SOLVER_THRESHOLD, p_override=1.5)
                         ncase = workload_cases(name)[0].n
                         if 512 <= ncase <= 16384:
                             # the same exact result without the sort (solver = TK_SOLVER_THRESHOLD),
@@ -355,11 +359,15 @@ def main():
         dist.destroy_process_group()
 
 
-def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3):
+def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, p_override=None):
     """Forward pass through another solver path (alternating projections with a fixed number of
-    sweeps, or the sort-free exact solver), per variant."""
+    sweeps, or the sort-free exact solver; p_override: another p on the first variant), per variant."""
     out = []
-    for c in workload_cases(workload):
+    cases = workload_cases(workload)
+    if p_override is not None:
+        import dataclasses
+        cases = [dataclasses.replace(cases[0], p=p_override)]
+    for c in cases:
         th = torch.from_numpy(c.theta()).to(dev)
         y = torch.empty_like(th)
         st = tk.new_state(c.rows, dev) if solver == tk.TK_SOLVER_THRESHOLD else None
