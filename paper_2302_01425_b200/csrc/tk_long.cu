@@ -287,6 +287,24 @@ __global__ void __launch_bounds__(TPB) long_prefix_kernel(const Problem P, LongW
   const RowSetup S = row_setup(M, skeys, n, k);
   if (!S.has_block) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  {
+    // A tile with no rank inside the window has nothing to sum: all of it capped (its last key at or
+    // above the window), or all of it below (its first key at or below the window).  The search only
+    // reads prefix sums at ranks wl..wh; of a skipped tile that can only be its first rank (= wh).
+    const int first = tile * TILE, last = min(first + TILE, n) - 1;
+    const float d_first = radix_key_to_float(skeys[first]) - S.piv;
+    const float d_last = radix_key_to_float(skeys[last]) - S.piv;
+    if (d_last >= S.W_hi || !(d_first > S.W_lo)) {
+      if (threadIdx.x == 0) {
+        const long long base0 = row * (long long)n;
+        ws.pin1[base0 + first] = 0.0f;
+        if (M.q4) { ws.pin2[base0 + first] = 0.0f; ws.pin3[base0 + first] = 0.0f; }
+        double* ts = ws.tsum + row * 3ll * tiles;
+        ts[tile] = 0.0; ts[tiles + tile] = 0.0; ts[2 * tiles + tile] = 0.0;
+      }
+      return;
+    }
+  }
   const int start = tile * TILE + threadIdx.x * IPT;     // blocked: 16 consecutive ranks per thread
   float e1[IPT], e2[IPT], e3[IPT];
   float s1 = 0.f, s2 = 0.f, s3 = 0.f;
