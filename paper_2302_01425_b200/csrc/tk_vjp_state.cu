@@ -79,9 +79,12 @@ __device__ __forceinline__ float finish(const Problem& P, const Math& M, const R
 
 // G lanes of a warp per row (G = 1..32, power of two), 32/G rows per warp.  Every lane keeps its
 // CH float4 chunks of theta and g in registers, so the row is read from memory once (n <= 4 G CH).
-template <int G, int CH>
+// GEN: q is neither 2 nor 4 (rho' through powf); a template flag so that the usual kernels carry no
+// trace of that branch.
+template <int G, int CH, bool GEN>
 __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
-  const Math M = make_math(P);
+  Math M = make_math(P);
+  M.gen = GEN;
   const int lane = threadIdx.x & 31;
   const int lig = lane % G;
   const long long row = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + lane / G;
@@ -178,9 +181,11 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
 }
 
 // one thread block per row
+template <bool GEN>
 __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
   __shared__ double red[2][8];
-  const Math M = make_math(P);
+  Math M = make_math(P);
+  M.gen = GEN;
   const int t = threadIdx.x, T = blockDim.x, lane = t & 31, warp = t >> 5;
   const long long row = blockIdx.x;
   const int n = P.n;
@@ -229,7 +234,7 @@ __global__ void __launch_bounds__(256) tk_vjp_state_cta(const Problem P) {
 // (no atomics, so results do not depend on scheduling) and finishes its own tile.
 __global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, double2* partial, int tiles) {
   __shared__ double red[2][8];
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const long long row = blockIdx.y;
   const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
   const RowCtx c = load_ctx(P, M, row);
@@ -256,7 +261,7 @@ __global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, doub
 
 __global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const double2* partial, int tiles) {
   __shared__ double red[2][8];
-  const Math M = make_math(P);
+  const Math M = make_math_q24(P);
   const long long row = blockIdx.y;
   const int tile = blockIdx.x, t = threadIdx.x, n = P.n;
   const RowCtx c = load_ctx(P, M, row);
@@ -294,11 +299,12 @@ cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t 
 }
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
+  const bool gen = P.qm1 > 0.0f;
   if (P.n <= 512) {
     // lanes per row: two float4 per lane (one for n <= 4), four for 256 < n <= 512
     if (P.n > 256) {
       const unsigned blocks = (unsigned)((P.rows + 7) / 8);
-      tk_vjp_state_group<32, 4><<<blocks, 256, 0, stream>>>(P);
+      (gen ? tk_vjp_state_group<32, 4, true> : tk_vjp_state_group<32, 4, false>)<<<blocks, 256, 0, stream>>>(P);
       return cudaGetLastError();
     }
     int G = 1;
@@ -307,17 +313,17 @@ cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
     const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
     switch (G) {
       case 1:
-        if (P.n <= 4) tk_vjp_state_group<1, 1><<<blocks, 256, 0, stream>>>(P);
-        else tk_vjp_state_group<1, 2><<<blocks, 256, 0, stream>>>(P);
+        if (P.n <= 4) (gen ? tk_vjp_state_group<1, 1, true> : tk_vjp_state_group<1, 1, false>)<<<blocks, 256, 0, stream>>>(P);
+        else (gen ? tk_vjp_state_group<1, 2, true> : tk_vjp_state_group<1, 2, false>)<<<blocks, 256, 0, stream>>>(P);
         break;
-      case 2: tk_vjp_state_group<2, 2><<<blocks, 256, 0, stream>>>(P); break;
-      case 4: tk_vjp_state_group<4, 2><<<blocks, 256, 0, stream>>>(P); break;
-      case 8: tk_vjp_state_group<8, 2><<<blocks, 256, 0, stream>>>(P); break;
-      case 16: tk_vjp_state_group<16, 2><<<blocks, 256, 0, stream>>>(P); break;
-      default: tk_vjp_state_group<32, 2><<<blocks, 256, 0, stream>>>(P); break;
+      case 2: (gen ? tk_vjp_state_group<2, 2, true> : tk_vjp_state_group<2, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
+      case 4: (gen ? tk_vjp_state_group<4, 2, true> : tk_vjp_state_group<4, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
+      case 8: (gen ? tk_vjp_state_group<8, 2, true> : tk_vjp_state_group<8, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
+      case 16: (gen ? tk_vjp_state_group<16, 2, true> : tk_vjp_state_group<16, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
+      default: (gen ? tk_vjp_state_group<32, 2, true> : tk_vjp_state_group<32, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
     }
   } else {
-    tk_vjp_state_cta<<<(unsigned)P.rows, 256, 0, stream>>>(P);
+    (gen ? tk_vjp_state_cta<true> : tk_vjp_state_cta<false>)<<<(unsigned)P.rows, 256, 0, stream>>>(P);
   }
   return cudaGetLastError();
 }
