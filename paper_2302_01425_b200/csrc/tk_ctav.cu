@@ -452,21 +452,24 @@ cudaError_t launch_ctav(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;
   P.N = cta_padded_length(P.n);
   if (P.N < 512) P.N = 512;
-  const int E = P.N > 16384 ? 32 : 16;      // one warp sorts 32 E keys; T = N / E threads
+  // one warp sorts 32 E keys; T = N / E threads.  32 keys per thread (forward pass only) from 16384
+  // elements: 512 threads per row there, and the only way to hold 32768
+  const int E = (P.N > 16384 || (P.N >= 2048 && P.what == W_FWD)) ? 32 : 16;
   if (E == 32 && P.what != W_FWD) return cudaErrorInvalidValue;
   const int T = P.N / E;
   const size_t smem = (size_t)(((P.N + (P.N >> PAD_SHIFT)) + 2) & ~1) * 4 + (size_t)3 * (T + 1) * 8 + 40 * 8 + 40 * 4 + 64;
   void (*kern)(const Problem) = nullptr;
   int slot;
-  if (E == 32) { kern = tk_ctav_kernel<32, 1024>; slot = 0; }
+  if (E == 32 && T <= 512) { kern = tk_ctav_kernel<32, 512>; slot = 3; }
+  else if (E == 32) { kern = tk_ctav_kernel<32, 1024>; slot = 0; }
   else if (T > 512) { kern = tk_ctav_kernel<16, 1024>; slot = 2; }
   else { kern = tk_ctav_kernel<16, 512>; slot = 1; }
-  static bool configured[3][64] = {};
+  static bool configured[4][64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
-    const int max_n = slot == 0 ? 32768 : 16384;
+    const int max_n = (slot == 0) ? 32768 : 16384;
     const int max_smem = (max_n + (max_n >> PAD_SHIFT) + 2) * 4 + 3 * 1025 * 8 + 40 * 8 + 40 * 4 + 64;
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (err != cudaSuccess) return err;
