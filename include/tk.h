@@ -124,6 +124,15 @@ tk_status tk_vjp(const float *theta, const float *grad_out, int64_t rows, int64_
                  double p, double lambda, int mode, float *grad_theta, const tk_opts *opts,
                  tk_stream stream);
 
+/* Jacobian-vector product (the Jacobian of Prop. 7 chained through y = grad R*(x - u),
+ * applied to a tangent instead of a cotangent): out_tangent[r, :] = J(theta[r, :]) tangent[r, :].
+ * All device, [rows*n] fp32.  opts->state_out must hold the row state a forward call saved
+ * (TK_ERR_UNSUPPORTED without it); rows of more than 32768 elements also need opts->workspace.
+ * For TK_MASK and TK_TOPKMAG the Jacobian is symmetric and the result equals tk_vjp's.        */
+tk_status tk_jvp(const float *theta, const float *tangent, int64_t rows, int64_t n, int64_t k,
+                 double p, double lambda, int mode, float *out_tangent, const tk_opts *opts,
+                 tk_stream stream);
+
 /* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
  * perm_out[i] = index of the i-th largest key (theta, or |theta| for
  * TK_TOPKMAG), equal keys in ascending index, -0 == +0.  sorted_out (may be

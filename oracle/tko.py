@@ -135,6 +135,23 @@ def vjp(theta, gout, k: int, p: float, lam: float, mode: int = MASK, flags: int 
     return grad
 
 
+def jvp(theta, tangent, k: int, p: float, lam: float, mode: int = MASK) -> np.ndarray:
+    """J(theta) tangent per row, assembled from the Jacobian's rows: row i of J is vjp(e_i)
+    (Prop. 7 gives the Jacobian; nothing is transposed by hand).  n calls of vjp: small cases."""
+    x = _f32(theta)
+    v = np.asarray(tangent, np.float64)
+    if v.shape != x.shape:
+        raise ValueError("tangent shape differs from theta")
+    rows, n = x.shape
+    out = np.empty((rows, n), np.float64)
+    e = np.zeros((rows, n), np.float32)
+    for i in range(n):
+        e[:, i] = 1.0
+        out[:, i] = np.sum(vjp(x, e, k, p, lam, mode) * v, axis=1)
+        e[:, i] = 0.0
+    return out
+
+
 def dykstra(theta, k: int, p: float, lam: float, mode: int = MASK, sweeps: int = 100,
             flags: int = 0, return_v: bool = False):
     x = _f32(theta)

@@ -24,7 +24,7 @@ TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
 ROWSTATE_BYTES = 16
 
 EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
-           "tk_argsort", "tk_fwd_noalloc")
+           "tk_jvp", "tk_argsort", "tk_fwd_noalloc")
 TK_NOALLOC_MAX_ELEMENTS = 1 << 18
 
 
@@ -72,6 +72,8 @@ def load() -> ctypes.CDLL:
     lib.tk_fwd_ex.argtypes = [vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_vjp.restype = ci
     lib.tk_vjp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_jvp.restype = ci
+    lib.tk_jvp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_argsort.restype = ci
     lib.tk_argsort.argtypes = [vp, i64, i64, ci, vp, vp, ctypes.POINTER(TkOpts), vp]
     _lib = lib
@@ -154,6 +156,16 @@ def tk_vjp(theta, grad_out, rows, n, k, p, lam, mode, grad_theta, *, state=None,
                        ctypes.byref(o), _stream())
     if rc != TK_OK:
         raise TkError(rc, "tk_vjp")
+
+
+def tk_jvp(theta, tangent, rows, n, k, p, lam, mode, out_tangent, *, state, workspace=None,
+           status_out=None) -> None:
+    o = _opts(state=state, workspace=workspace, status_out=status_out)
+    rc = load().tk_jvp(_dev(theta, torch.float32, "theta"), _dev(tangent, torch.float32, "tangent"),
+                       rows, n, k, p, lam, mode, _dev(out_tangent, torch.float32, "out_tangent"),
+                       ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_jvp")
 
 
 def tk_argsort(theta, rows, n, mode, perm_out, sorted_out=None, *, workspace=None,

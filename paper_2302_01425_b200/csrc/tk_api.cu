@@ -216,6 +216,37 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 
+tk_status tk_jvp(const float* theta, const float* tangent, int64_t rows, int64_t n, int64_t k,
+                 double p, double lambda, int mode, float* out_tangent, const tk_opts* opts,
+                 tk_stream stream) {
+  int q4 = 0;
+  double qm1 = 0.0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4, &qm1);
+  if (s != TK_OK) return s;
+  if (rows == 0) return TK_OK;
+  if (tangent == nullptr || out_tangent == nullptr) return TK_ERR_INVALID_ARG;
+  if (!(opts && opts->state_out)) return TK_ERR_UNSUPPORTED;       // from the forward pass's row state only
+  tk::Problem P;
+  fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
+  P.gout = tangent;
+  P.out = out_tangent;
+  P.what = tk::W_VJP;
+  P.jvp = 1;
+  P.state_in = opts->state_out;
+  P.status = opts->status_out;
+  P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(tangent) && aligned16(out_tangent);
+  cudaError_t e;
+  if (n <= tk::kMaxKeyOnlyN) {
+    e = tk::launch_vjp_state(P, (cudaStream_t)stream);
+  } else {
+    s = check_workspace(opts, rows, n);
+    if (s != TK_OK) return s;
+    e = tk::launch_vjp_state_long(P, tk::long_workspace_partials(opts->workspace, rows, (int)n),
+                                  (cudaStream_t)stream);
+  }
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
 tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int32_t* perm_out,
                      float* sorted_out, const tk_opts* opts, tk_stream stream) {
   if (rows < 0 || n < 1 || mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;

@@ -37,6 +37,7 @@ struct Problem {
   int vec4;                 // rows may be accessed as float4
   float lam, inv_lam, lam3; // lambda, 1/lambda, lambda^3
   int sweeps;               // Dykstra path
+  int jvp;                  // tk_vjp_state kernels: the tangent goes through J instead of the cotangent through J^T
 };
 
 // ---------------------------------------------------------------- keys

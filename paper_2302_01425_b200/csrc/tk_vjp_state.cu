@@ -13,6 +13,10 @@ namespace tk {
 
 namespace {
 
+// JVP (P.jvp): J is symmetric for the mask and the magnitude modes (in sorted coordinates it is
+// diag(rho') - rho' rho'^T / D, and signs enter as S J S), so the same code serves.  For topk,
+// y = theta o mask(theta): the VJP is g o mask + J_mask^T (theta o g), the JVP is v o mask +
+// theta o (J_mask v): the weight theta moves from inside the block mean to outside it.
 struct RowCtx {
   float pivot, offset, wid;
   bool has_block;
@@ -53,7 +57,7 @@ __device__ __forceinline__ void accumulate_f64(const Problem& P, const Math& M, 
   float key = sort_key(x, M.mag);
   if (classify(c, key, tt) == 1) {
     double dr = (double)M.drho(tt);
-    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? x : 1.0f);
+    float chi = M.mag ? (signbit(x) ? -1.0f : 1.0f) : ((P.mode == TK_TOPK && !P.jvp) ? x : 1.0f);
     D += dr;
     A += dr * ((double)chi * (double)g);
   }
@@ -65,9 +69,10 @@ __device__ __forceinline__ float finish(const Problem& P, const Math& M, const R
   float key = sort_key(x, M.mag);
   int cls = classify(c, key, tt);
   float sgn = (M.mag && signbit(x)) ? -1.0f : 1.0f;
-  float chi = M.mag ? sgn : (P.mode == TK_TOPK ? x : 1.0f);
+  const bool jt = P.mode == TK_TOPK && P.jvp;
+  float chi = M.mag ? sgn : ((P.mode == TK_TOPK && !jt) ? x : 1.0f);
   float o = 0.0f;
-  if (cls == 1) o = M.drho(tt) * (fmaf(chi, g, -ratio) - delta);
+  if (cls == 1) o = (jt ? x : 1.0f) * M.drho(tt) * (fmaf(chi, g, -ratio) - delta);
   else if (cls == 2 && M.mag) o = chi * g * M.top_slope(key);
   o *= sgn;
   if (P.mode == TK_TOPK) {
@@ -119,8 +124,9 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
   // One classification per element: w = sign * rho' on the pooled block (else 0) and the part of
   // the result that does not depend on the block mean; then
   //   o = w ((chi g - r0) - delta) + fixed,   r0 = fl(A / D),   delta = (sum w' (chi g - r0) - m r0) / D.
+  const bool jt = P.mode == TK_TOPK && P.jvp;          // topk JVP: theta multiplies outside the block mean
   auto chi_of = [&](float xv) -> float {
-    return M.mag ? (signbit(xv) ? -1.0f : 1.0f) : (P.mode == TK_TOPK ? xv : 1.0f);
+    return M.mag ? (signbit(xv) ? -1.0f : 1.0f) : ((P.mode == TK_TOPK && !jt) ? xv : 1.0f);
   };
   float w[CH][4], fixed[CH][4];
   float A = 0.f, D = 0.f;
@@ -169,7 +175,7 @@ __global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
     float o[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      o[j] = fmaf(w[ch][j], fmaf(chi_of(x[ch][j]), g[ch][j], -ratio) - delta, fixed[ch][j]);
+      o[j] = fmaf(w[ch][j] * (jt ? x[ch][j] : 1.0f), fmaf(chi_of(x[ch][j]), g[ch][j], -ratio) - delta, fixed[ch][j]);
     }
     if (P.vec4) {
       if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o[0], o[1], o[2], o[3]);

@@ -403,3 +403,41 @@ def test_general_p_limits():
         with pytest.raises(tk.TkError) as e:
             tk.tk_fwd(th, 4, 64, 2, p_bad, 1.0, tk.TK_MASK, out)
         assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_jvp_matches_oracle_and_is_the_adjoint_of_the_vjp(mode, p):
+    from oracle import tko
+    from parity import rel_err, TOL
+    # element by element against the oracle's Jacobian on small rows
+    for n, k, lam, rows, seed in [(8, 3, 0.7, 40, 601), (33, 7, 0.3, 12, 602), (100, 10, 2.0, 6, 603),
+                                  (300, 40, 1.0, 3, 604), (1500, 150, 1.0, 1, 605)]:
+        x = rows_of(n, rows, seed)
+        v = wl.cotangent_like(x, seed)
+        th, vt = torch.from_numpy(x).cuda(), torch.from_numpy(v).cuda()
+        out, st, jv = torch.empty_like(th), tk.new_state(rows), torch.empty_like(th)
+        tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, state_out=st)
+        tk.tk_jvp(th, vt, rows, n, k, p, lam, mode, jv, state=st)
+        torch.cuda.synchronize()
+        ref = tko.jvp(x, v, k, p, lam, mode)
+        assert float(rel_err(jv.cpu().numpy(), ref).max()) <= 5 * TOL, (n, k, lam)   # n-term sums of 1e-5 entries
+    # <g, J v> = <J^T g, v> at a size the oracle's n^2 assembly cannot reach
+    rows, n, k, lam = 4096, 400, 28, 1.0
+    x = rows_of(n, rows, 610)
+    th = torch.from_numpy(x).cuda()
+    g = torch.from_numpy(wl.cotangent_like(x, 611)).cuda()
+    v = torch.from_numpy(wl.cotangent_like(x, 612)).cuda()
+    out, st = torch.empty_like(th), tk.new_state(rows)
+    jv, jtg = torch.empty_like(th), torch.empty_like(th)
+    tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, state_out=st)
+    tk.tk_jvp(th, v, rows, n, k, p, lam, mode, jv, state=st)
+    tk.tk_vjp(th, g, rows, n, k, p, lam, mode, jtg, state=st)
+    torch.cuda.synchronize()
+    lhs = (g.double() * jv.double()).sum(dim=1)
+    rhs = (jtg.double() * v.double()).sum(dim=1)
+    scale = (g.double().abs() * jv.double().abs()).sum(dim=1) + 1.0
+    assert float(((lhs - rhs).abs() / scale).max()) <= 1e-5
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_jvp(th, v, rows, n, k, p, lam, mode, jv, state=None)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED

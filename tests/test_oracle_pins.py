@@ -527,6 +527,32 @@ def test_vjp_matches_finite_differences(p, mode):
     assert checked >= 4
 
 
+@pytest.mark.parametrize("mode", [tko.MASK, tko.TOPK, tko.TOPKMAG])
+def test_jvp_is_the_finite_difference_jacobian_applied_to_the_tangent(mode):
+    """p = 2: the operator is piecewise linear, central differences are exact away from kinks."""
+    rng = np.random.default_rng(43)
+    checked = 0
+    for trial in range(10):
+        n, k, lam = 8, 3, 0.7
+        x = rng.standard_normal(n).astype(np.float32)
+        _, d0 = tko.fwd(x, k, 2.0, lam, mode, details=True)
+        stable = True
+        for j in range(n):
+            for sgn in (-1, 1):
+                xx = x.copy(); xx[j] = np.float32(xx[j] + sgn * 2e-3)
+                _, d1 = tko.fwd(xx, k, 2.0, lam, mode, details=True)
+                stable &= (np.array_equal(d0["perm"], d1["perm"]) and np.array_equal(d0["block_lo"], d1["block_lo"])
+                           and np.array_equal(d0["block_hi"], d1["block_hi"]))
+        if not stable:
+            continue
+        v = rng.standard_normal(n)
+        Jfd = jacobian_fd(x, k, 2.0, lam, mode)
+        got = tko.jvp(x[None, :], v[None, :], k, 2.0, lam, mode)[0]
+        assert np.max(np.abs(got - Jfd @ v)) < 1e-7 * max(1.0, np.max(np.abs(Jfd)))
+        checked += 1
+    assert checked >= 3
+
+
 @pytest.mark.parametrize("p", [2.0, P43])
 def test_mask_jacobian_is_symmetric_with_zero_row_sums(p):
     x = random_rows(1, 14, 51)[0]
