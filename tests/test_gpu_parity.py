@@ -441,3 +441,33 @@ def test_jvp_matches_oracle_and_is_the_adjoint_of_the_vjp(mode, p):
     with pytest.raises(tk.TkError) as e:
         tk.tk_jvp(th, v, rows, n, k, p, lam, mode, jv, state=None)
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
+def test_randomised_shapes_modes_and_lambdas():
+    """A seeded sweep over row lengths around every kernel boundary, k anywhere in 1..n, lambda from
+    0.05 to 100, all modes, exact ties and exact zeros: every case through the full parity harness."""
+    from parity import run_case
+    rng = np.random.Generator(np.random.PCG64(2024))
+    lengths = [1, 2, 3, 5, 8, 9, 13, 16, 17, 31, 32, 33, 64, 65, 100, 128, 129, 200, 256, 257, 300, 400, 512,
+               513, 700, 1000, 1024, 1025, 1500, 2048, 2049, 3000, 4096, 5000, 8192, 10000, 16384, 16385,
+               20000, 32768]
+    for it in range(160):
+        n = int(rng.choice(lengths))
+        k = int(rng.integers(1, n + 1))
+        if rng.random() < 0.5:
+            k = max(1, min(n, int(n * rng.choice([0.01, 0.1, 0.25, 0.5, 0.9]))))
+        lam = float(rng.choice([0.05, 0.1, 0.3, 1.0, 3.0, 10.0, 100.0]))
+        p = float(rng.choice([2.0, P43]))
+        mode = int(rng.integers(0, 3))
+        rows = int(rng.choice([1, 3, 7, 37])) if n > 2048 else int(rng.choice([1, 5, 37, 130, 1000]))
+        scale = float(rng.choice([0.5, 1.0, 1.0, 2.0]))
+        x = wl.normal_rows(rows, n, 9000 + it, scale)
+        ties = rng.random() < 0.2 and n >= 8
+        zeros = rng.random() < 0.1
+        if ties:
+            x[:, : n // 4] = x[:, n // 2: n // 2 + n // 4]
+        if zeros:
+            x[:, ::3] = 0.0
+        g = wl.cotangent_like(x, 9000 + it)
+        run_case(x, k, p, lam, mode, g,
+                 label=f"it={it} n={n} k={k} lam={lam} p={p:.3f} mode={mode} rows={rows} ties={ties} zeros={zeros}")
