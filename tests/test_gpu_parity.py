@@ -471,3 +471,32 @@ def test_randomised_shapes_modes_and_lambdas():
         g = wl.cotangent_like(x, 9000 + it)
         run_case(x, k, p, lam, mode, g,
                  label=f"it={it} n={n} k={k} lam={lam} p={p:.3f} mode={mode} rows={rows} ties={ties} zeros={zeros}")
+
+
+def test_unaligned_base_pointers_take_the_scalar_path_and_agree():
+    """theta / cotangent / outputs that start 4 or 12 bytes off a 16-byte boundary cannot use 128-bit
+    accesses; the scalar path must give the same results (the summation order of the VJP's block
+    sums may differ: one ulp)."""
+    for n, k in [(8, 2), (64, 5), (300, 30), (512, 64), (1024, 100), (4096, 512), (16384, 999), (32768, 100)]:
+        rows = 33 if n <= 1024 else 3
+        for mode, p in [(tk.TK_MASK, 2.0), (tk.TK_TOPK, P43), (tk.TK_TOPKMAG, 2.0)]:
+            base = torch.randn(rows * n, device="cuda")
+            gbase = torch.randn(rows * n, device="cuda")
+            got = []
+            for off in (0, 1, 3):
+                bufs = [torch.empty(rows * n + 4, device="cuda") for _ in range(5)]
+                x, g, o, d, d2 = [b[off:off + rows * n] for b in bufs]
+                x.copy_(base); g.copy_(gbase)
+                st = tk.new_state(rows)
+                tk.tk_fwd_ex(x, rows, n, k, p, 0.7, mode, o, state_out=st)
+                tk.tk_vjp(x, g, rows, n, k, p, 0.7, mode, d, state=st)
+                if n <= 16384:
+                    tk.tk_vjp(x, g, rows, n, k, p, 0.7, mode, d2)
+                else:
+                    d2.zero_()
+                torch.cuda.synchronize()
+                got.append((o.clone(), d.clone(), d2.clone()))
+            for o, d, d2 in got[1:]:
+                assert torch.equal(o, got[0][0]), (n, mode)
+                for a, b in ((d, got[0][1]), (d2, got[0][2])):
+                    assert float(((a - b).abs() / b.abs().clamp(min=1.0)).max()) <= 1e-6, (n, mode)
