@@ -333,9 +333,10 @@ def main():
                             entry["dykstra_forward_10_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
                         if name in ("sweep_n64", "sweep_n4096"):
-                            # p = 1.5 (q = 3): no closed-form block solve, sort-free solver with Newton steps
+                            # p = 1.5 (q = 3): no closed-form block solve; the library picks the path
+                            # (n = 64: sorting kernel + per-row Newton; n = 4096: sort-free solver)
                             entry["general_p_1.5_forward"] = time_solver_forward(
-                                name, dev, tk, torch, tk.TK_SOLVER_THRESHOLD, p_override=1.5)
+                                name, dev, tk, torch, tk.TK_SOLVER_AUTO, p_override=1.5)
                         ncase = workload_cases(name)[0].n
                         if 512 <= ncase <= 16384:
                             # the same exact result without the sort (solver = TK_SOLVER_THRESHOLD),

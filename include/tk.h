@@ -22,9 +22,11 @@
  *  - 1 <= k <= n, lambda > 0, p > 1.  q = p/(p-1) within 1e-6 of 2 or 4 (p = 2,
  *    p = 4/3: closed-form block solves, App. A.6) runs on every path.  Any other
  *    1 < p <= 1.5 (3 <= q <= 64; Sec. 7, "sensitivity to the choice of p") runs
- *    for TK_MASK and TK_TOPK on rows of up to 16384 elements: the forward pass
- *    through the sort-free solver whatever tk_opts.solver says (no permutation
- *    output), tk_vjp from saved row state only.  Everything else:
+ *    for TK_MASK and TK_TOPK on rows of up to 16384 elements, without a
+ *    permutation output: rows of up to 128 elements are sorted and solved by a
+ *    Newton iteration per row (forward pass and tk_vjp with or without saved
+ *    state); longer rows go through the sort-free solver whatever
+ *    tk_opts.solver says, and tk_vjp needs the saved row state.  Everything else:
  *    TK_ERR_UNSUPPORTED (p > 2 makes rho' unbounded at 0; for 1.5 < p < 2 rho''
  *    is, and fp32 keys cannot carry the VJP to 1e-5).  Outputs must not alias
  *    inputs.

@@ -30,6 +30,7 @@ void* long_workspace_partials(void* workspace, long long rows, int n);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
 constexpr int kMaxKeyOnlyN = 32768;  // longest row the key-only forward pass holds on chip (no workspace)
+constexpr int kMaxGeneralSortedN = 128;   // general p: longest row solved by one lane's Newton iteration (tk_rows.cu)
 constexpr int kMaxGroupN = 512;      // longest row a single warp holds in registers as (key, index) words
 constexpr int kMaxWalkN = 1024;      // longest row of the warp-autonomous kernel (tk_rows.cu)
 
@@ -129,9 +130,13 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
   if (out == nullptr) return TK_ERR_INVALID_ARG;
   int solver = opts ? opts->solver : TK_SOLVER_AUTO;
   if (solver < TK_SOLVER_AUTO || solver > TK_SOLVER_THRESHOLD) return TK_ERR_INVALID_ARG;
-  if (qm1 > 0.0) {                 // general p: only the sort-free solver has no closed form to rely on
+  if (qm1 > 0.0) {
+    // general p: no closed-form block solve.  Rows of up to 128 elements: the sorting kernel with a
+    // per-row Newton iteration on the threshold function; longer rows (and every explicit request
+    // for it): the sort-free solver.  No permutation output either way.
     if (solver == TK_SOLVER_PAV || solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
-    solver = TK_SOLVER_THRESHOLD;
+    if (opts && opts->perm_out) return TK_ERR_UNSUPPORTED;
+    if (n > tk::kMaxGeneralSortedN) solver = TK_SOLVER_THRESHOLD;
   }
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
@@ -181,7 +186,8 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
   if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
-  if (qm1 > 0.0 && !(opts && opts->state_out)) return TK_ERR_UNSUPPORTED;   // general p: from saved state only
+  // general p: from saved state, or recomputed by the sorting kernel for rows of up to 128 elements
+  if (qm1 > 0.0 && !(opts && opts->state_out) && n > tk::kMaxGeneralSortedN) return TK_ERR_UNSUPPORTED;
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.gout = grad_out;

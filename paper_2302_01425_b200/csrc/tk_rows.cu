@@ -135,6 +135,72 @@ __device__ __forceinline__ void solve_row_walk(const float* sk, int n, int k, co
   R.piv = piv; R.u = u; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = has_block ? 1 : 0;
 }
 
+// Any other q (rho(t) = (t/lambda)^(q-1) through powf; mask and top-k modes): H is no polynomial, so
+// the block is not grown but gamma is found as the root of the threshold function
+//   F(tau) = #{s_i >= tau + lambda} - k + sum_{tau < s_i < tau + lambda} rho(s_i - tau)
+// by one thread on its sorted row: safeguarded Newton inside the bracket (s_{k-1} - lambda, s_k),
+// every pass over the window ranks only (those between the bracket's ends and a cap above), one
+// Newton step on the current set's equation sum rho = m per pass, bisection when the step leaves
+// the bracket.  The pass that sees the set it was computed from and has a rounding-sized step left
+// is at the root; the block is that set.  Cost: (passes) x (window) powf pairs per row, so this
+// serves short rows; longer ones go to the block-per-row solver of tk_thr.cu.
+__device__ __forceinline__ void solve_row_newton(const float* sk, int n, int k, const Math& M, const Problem& P,
+                                                 RowSol& R, int& flags) {
+  auto key = [&](int i) -> float { return sk[i]; };
+  const float c = key(k - 1);
+  const float lam = P.lam;
+  const bool has_block = (k < n) && (c - lam < key(k));
+  const float piv = c;
+  int a0 = k, b0 = k;
+  float u = 0.0f;
+  if (has_block) {
+    // window ranks [wl, wh): keys strictly between c - lambda and c + lambda
+    int wl = k - 1, wh = k + 1;
+    while (wl > 0 && key(wl - 1) - piv < lam) --wl;
+    while (wh < n && key(wh) - piv > -lam) ++wh;
+    float lo = -lam, hi = key(k) - piv;            // offsets with F >= 0 at lo, F <= 0 at hi
+    float off = 0.5f * (lo + hi);
+    int prev_ct = -1, prev_cm = -1;
+    bool done = false;
+#pragma unroll 1
+    for (int it = 0; it < 64 && !done; ++it) {
+      int ct = wl, cm = 0;                          // ranks above the window are capped whatever gamma is
+      float s1 = 0.f, s2 = 0.f;
+      for (int i = wl; i < wh; ++i) {
+        const float tt = (key(i) - piv) - off;
+        const bool top = tt >= lam;
+        const bool mid = tt > 0.0f && !top;
+        ct += top; cm += mid;
+        if (mid) { s1 += M.rho(tt); s2 += M.drho(tt); }
+      }
+      const int m = k - ct;
+      const float Fv = (float)(ct - k) + s1;
+      float du = 0.0f;
+      bool have = false;
+      if (cm > 0 && m >= 1 && s2 > 0.0f) {
+        du = (s1 - (float)m) / s2;
+        have = true;
+        if (ct == prev_ct && cm == prev_cm && fabsf(du) <= 1e-6f * lam) { a0 = ct; b0 = ct + cm; off += du; done = true; }
+      }
+      if (!done) {
+        if (Fv > 0.0f) lo = fmaxf(lo, off); else hi = fminf(hi, off);
+        const float cand = off + du;
+        const bool inside = have && cand > lo && cand < hi && (it & 7) != 7;
+        prev_ct = inside ? ct : -1; prev_cm = inside ? cm : -1;
+        const float next = inside ? cand : 0.5f * (lo + hi);
+        if (next == off || !(hi > lo)) { a0 = ct; b0 = ct + cm; if (have) off += du; done = true; }
+        else off = next;
+      }
+    }
+    if (!done) flags |= TK_FLAG_NOT_CONVERGED;
+    u = off;
+    if (b0 > a0) u = settle_offset(M, piv, u, a0, b0, n, key);
+    else { a0 = k; b0 = k; }
+  }
+  const bool block = b0 > a0;
+  R.piv = piv; R.u = block ? u : 0.0f; R.c = c; R.a0 = a0; R.b0 = b0; R.has_block = block ? 1 : 0;
+}
+
 // The same growth by a whole warp for one row (rows of more than 128 elements have a warp to
 // themselves): 32 candidates per step.  Lane i tests rank b + i (or a - 1 - i) against the block
 // with the i candidates before it already pooled -- its power sums are the block's plus an
@@ -247,8 +313,10 @@ struct RowsGeom {
   static constexpr int STRIDE = N | 1;                     // odd: lane r walking row r meets no bank conflict
 };
 
-template <int G, int E, int B, bool Q4, bool MAG>
+// QM: 0 for q = 2, 1 for q = 4, 2 for any other q (short rows, mask and top-k modes)
+template <int G, int E, int B, int QM, bool MAG>
 __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) tk_rows_kernel(const Problem P) {
+  constexpr bool Q4 = QM == 1, GEN = QM == 2;
   constexpr int RPB = RowsGeom<G, E, B>::RPB, R = RowsGeom<G, E, B>::R, BATCHES = B;
   constexpr int STRIDE = RowsGeom<G, E, B>::STRIDE;
   constexpr int WARPS = kRowsThreads / 32;
@@ -260,8 +328,8 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) 
   const unsigned mask = kGroupBits << (gw * G);
   const long long row0 = ((long long)blockIdx.x * WARPS + warp) * R;
   const int n = P.n, k = P.k;
-  Math M = make_math_q24(P);
-  M.q4 = Q4; M.mag = MAG;
+  Math M = make_math(P);
+  M.q4 = Q4; M.mag = MAG; M.gen = GEN;      // compile-time constants from here on
   int flags = 0;
 
   // elements 4 h .. 4 h + 3 of the lane's E consecutive elements of a row (zeros past the row's end)
@@ -312,7 +380,7 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) 
   RowSol mine;
   mine.piv = 0.f; mine.u = 0.f; mine.c = 0.f; mine.a0 = k; mine.b0 = k; mine.has_block = 0;
   bool coop = false;
-  if (G == 32 && E >= 16) {                      // rows of more than 256 elements: blocks can be large
+  if (G == 32 && E >= 16 && !GEN) {              // rows of more than 256 elements: blocks can be large
     int w = 0;
     if (lane < R && row0 + lane < P.rows) w = window_ranks(sm[warp][lane % R], n, k, M);
     coop = __any_sync(0xffffffffu, w > kSerialGrowthMax);
@@ -328,7 +396,8 @@ __global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) 
       }
     }
   } else if (lane < R && row0 + lane < P.rows) {
-    solve_row_walk<Q4, MAG>(sm[warp][lane % R], n, k, M, P, mine);
+    if (GEN) solve_row_newton(sm[warp][lane % R], n, k, M, P, mine, flags);
+    else solve_row_walk<Q4, MAG>(sm[warp][lane % R], n, k, M, P, mine);
   }
   if (lane < R && row0 + lane < P.rows && P.state_out) {
     tk_rowstate st;
@@ -507,12 +576,21 @@ cudaError_t launch_rows_gb(const Problem& P, cudaStream_t stream) {
   const long long per_block = (long long)(kRowsThreads / 32) * RowsGeom<G, E, B>::R;
   const unsigned blocks = (unsigned)((P.rows + per_block - 1) / per_block);
   const bool mag = P.mode == TK_TOPKMAG;
+  if (P.qm1 > 0.0f) {                          // any other q: rows of up to 128 elements, not the magnitude mode
+    if constexpr (G <= 16 && E <= 16) {
+      if (mag) return cudaErrorInvalidValue;
+      tk_rows_kernel<G, E, B, 2, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+      return cudaGetLastError();
+    } else {
+      return cudaErrorInvalidValue;
+    }
+  }
   if (P.q4) {
-    if (mag) tk_rows_kernel<G, E, B, true, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, E, B, true, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, E, B, 1, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, E, B, 1, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   } else {
-    if (mag) tk_rows_kernel<G, E, B, false, true><<<blocks, kRowsThreads, 0, stream>>>(P);
-    else tk_rows_kernel<G, E, B, false, false><<<blocks, kRowsThreads, 0, stream>>>(P);
+    if (mag) tk_rows_kernel<G, E, B, 0, true><<<blocks, kRowsThreads, 0, stream>>>(P);
+    else tk_rows_kernel<G, E, B, 0, false><<<blocks, kRowsThreads, 0, stream>>>(P);
   }
   return cudaGetLastError();
 }

@@ -83,7 +83,9 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     ws_bytes = tk.tk_workspace_bytes(rows, n, k, p, mode)
     ws = torch.empty(max(ws_bytes, 1), dtype=torch.uint8, device=dev) if ws_bytes else None
-    sorts = solver != tk.TK_SOLVER_THRESHOLD          # the sort-free solver has no permutation to give
+    q = p / (p - 1.0)
+    general = min(abs(q - 2.0), abs(q - 4.0)) > 1e-6  # no closed-form block solve: no permutation output either
+    sorts = solver != tk.TK_SOLVER_THRESHOLD and not general   # the sort-free solver has no permutation to give
     tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, perm_out=perm if sorts else None, state_out=state,
                  workspace=ws, status_out=status, solver=solver)
     torch.cuda.synchronize()
@@ -139,12 +141,13 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
             kth = np.sort(np.abs(theta), axis=1)[:, ::-1][:, k - 1]
             free = (theta == 0.0) & (kth == 0.0)[:, None]
         for name, kwargs in (("vjp_state", {"state": state}), ("vjp_recompute", {})):
-            if name == "vjp_recompute" and (ws_bytes or not sorts):
+            recomputes = sorts or (general and solver == tk.TK_SOLVER_AUTO and n <= 128)
+            if name == "vjp_recompute" and (ws_bytes or not recomputes):
                 continue
             # rows left out: near-ties at a block edge in the solve this VJP rests on (the saved
             # state of the first call; its own solve, the one of the second call, when it recomputes)
             keep = np.ones(rows, bool)
-            keep[bad if name == "vjp_state" else bad_noperm] = False
+            keep[bad if (name == "vjp_state" or not sorts) else bad_noperm] = False
             grad = torch.full((rows, n), float("nan"), device=dev)
             tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, workspace=ws, **kwargs)
             torch.cuda.synchronize()

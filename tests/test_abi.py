@@ -74,7 +74,7 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert fwd(4, 8, 2, 1.8, 1.0, 0) == b.TK_ERR_UNSUPPORTED        # 2 < q < 3
     assert fwd(4, 8, 2, 1.5, 1.0, 2) == b.TK_ERR_UNSUPPORTED        # q = 3 with the magnitude mode
     assert fwd(1, 20000, 2, 1.5, 1.0, 0) == b.TK_ERR_UNSUPPORTED    # q = 3 on a row held in global memory
-    assert lib.tk_vjp(fake, fake, 4, 8, 2, 1.5, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED  # no saved state
+    assert lib.tk_vjp(fake, fake, 4, 200, 2, 1.5, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED  # q = 3, n > 128, no saved state
     assert fwd(4, 8, 2, 2.0, 1.0, 0, theta=None) == b.TK_ERR_INVALID_ARG
     assert fwd(4, 8, 2, P43, 1.0, 0, out=None) == b.TK_ERR_INVALID_ARG
     assert fwd(0, 8, 2, 2.0, 1.0, 0) == b.TK_OK                     # rows = 0: nothing to do

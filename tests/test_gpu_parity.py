@@ -384,16 +384,34 @@ def test_general_p_matches_oracle(mode, p):
         res = run_case(x, k, p, lam, mode, g, label=f"p={p} n={n} k={k} lam={lam} mode={mode}",
                        solver=tk.TK_SOLVER_THRESHOLD)
         assert "vjp_state_max_rel" in res
+    # rows of up to 128 elements take the sorting kernel with a per-row Newton iteration (solver AUTO):
+    # forward, VJP from state and recomputing VJP
+    for n, k, lam, rows, seed in [(8, 3, 0.5, 200, 511), (16, 2, 1.0, 130, 512), (64, 2, 0.3, 300, 513),
+                                  (64, 20, 3.0, 64, 514), (100, 10, 1.0, 40, 515), (128, 64, 10.0, 33, 516)]:
+        x = rows_of(n, rows, seed)
+        g = wl.cotangent_like(x, seed)
+        res = run_case(x, k, p, lam, mode, g, label=f"sorted p={p} n={n} k={k} lam={lam} mode={mode}")
+        assert "vjp_state_max_rel" in res and "vjp_recompute_max_rel" in res
 
 
 def test_general_p_limits():
     th = torch.randn((4, 64), device="cuda")
     out = torch.empty_like(th)
-    tk.tk_fwd(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out)                     # solver AUTO: routed to the sort-free solver
+    tk.tk_fwd(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out)                     # solver AUTO, short row: the sorting kernel
     ref = torch.empty_like(th)
     tk.tk_fwd_ex(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, ref, solver=tk.TK_SOLVER_THRESHOLD)
     torch.cuda.synchronize()
-    assert torch.equal(out, ref)
+    assert float((out - ref).abs().max()) <= 1e-6
+    th2 = torch.randn((4, 300), device="cuda")
+    out2, ref2 = torch.empty_like(th2), torch.empty_like(th2)
+    tk.tk_fwd(th2, 4, 300, 9, 1.5, 1.0, tk.TK_MASK, out2)                  # longer row: routed to the sort-free solver
+    tk.tk_fwd_ex(th2, 4, 300, 9, 1.5, 1.0, tk.TK_MASK, ref2, solver=tk.TK_SOLVER_THRESHOLD)
+    torch.cuda.synchronize()
+    assert torch.equal(out2, ref2)
+    g2 = torch.randn_like(th2)
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_vjp(th2, g2, 4, 300, 9, 1.5, 1.0, tk.TK_MASK, out2)          # no saved state on a row of more than 128
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
     for kwargs in ({"solver": tk.TK_SOLVER_PAV}, {"solver": tk.TK_SOLVER_DYKSTRA},
                    {"perm_out": torch.empty((4, 64), dtype=torch.int32, device="cuda")}):
         with pytest.raises(tk.TkError) as e:
