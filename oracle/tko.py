@@ -163,3 +163,26 @@ def dykstra(theta, k: int, p: float, lam: float, mode: int = MASK, sweeps: int =
     if rc:
         raise ValueError("tko_dykstra: invalid argument")
     return (out, v) if return_v else out
+
+
+def topk_loss(theta, target, k: int, p: float, lam: float):
+    """Smooth top-k loss (Sec. 6, "Smooth top-k loss"): per row
+        loss = f(x, 1_k) - <x, t>,   f(x, 1_k) = max_{y in P(1_k)} <y, x> - R(y)
+    (Prop. "Relaxed operator" with phi(x) = x, for which the conjugate of f_phi is the indicator of
+    the permutahedron P(1_k)), t the one-hot vector of target (t = 0 where target is outside
+    [0, n)), R(y) = (lambda/p) sum |y_i|^p.  The maximiser is the relaxed top-k mask y*, so f is
+    evaluated at it; the gradient in x is y* - t (same proposition: grad_1 f = y*).
+    Returns (loss (rows,), grad (rows, n)), float64."""
+    x = _f32(theta)
+    rows, n = x.shape
+    tgt = np.asarray(target, np.int64).reshape(rows)
+    y = fwd(x, k, p, lam, MASK)
+    x64 = x.astype(np.float64)
+    f = np.sum(y * x64, axis=1) - (lam / p) * np.sum(np.abs(y) ** p, axis=1)
+    loss = f.copy()
+    grad = y.copy()
+    for r in range(rows):
+        if 0 <= tgt[r] < n:
+            loss[r] -= x64[r, tgt[r]]
+            grad[r, tgt[r]] -= 1.0
+    return loss, grad

@@ -570,6 +570,88 @@ def test_topkmag_p2_top_singletons_have_slope_one_over_one_plus_lambda():
     assert np.allclose(grad[:2], 1.0 / (1.0 + lam)) and np.all(grad[2:] == 0.0)
 
 
+# ---------------------------------------------------------------- smooth top-k loss
+def sum_of_k_largest(u, k):
+    return np.sort(u)[::-1][:k].sum()
+
+
+def conj_R(t, p, lam):
+    """R*(t) = sum |t_i|^q / (q lambda^(q-1)) for R(y) = (lambda/p) sum |y_i|^p."""
+    q = q_of(p)
+    return np.sum(np.abs(t) ** q) / (q * lam ** (q - 1.0))
+
+
+@pytest.mark.parametrize("p", [2.0, P43, 1.5])
+def test_topk_loss_value_sits_between_primal_and_dual_bounds(p):
+    """f(x, 1_k) = max_{y in P(1_k)} <y,x> - R(y) = min_u R*(x - u) + (sum of the k largest u):
+    every feasible y bounds it from below, every u from above, and the two bounds meet at the
+    oracle's value (checked with y, u that the oracle did not produce)."""
+    rng = np.random.default_rng(5)
+    for n, k, lam in [(6, 2, 1.0), (9, 3, 0.3), (17, 5, 2.0)]:
+        x = random_rows(1, n, 40 + n)[0]
+        x64 = x.astype(np.float64)
+        loss, _ = tko.topk_loss(x, [-1], k, p, lam)
+        f = loss[0]
+        best_lo, best_hi = -np.inf, np.inf
+        ystar = mask_by_threshold(x64, k, p, lam)          # KKT form, shares nothing with sort + PAV
+        q = q_of(p)
+        for trial in range(400):
+            if trial == 0:
+                y = ystar
+            elif trial == 1:
+                y = np.zeros(n); y[np.argsort(-x64)[:k]] = 1.0      # a vertex: the hard mask
+            else:
+                y = np.clip(ystar + rng.normal(size=n) * 10.0 ** rng.integers(-6, 0), 0, 1)
+                y = np.clip(y * (k / y.sum()), 0, 1)
+                if abs(y.sum() - k) > 1e-12:
+                    continue
+            lo = y @ x64 - (lam / p) * np.sum(np.abs(y) ** p)
+            assert lo <= f + 1e-10
+            best_lo = max(best_lo, lo)
+            u = x64 - lam * ystar ** (1.0 / (q - 1.0)) if trial == 0 else x64 * rng.uniform(0, 1) + rng.normal(size=n) * 0.3
+            hi = conj_R(x64 - u, p, lam) + sum_of_k_largest(u, k)
+            assert hi >= f - 1e-10
+            best_hi = min(best_hi, hi)
+        assert abs(best_lo - f) <= 1e-10 and abs(best_hi - f) <= 1e-9
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_topk_loss_gradient_is_the_finite_difference_of_its_value(p):
+    x = random_rows(3, 12, 91)
+    tgt = np.array([0, 7, 11])
+    loss, grad = tko.topk_loss(x, tgt, 4, p, 0.7)
+    h = 1e-3                                            # inputs are float32: a step it represents
+    for r in range(3):
+        for i in range(12):
+            xp, xm = x.copy(), x.copy()
+            xp[r, i] += np.float32(h); xm[r, i] -= np.float32(h)
+            d = float(xp[r, i]) - float(xm[r, i])
+            fd = (tko.topk_loss(xp, tgt, 4, p, 0.7)[0][r] - tko.topk_loss(xm, tgt, 4, p, 0.7)[0][r]) / d
+            assert abs(fd - grad[r, i]) <= 5e-3, (r, i, fd, grad[r, i])
+    assert np.allclose(grad.sum(axis=1), 4 - 1, atol=1e-12)   # <y*, 1> = k, <t, 1> = 1
+
+
+def test_topk_loss_limits_and_two_element_closed_form():
+    x = random_rows(5, 20, 17, scale=3.0)
+    tgt = np.array([3, 3, -1, 20, 0])                      # rows 2 and 3: no target, loss = f
+    lam0 = 1e-6
+    loss, grad = tko.topk_loss(x, tgt, 3, 2.0, lam0)
+    for r in range(5):
+        hard = sum_of_k_largest(x[r].astype(np.float64), 3)
+        t = float(x[r, tgt[r]]) if 0 <= tgt[r] < 20 else 0.0
+        # lambda -> 0: f -> sum of the k largest, from below and by no more than R's largest value on P(1_k)
+        assert hard - t - lam0 * 3 / 2.0 - 1e-8 <= loss[r] <= hard - t + 1e-8
+    # n = 2, k = 1, p = 2: y1 = clip(1/2 + (x1 - x2)/(2 lam), 0, 1), y2 = 1 - y1
+    for x1, x2, lam in [(0.3, 0.1, 1.0), (2.0, -1.0, 0.5), (-0.2, 0.4, 3.0)]:
+        y1 = min(1.0, max(0.0, 0.5 + (np.float32(x1).astype(float) - np.float32(x2).astype(float)) / (2 * lam)))
+        y = np.array([y1, 1 - y1])
+        xv = np.array([np.float32(x1), np.float32(x2)], dtype=np.float64)
+        want = y @ xv - 0.5 * lam * (y ** 2).sum() - xv[1]
+        got, g = tko.topk_loss(np.array([[x1, x2]], np.float32), [1], 1, 2.0, lam)
+        assert abs(got[0] - want) <= 1e-12
+        assert np.allclose(g[0], y - np.array([0.0, 1.0]), atol=1e-12)
+
+
 def test_invalid_arguments_are_rejected():
     x = np.zeros((1, 4), np.float32)
     for k, p, lam in [(0, 2.0, 1.0), (5, 2.0, 1.0), (2, 1.0, 1.0), (2, 2.0, 0.0)]:
