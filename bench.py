@@ -326,7 +326,7 @@ def main():
                                  "ms_per_step": r["ms_total"] / r["steps"],
                                  "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
                                  "kernels": r["kernels"], "config": r["config"]}
-                        if name.startswith("sweep_n") and int(name[7:]) <= 4096:
+                        if name.startswith("sweep_n"):
                             entry["dykstra_forward_100_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
                         if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
@@ -372,8 +372,10 @@ def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, 
         th = torch.from_numpy(c.theta()).to(dev)
         y = torch.empty_like(th)
         st = tk.new_state(c.rows, dev) if solver == tk.TK_SOLVER_THRESHOLD else None
+        wsb = tk.tk_workspace_bytes(c.rows, c.n, c.k, c.p, c.mode, solver) if solver == tk.TK_SOLVER_DYKSTRA else 0
+        ws = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
         run = lambda: tk.tk_fwd_ex(th, c.rows, c.n, c.k, c.p, c.lam, c.mode, y, solver=solver, sweeps=sweeps,
-                                   state_out=st)
+                                   state_out=st, workspace=ws)
         run()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -384,7 +386,7 @@ def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, 
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / launches
         out.append({"p": round(c.p, 6), "avg_us": us, "elements_per_s": c.elements / (us * 1e-6)})
-        del th, y
+        del th, y, ws
     return out
 
 

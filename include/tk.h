@@ -57,7 +57,8 @@ typedef enum {
   TK_SOLVER_AUTO = 0,
   TK_SOLVER_PAV = 1,      /* exact pooling of adjacent violators (Sec. 5, App. B.2)          */
   TK_SOLVER_DYKSTRA = 2,  /* alternating projections on odd/even pairs (Algorithm 1; for
-                             p != 2 the dual block coordinate ascent of App. A.8)            */
+                             p != 2 the dual block coordinate ascent of App. A.8); rows of
+                             up to 131072 elements, those above 16384 with a workspace       */
   TK_SOLVER_THRESHOLD = 3 /* the same exact result as TK_SOLVER_PAV without sorting: root of
                              the capped-simplex threshold function (Sec. 3, P(1_k)); rows of
                              up to 16384 elements; no permutation output                     */
@@ -103,9 +104,9 @@ typedef struct {
 
 /* Scratch bytes tk_fwd_ex / tk_vjp / tk_argsort need for this shape: 0 for rows
  * of up to 16384 elements.  Rows of 16385..32768 elements need it only when a
- * permutation is returned (perm_out, tk_argsort) or tk_vjp has no saved row
- * state; the plain forward pass and the VJP from state run without.  solver as
- * in tk_opts.                                                                  */
+ * permutation is returned (perm_out, tk_argsort), tk_vjp has no saved row
+ * state, or the solver is TK_SOLVER_DYKSTRA; the plain forward pass and the VJP
+ * from state run without.  solver as in tk_opts.                               */
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver);
 
 /* Forward pass (Prop. 2 with Prop. 5 / Prop. 6): out[r, :] = operator(theta[r, :]).
@@ -134,6 +135,22 @@ tk_status tk_vjp(const float *theta, const float *grad_out, int64_t rows, int64_
 tk_status tk_jvp(const float *theta, const float *tangent, int64_t rows, int64_t n, int64_t k,
                  double p, double lambda, int mode, float *out_tangent, const tk_opts *opts,
                  tk_stream stream);
+
+/* Smooth top-k loss (Sec. 6, "Smooth top-k loss"; a Fenchel-Young loss built on Prop. "Relaxed
+ * operator" with phi(x) = x):
+ *   loss[r] = f(theta_r, 1_k) - theta[r, target[r]],
+ *   f(x, 1_k) = max_{y in P(1_k)} <y, x> - R(y) = <y*, x> - (lambda/p) sum_i (y*_i)^p,
+ * y* the relaxed top-k mask of the row, and its gradient in theta (grad_1 f = y*):
+ *   grad[r, :] = y* - onehot(target[r]).
+ * theta: device [rows*n] fp32; target: device [rows] int32 class index, a value outside [0, n)
+ * (or target == NULL) means no target for that row: loss = f, grad = y*; loss: device [rows]
+ * fp32; grad: device [rows*n] fp32 (it also serves as the buffer the mask is computed in).
+ * opts as for tk_fwd_ex (solver, workspace, status word, row state of the mask); every limit of
+ * tk_fwd_ex in TK_MASK mode applies.  Two launches: the forward pass, then one pass over
+ * (theta, y*) that reduces each row and subtracts the target.                                  */
+tk_status tk_topk_loss(const float *theta, const int32_t *target, int64_t rows, int64_t n, int64_t k,
+                       double p, double lambda, float *loss, float *grad, const tk_opts *opts,
+                       tk_stream stream);
 
 /* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
  * perm_out[i] = index of the i-th largest key (theta, or |theta| for

@@ -24,7 +24,7 @@ TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
 ROWSTATE_BYTES = 16
 
 EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
-           "tk_jvp", "tk_argsort", "tk_fwd_noalloc")
+           "tk_jvp", "tk_argsort", "tk_fwd_noalloc", "tk_topk_loss")
 TK_NOALLOC_MAX_ELEMENTS = 1 << 18
 
 
@@ -74,6 +74,8 @@ def load() -> ctypes.CDLL:
     lib.tk_vjp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_jvp.restype = ci
     lib.tk_jvp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_topk_loss.restype = ci
+    lib.tk_topk_loss.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, vp, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_argsort.restype = ci
     lib.tk_argsort.argtypes = [vp, i64, i64, ci, vp, vp, ctypes.POINTER(TkOpts), vp]
     _lib = lib
@@ -166,6 +168,16 @@ def tk_jvp(theta, tangent, rows, n, k, p, lam, mode, out_tangent, *, state, work
                        ctypes.byref(o), _stream())
     if rc != TK_OK:
         raise TkError(rc, "tk_jvp")
+
+
+def tk_topk_loss(theta, target, rows, n, k, p, lam, loss, grad, *, solver=TK_SOLVER_AUTO, sweeps=0,
+                 state_out=None, workspace=None, status_out=None) -> None:
+    o = _opts(solver, sweeps, None, state_out, workspace, status_out)
+    rc = load().tk_topk_loss(_dev(theta, torch.float32, "theta"), _dev(target, torch.int32, "target"),
+                             rows, n, k, p, lam, _dev(loss, torch.float32, "loss"),
+                             _dev(grad, torch.float32, "grad"), ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_topk_loss")
 
 
 def tk_argsort(theta, rows, n, mode, perm_out, sorted_out=None, *, workspace=None,

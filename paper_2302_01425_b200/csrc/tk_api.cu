@@ -18,6 +18,12 @@ cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
 cudaError_t launch_thr(const Problem& P, cudaStream_t stream);
 // alternating-projection solver path (tk_dykstra.cu)
 cudaError_t launch_dykstra(const Problem& P, cudaStream_t stream);
+int dykstra_cluster_max_n();
+cudaError_t launch_dykstra_cluster(const Problem& P, const uint32_t* keys, const int32_t* idx,
+                                   cudaStream_t stream);
+// smooth top-k loss from the relaxed mask (tk_loss.cu)
+cudaError_t launch_loss(const float* theta, const int32_t* target, float* grad, float* loss, long long rows,
+                        int n, double p, double lambda, int q4, double qm1, int vec4, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
 cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream);
@@ -27,6 +33,7 @@ cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_ds
                         cudaStream_t stream);
 tk_rowstate* long_workspace_state(void* workspace, long long rows, int n);
 void* long_workspace_partials(void* workspace, long long rows, int n);
+void long_workspace_sorted(void* workspace, long long rows, int n, const uint32_t** keys, const int32_t** idx);
 
 constexpr int kMaxOnChipN = 16384;   // longest row the block-per-row kernels hold in shared memory
 constexpr int kMaxKeyOnlyN = 32768;  // longest row the key-only forward pass holds on chip (no workspace)
@@ -151,11 +158,24 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
     return et == cudaSuccess ? TK_OK : TK_ERR_CUDA;
   }
   if (solver == TK_SOLVER_DYKSTRA) {
-    // Forward pass only: rows held on chip; no row state (the iterate of a fixed number of
+    // Forward pass only: the iterate stays on chip; no row state (the iterate of a fixed number of
     // sweeps has no exact block structure to save); phi even with p = 4/3 has no closed-form pair step.
-    if (n > tk::kMaxOnChipN || (opts && opts->state_out)) return TK_ERR_UNSUPPORTED;
+    if (n > tk::dykstra_cluster_max_n() || (opts && opts->state_out)) return TK_ERR_UNSUPPORTED;
     if (mode == TK_TOPKMAG && q4) return TK_ERR_UNSUPPORTED;
     P.sweeps = opts ? opts->sweeps : 0;
+    if (n > tk::kMaxOnChipN) {
+      // rows shared by a thread-block cluster: sorted in global memory first (needs the workspace)
+      s = check_workspace(opts, rows, n);
+      if (s != TK_OK) return s;
+      tk::Problem A = P;
+      A.what = tk::W_ARGSORT; A.out = nullptr;
+      cudaError_t ea = tk::launch_long(A, opts->workspace, nullptr, true, (cudaStream_t)stream);
+      if (ea != cudaSuccess) return TK_ERR_CUDA;
+      const uint32_t* keys = nullptr; const int32_t* idx = nullptr;
+      tk::long_workspace_sorted(opts->workspace, rows, (int)n, &keys, &idx);
+      ea = tk::launch_dykstra_cluster(P, keys, idx, (cudaStream_t)stream);
+      return ea == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+    }
     cudaError_t ed = tk::launch_dykstra(P, (cudaStream_t)stream);
     return ed == cudaSuccess ? TK_OK : TK_ERR_CUDA;
   }
@@ -250,6 +270,24 @@ tk_status tk_jvp(const float* theta, const float* tangent, int64_t rows, int64_t
     e = tk::launch_vjp_state_long(P, tk::long_workspace_partials(opts->workspace, rows, (int)n),
                                   (cudaStream_t)stream);
   }
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_topk_loss(const float* theta, const int32_t* target, int64_t rows, int64_t n, int64_t k,
+                       double p, double lambda, float* loss, float* grad, const tk_opts* opts,
+                       tk_stream stream) {
+  int q4 = 0;
+  double qm1 = 0.0;
+  tk_status s = check_common(theta, rows, n, k, p, lambda, TK_MASK, &q4, &qm1);
+  if (s != TK_OK) return s;
+  if (rows == 0) return TK_OK;
+  if (loss == nullptr || grad == nullptr) return TK_ERR_INVALID_ARG;
+  // the relaxed mask y* into grad (every check of the forward pass applies), then one pass over (theta, y*)
+  s = tk_fwd_ex(theta, rows, n, k, p, lambda, TK_MASK, grad, opts, stream);
+  if (s != TK_OK) return s;
+  const int vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(grad);
+  cudaError_t e = tk::launch_loss(theta, target, grad, loss, rows, (int)n, p, lambda, q4, qm1, vec4,
+                                  (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 

@@ -19,6 +19,14 @@
 //
 // Each thread (lane) owns an even number of consecutive sorted ranks, so every C1
 // pair is thread-local and one C2 pair per thread crosses to the next thread.
+//
+// Rows of 16385..131072 elements do not fit one thread block's registers: a
+// thread-block cluster of up to 8 blocks shares the row, 16384 consecutive sorted
+// ranks per block, and the one pair that crosses from a block to the next is
+// exchanged through distributed shared memory.  The sort of such a row is the
+// global-memory radix sort (tk_long.cu); the iterate never leaves the chip.
+#include <cooperative_groups.h>
+
 #include "tk_common.cuh"
 #include "tk_cta_sort.cuh"
 #include "tk_group_sort.cuh"
@@ -234,9 +242,90 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
 }
 
+// ------------------------------------------------------------------ rows of 16385..131072 elements
+// keys, idx: the row-major result of the global-memory radix sort (keys as the complemented
+// order-preserving words it sorts ascending, idx = original index of each rank).  Block c of a
+// row's cluster owns ranks [c * kClusterSpan, (c + 1) * kClusterSpan).
+constexpr int kClusterE = 16;
+constexpr int kClusterT = 1024;
+constexpr int kClusterSpan = kClusterE * kClusterT;
+
+__global__ void __launch_bounds__(kClusterT, 1) tk_cluster_dykstra_kernel(const Problem P, const uint32_t* keys,
+                                                                          const int32_t* idx) {
+  namespace cg = cooperative_groups;
+  constexpr int E = kClusterE, T = kClusterT;
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ float xch[T];
+  const int t = threadIdx.x, n = P.n;
+  const int C = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
+  const long long row = blockIdx.x / C;
+  const Math M = make_math_q24(P);
+  const int rank0 = (c * T + t) * E;
+  const uint32_t* k_row = keys + row * (long long)n;
+  float s[E], y[E];
+#pragma unroll
+  for (int i = 0; i < E; ++i) s[i] = (rank0 + i < n) ? key2f(~__ldg(k_row + rank0 + i)) : 0.0f;
+  // The neighbour's slot is in this block's array, or in the adjacent block's through the cluster's
+  // shared-memory window.  Every exchange is write, cluster barrier, read; the solver calls sync()
+  // (a cluster barrier too) before the next exchange overwrites the slots, and ends on one, so no
+  // block leaves while a neighbour still reads its array.
+  const float* xch_next = (c + 1 < C) ? cluster.map_shared_rank(xch, c + 1) : xch;
+  const float* xch_prev = (c > 0) ? cluster.map_shared_rank(xch, c - 1) : xch;
+  const bool has_next = !(c == C - 1 && t == T - 1), has_prev = !(c == 0 && t == 0);
+  auto next_of = [&](float x) -> float {
+    xch[t] = x; cluster.sync();
+    return (t + 1 < T) ? xch[t + 1] : (has_next ? xch_next[0] : 0.0f);
+  };
+  auto prev_of = [&](float x) -> float {
+    xch[t] = x; cluster.sync();
+    return (t > 0) ? xch[t - 1] : (has_prev ? xch_prev[T - 1] : 0.0f);
+  };
+  auto sync = [&]() { cluster.sync(); };
+  solve_pairs<E>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
+
+  // un-permute: out[sigma_i] = y_i (times the sign of theta for the magnitude mode, times theta for
+  // topk).  The row was just read by the sort, so these scattered accesses are served by L2.
+  const int32_t* i_row = idx + row * (long long)n;
+  const float* x_row = P.theta + row * (long long)n;
+  float* o_row = P.out + row * (long long)n;
+#pragma unroll
+  for (int i = 0; i < E; ++i) {
+    if (rank0 + i >= n) continue;
+    const int j = __ldg(i_row + rank0 + i);
+    float q = y[i];
+    if (M.mag || P.mode == TK_TOPK) {
+      const float th = __ldg(x_row + j);
+      if (M.mag) q = (__float_as_uint(th) >> 31) ? -q : q; else q *= th;
+    }
+    o_row[j] = q;
+  }
+}
+
 }  // namespace
 
 int cta_padded_length(int n);
+
+int dykstra_cluster_max_n() { return 8 * kClusterSpan; }
+
+// Alternating projections on rows already sorted into global memory (keys, idx as above).
+cudaError_t launch_dykstra_cluster(const Problem& P, const uint32_t* keys, const int32_t* idx,
+                                   cudaStream_t stream) {
+  const int C = (P.n + kClusterSpan - 1) / kClusterSpan;
+  if (C < 1 || C > 8) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(P.rows * C));
+  cfg.blockDim = dim3(kClusterT);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = (unsigned)C;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tk_cluster_dykstra_kernel, P, keys, idx);
+}
 
 cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
   Problem P = P0;

@@ -669,6 +669,16 @@ cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_ds
   return cudaGetLastError();
 }
 
+// Where launch_long leaves the sorted rows: keys as the complemented order-preserving words (so that
+// key2f(~word) is the key), idx the original index of each rank (W_ARGSORT or perm_out only).
+void long_workspace_sorted(void* workspace, long long rows, int n, const uint32_t** keys, const int32_t** idx) {
+  const int tiles = (n + TILE - 1) / TILE;
+  size_t total = 0;
+  const LongWs ws = carve(workspace, rows, n, tiles, &total);
+  *keys = ws.keyB;
+  *idx = ws.idxB;
+}
+
 tk_rowstate* long_workspace_state(void* workspace, long long rows, int n) {
   const int tiles = (n + TILE - 1) / TILE;
   size_t total = 0;

@@ -301,6 +301,49 @@ def test_dykstra_path_matches_oracle_sweeps(p):
                 assert err <= TOL, (mode, n, k, lam, sweeps, err)
 
 
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_dykstra_cluster_rows_match_oracle_sweeps(p):
+    """Rows of 16385..131072 elements: the iterate is shared by a thread-block cluster (2, 3, 5 and 8
+    blocks here, ragged and full last blocks); same sweep count in the oracle, <= 1e-5; exact
+    permutation; a second call on the same workspace gives the same bits."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    modes = [tk.TK_MASK, tk.TK_TOPK] + ([tk.TK_TOPKMAG] if p == 2.0 else [])
+    shapes = [(16385, 2048, 1.0, 2, 10), (32768, 4096, 1.0, 3, 100), (40001, 777, 0.3, 2, 10),
+              (70000, 7000, 1.0, 1, 10), (131072, 16384, 2.0, 1, 3)]
+    for mode in modes:
+        for n, k, lam, rows, sweeps in shapes:
+            x = rows_of(n, rows, 900 + n % 97)
+            x[0, 5] = x[0, 9]                                   # a tie for the stable order
+            th = torch.from_numpy(x).cuda()
+            ws = torch.empty(tk.tk_workspace_bytes(rows, n, k, p, mode, tk.TK_SOLVER_DYKSTRA), dtype=torch.uint8,
+                             device="cuda")
+            assert ws.numel() > 0
+            outs = []
+            for _ in range(2):
+                out = torch.full_like(th, float("nan"))
+                perm = torch.empty((rows, n), dtype=torch.int32, device="cuda")
+                tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=sweeps,
+                             perm_out=perm, workspace=ws)
+                torch.cuda.synchronize()
+                outs.append(out.cpu().numpy())
+            ref = tko.dykstra(x, k, p, lam, mode, sweeps=sweeps)
+            assert np.isfinite(outs[0]).all()
+            assert np.array_equal(outs[0], outs[1])
+            assert np.array_equal(perm.cpu().numpy(), tko.argsort(x, mode)[0])
+            err = rel_err(outs[0], ref).max()
+            assert err <= TOL, (mode, n, k, lam, sweeps, err)
+    # without a workspace, and beyond eight blocks: refused before any launch
+    th = torch.zeros((1, 20000), device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 1, 20000, 5, 2.0, 1.0, tk.TK_MASK, torch.empty_like(th), solver=tk.TK_SOLVER_DYKSTRA)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+    th = torch.zeros((1, 131073), device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(th, 1, 131073, 5, 2.0, 1.0, tk.TK_MASK, torch.empty_like(th), solver=tk.TK_SOLVER_DYKSTRA)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
 def test_dykstra_default_sweeps_and_limits():
     from oracle import tko
     x = rows_of(64, 16, 77)
