@@ -329,6 +329,9 @@ def main():
                         if name.startswith("sweep_n"):
                             entry["dykstra_forward_100_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
+                        if name == "class_logit":
+                            # the loss the paper trains that classifier with (k = 3), on the same logits
+                            entry["smooth_topk_loss_k3"] = time_topk_loss(name, dev, tk, torch, k=3, peak=peak)
                         if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
                             entry["dykstra_forward_10_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
@@ -387,6 +390,32 @@ def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, 
         us = e0.elapsed_time(e1) * 1e3 / launches
         out.append({"p": round(c.p, 6), "avg_us": us, "elements_per_s": c.elements / (us * 1e-6)})
         del th, y, ws
+    return out
+
+
+def time_topk_loss(workload, dev, tk, torch, k, peak, launches=10):
+    """tk_topk_loss (forward pass + reduction pass) on the workload's logits, p = 2 and p = 4/3.
+    Algorithmic bytes: theta read once, gradient written once (8 B per element)."""
+    out = []
+    c = workload_cases(workload)[0]
+    th = torch.from_numpy(c.theta()).to(dev)
+    tgt = torch.randint(0, c.n, (c.rows,), dtype=torch.int32, device=dev)
+    loss = torch.empty((c.rows,), device=dev)
+    grad = torch.empty_like(th)
+    for p in (2.0, 4.0 / 3.0):
+        run = lambda: tk.tk_topk_loss(th, tgt, c.rows, c.n, k, p, c.lam, loss, grad)
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(launches):
+            run()
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / launches
+        out.append({"p": round(p, 6), "avg_us": us, "elements_per_s": c.elements / (us * 1e-6),
+                    "frac_of_hbm_peak": BYTES_FWD * c.elements / (us * 1e-6) / 1e9 / peak})
     return out
 
 

@@ -344,6 +344,60 @@ def test_dykstra_cluster_rows_match_oracle_sweeps(p):
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
 
 
+def test_smooth_topk_loss_matches_oracle():
+    """tk_topk_loss: loss value and gradient (mask - target) against the oracle; rows with no target;
+    both row layouts of the reduction pass (warp per row, block per row), vector and scalar access."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    shapes = [(1, 1, 1, 1.0, 2.0), (5, 2, 1, 0.5, 2.0), (64, 10, 3, 1.0, P43), (33, 100, 3, 0.3, 2.0),
+              (64, 1000, 3, 0.5, P43), (9, 1001, 5, 0.5, 2.0), (17, 2048, 64, 1.0, 2.0), (5, 5000, 50, 0.2, P43),
+              (3, 16384, 2048, 1.0, 2.0), (40, 64, 8, 1.0, 1.5), (3, 4096, 100, 0.7, 1.5)]
+    for rows, n, k, lam, p in shapes:
+        x = rows_of(n, rows, 500 + n + rows, scale=3.0)
+        rng = np.random.default_rng(n)
+        tgt = rng.integers(0, n, size=rows).astype(np.int32)
+        if rows > 2:
+            tgt[1] = -1
+            tgt[2] = n
+        th = torch.from_numpy(x).cuda()
+        loss = torch.full((rows,), float("nan"), device="cuda")
+        grad = torch.full_like(th, float("nan"))
+        tk.tk_topk_loss(th, torch.from_numpy(tgt).cuda(), rows, n, k, p, lam, loss, grad)
+        torch.cuda.synchronize()
+        lref, gref = tko.topk_loss(x, tgt, k, p, lam)
+        assert rel_err(loss.cpu().numpy(), lref).max() <= TOL, (rows, n, k, lam, p)
+        assert rel_err(grad.cpu().numpy(), gref).max() <= TOL, (rows, n, k, lam, p)
+    # no target array at all: the value f itself and the mask
+    x = rows_of(100, 7, 3)
+    th = torch.from_numpy(x).cuda()
+    loss = torch.empty((7,), device="cuda")
+    grad = torch.empty_like(th)
+    tk.tk_topk_loss(th, None, 7, 100, 3, 2.0, 1.0, loss, grad)
+    torch.cuda.synchronize()
+    lref, gref = tko.topk_loss(x, -np.ones(7), 3, 2.0, 1.0)
+    assert rel_err(loss.cpu().numpy(), lref).max() <= TOL
+    assert rel_err(grad.cpu().numpy(), tko.fwd(x, 3, 2.0, 1.0, tko.MASK)).max() <= TOL
+
+
+def test_smooth_topk_loss_class_logit_full_size():
+    """8192 x 1000 logits with forced ties, k = 3 and k = 5, p = 4/3 and 2: every row's loss and gradient."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    case = wl.class_logit_case()
+    x = case.theta()
+    rows, n = x.shape
+    tgt = np.random.default_rng(11).integers(0, n, size=rows).astype(np.int32)
+    th, tg = torch.from_numpy(x).cuda(), torch.from_numpy(tgt).cuda()
+    for k, p in [(3, P43), (5, 2.0)]:
+        loss = torch.empty((rows,), device="cuda")
+        grad = torch.empty_like(th)
+        tk.tk_topk_loss(th, tg, rows, n, k, p, case.lam, loss, grad)
+        torch.cuda.synchronize()
+        lref, gref = tko.topk_loss(x, tgt, k, p, case.lam)
+        assert rel_err(loss.cpu().numpy(), lref).max() <= TOL
+        assert rel_err(grad.cpu().numpy(), gref).max() <= TOL
+
+
 def test_dykstra_default_sweeps_and_limits():
     from oracle import tko
     x = rows_of(64, 16, 77)
