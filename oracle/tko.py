@@ -186,3 +186,19 @@ def topk_loss(theta, target, k: int, p: float, lam: float):
             loss[r] -= x64[r, tgt[r]]
             grad[r, tgt[r]] -= 1.0
     return loss, grad
+
+
+def hard(theta, k: int, mode: int = MASK) -> np.ndarray:
+    """The hard operators of Sec. 3 ("Review of operators"): with sigma the (stable, descending)
+    argsort of x -- of |x| for topkmag -- topkmask(x) has ones at sigma_1..sigma_k and zeros
+    elsewhere, topk(x) = x * topkmask(x), topkmag(x) = x * topkmask(|x|).  This is what the
+    "straight-through" use of Sec. 6 runs in the forward pass.  (rows, n) float64."""
+    x = _f32(theta)
+    rows, n = x.shape
+    if not 1 <= k <= n:
+        raise ValueError("k out of range")
+    perm, _ = argsort(x, mode)
+    keep = np.zeros((rows, n), np.float64)
+    for r in range(rows):
+        keep[r, perm[r, :k]] = 1.0
+    return keep if mode == MASK else keep * x.astype(np.float64)

@@ -652,6 +652,28 @@ def test_topk_loss_limits_and_two_element_closed_form():
         assert np.allclose(g[0], y - np.array([0.0, 1.0]), atol=1e-12)
 
 
+def test_hard_operators_match_the_paper_example_and_the_small_lambda_limit():
+    """tko.hard against the worked example of Sec. 3 (golden file) and against the relaxed
+    operators as lambda -> 0 (no ties: the limit is unique)."""
+    gold = {}
+    with open(os.path.join(GOLDEN, "hard_operators_example.txt")) as fh:
+        for line in fh:
+            if line.strip() and not line.startswith("#"):
+                key, *vals = line.split()
+                gold[key] = [int(v) for v in vals]
+    x = np.array([[0.5, -3.0, 2.0]], np.float32)       # x3 >= x1 >= x2 and |x2| >= |x3| >= |x1|
+    k = gold["k"][0]
+    assert tko.hard(x, k, tko.MASK)[0].tolist() == gold["topkmask"]
+    assert tko.hard(x, k, tko.TOPK)[0].tolist() == (np.array(gold["topk_keep"]) * x[0].astype(float)).tolist()
+    assert tko.hard(x, k, tko.TOPKMAG)[0].tolist() == (np.array(gold["topkmag_keep"]) * x[0].astype(float)).tolist()
+    xs = random_rows(6, 40, 3)
+    for mode in (tko.MASK, tko.TOPK, tko.TOPKMAG):
+        soft = tko.fwd(xs, 7, 2.0, 1e-7, mode)
+        assert np.max(np.abs(soft - tko.hard(xs, 7, mode))) <= 1e-5
+    tied = np.array([[1.0, 2.0, 2.0, 2.0, 0.0]], np.float32)     # ties: the earlier index wins
+    assert tko.hard(tied, 2, tko.MASK)[0].tolist() == [0, 1, 1, 0, 0]
+
+
 def test_invalid_arguments_are_rejected():
     x = np.zeros((1, 4), np.float32)
     for k, p, lam in [(0, 2.0, 1.0), (5, 2.0, 1.0), (2, 1.0, 1.0), (2, 2.0, 0.0)]:
