@@ -70,7 +70,9 @@ __device__ __forceinline__ void lane_sort_f<32>(float (&r)[32]) {
 template <int G, int E>
 __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned mask) {
   lane_sort_f<E>(r);
-#pragma unroll
+  // wide groups: the rounds and lane stages are loops (a round is a few hundred instructions; the
+  // unrolled network was thousands that every warp fetched once per row)
+#pragma unroll (G >= 16 ? 1 : 5)
   for (int size = 2; size <= G; size <<= 1) {
     {
       const bool keepmax = (lig & (size >> 1)) == 0;
@@ -90,7 +92,7 @@ __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned
         }
       }
     }
-#pragma unroll
+#pragma unroll (G >= 16 ? 1 : 5)
     for (int st = size >> 2; st >= 1; st >>= 1) {
       const bool keepmax = (lig & st) == 0;
 #pragma unroll
