@@ -100,7 +100,18 @@ typedef struct {
   void *workspace;         /* device scratch, 256-byte aligned, or NULL                       */
   size_t workspace_bytes;
   int32_t *status_out;     /* one device word, OR of TK_FLAG_*; the caller zeroes it          */
+  int flags;               /* OR of TK_OPT_*                                                  */
 } tk_opts;
+
+/* tk_fwd_ex only: the "straight-through" use of Sec. 6 (experiments, weight pruning).  out
+ * receives the HARD operator of Sec. 3 -- topkmask: ones at the k largest entries; topk: theta
+ * there, zero elsewhere; topkmag: the same on |theta| -- equal keys kept in ascending index,
+ * while state_out still receives the row state of the RELAXED operator, so that tk_vjp / tk_jvp
+ * from that state give the relaxed operator's derivative for the backward pass.  The hard
+ * output is read off the permutation: perm_out is required (TK_ERR_INVALID_ARG without it), and
+ * the solver must be one that sorts (not TK_SOLVER_THRESHOLD; general p has no permutation
+ * output: TK_ERR_UNSUPPORTED).                                                              */
+#define TK_OPT_STRAIGHT_THROUGH 1
 
 /* Scratch bytes tk_fwd_ex / tk_vjp / tk_argsort need for this shape: 0 for rows
  * of up to 16384 elements.  Rows of 16385..32768 elements need it only when a

@@ -21,6 +21,7 @@ TK_SOLVER_AUTO, TK_SOLVER_PAV, TK_SOLVER_DYKSTRA, TK_SOLVER_THRESHOLD = 0, 1, 2,
 TK_OK = 0
 TK_ERR_INVALID_ARG, TK_ERR_UNSUPPORTED, TK_ERR_WORKSPACE, TK_ERR_CUDA, TK_ERR_NOT_CONVERGED = 1, 2, 3, 4, 5
 TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
+TK_OPT_STRAIGHT_THROUGH = 1
 ROWSTATE_BYTES = 16
 
 EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
@@ -37,6 +38,7 @@ class TkOpts(ctypes.Structure):
         ("workspace", ctypes.c_void_p),
         ("workspace_bytes", ctypes.c_size_t),
         ("status_out", ctypes.c_void_p),
+        ("flags", ctypes.c_int),
     ]
 
 
@@ -103,8 +105,9 @@ def _stream() -> int:
 
 
 def _opts(solver=TK_SOLVER_AUTO, sweeps=0, perm_out=None, state=None, workspace=None,
-          status_out=None) -> TkOpts:
+          status_out=None, flags=0) -> TkOpts:
     o = TkOpts()
+    o.flags = int(flags)
     o.solver, o.sweeps = int(solver), int(sweeps)
     o.perm_out = _dev(perm_out, torch.int32, "perm_out")
     o.state_out = None if state is None else _dev(state, torch.uint8, "state")
@@ -142,8 +145,8 @@ def tk_fwd_noalloc(theta: torch.Tensor, rows: int, n: int, k: int, p: float, lam
 
 
 def tk_fwd_ex(theta, rows, n, k, p, lam, mode, out, *, solver=TK_SOLVER_AUTO, sweeps=0,
-              perm_out=None, state_out=None, workspace=None, status_out=None) -> None:
-    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out)
+              perm_out=None, state_out=None, workspace=None, status_out=None, flags=0) -> None:
+    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out, flags)
     rc = load().tk_fwd_ex(_dev(theta, torch.float32, "theta"), rows, n, k, p, lam, mode,
                           _dev(out, torch.float32, "out"), ctypes.byref(o), _stream())
     if rc != TK_OK:

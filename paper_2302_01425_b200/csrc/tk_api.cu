@@ -24,6 +24,9 @@ cudaError_t launch_dykstra_cluster(const Problem& P, const uint32_t* keys, const
 // smooth top-k loss from the relaxed mask (tk_loss.cu)
 cudaError_t launch_loss(const float* theta, const int32_t* target, float* grad, float* loss, long long rows,
                         int n, double p, double lambda, int q4, double qm1, int vec4, cudaStream_t stream);
+// hard operators from the permutation (tk_hard.cu)
+cudaError_t launch_hard(const float* theta, const int32_t* perm, float* out, long long rows, int n, int k,
+                        int mode, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
 cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream);
@@ -127,8 +130,8 @@ size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode
   return tk::long_workspace_bytes(rows, (int)n);
 }
 
-tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
-                    double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
+static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
+                             double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
   int q4 = 0;
   double qm1 = 0.0;
   tk_status s = check_common(theta, rows, n, k, p, lambda, mode, &q4, &qm1);
@@ -189,6 +192,19 @@ tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, doub
     return el == cudaSuccess ? TK_OK : TK_ERR_CUDA;
   }
   cudaError_t e = tk::launch_on_chip(P, (cudaStream_t)stream);
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_fwd_ex(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
+                    double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
+  const bool st = opts && (opts->flags & TK_OPT_STRAIGHT_THROUGH);
+  if (opts && (opts->flags & ~TK_OPT_STRAIGHT_THROUGH)) return TK_ERR_INVALID_ARG;
+  if (st && rows > 0 && opts->perm_out == nullptr) return TK_ERR_INVALID_ARG;
+  if (st && opts->solver == TK_SOLVER_THRESHOLD) return TK_ERR_UNSUPPORTED;
+  tk_status s = fwd_relaxed(theta, rows, n, k, p, lambda, mode, out, opts, stream);
+  if (s != TK_OK || !st || rows == 0) return s;
+  // the relaxed pass has left the permutation (and the row state); the hard operator replaces its output
+  cudaError_t e = tk::launch_hard(theta, opts->perm_out, out, rows, (int)n, (int)k, mode, (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 
@@ -281,7 +297,7 @@ tk_status tk_topk_loss(const float* theta, const int32_t* target, int64_t rows, 
   tk_status s = check_common(theta, rows, n, k, p, lambda, TK_MASK, &q4, &qm1);
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
-  if (loss == nullptr || grad == nullptr) return TK_ERR_INVALID_ARG;
+  if (loss == nullptr || grad == nullptr || (opts && opts->flags)) return TK_ERR_INVALID_ARG;
   // the relaxed mask y* into grad (every check of the forward pass applies), then one pass over (theta, y*)
   s = tk_fwd_ex(theta, rows, n, k, p, lambda, TK_MASK, grad, opts, stream);
   if (s != TK_OK) return s;

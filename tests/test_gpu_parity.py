@@ -398,6 +398,38 @@ def test_smooth_topk_loss_class_logit_full_size():
         assert rel_err(grad.cpu().numpy(), gref).max() <= TOL
 
 
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+def test_straight_through_hard_forward_relaxed_backward(mode):
+    """TK_OPT_STRAIGHT_THROUGH: the forward output is the hard operator, bit for bit (ties by index),
+    and the VJP from the saved state is the relaxed operator's."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    for n, k, lam, p, rows in [(1, 1, 1.0, 2.0, 3), (8, 3, 0.5, 2.0, 40), (64, 2, 0.1, P43, 33), (400, 28, 1.0, 2.0, 9),
+                               (1000, 5, 0.5, P43, 5), (5000, 500, 0.3, 2.0, 3), (20000, 100, 1.0, 2.0, 2)]:
+        x = rows_of(n, rows, 700 + n)
+        if n >= 8:
+            x[0, 1] = x[0, 5] = x[0, 7] = x[0].max() if mode != tk.TK_TOPKMAG else np.abs(x[0]).max()   # ties at the top
+        g = wl.cotangent_like(x, 701 + n)
+        th, gt = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+        out = torch.full_like(th, float("nan"))
+        grad = torch.empty_like(th)
+        perm = torch.empty((rows, n), dtype=torch.int32, device="cuda")
+        state = tk.new_state(rows)
+        wsb = tk.tk_workspace_bytes(rows, n, k, p, mode)
+        ws = torch.empty(wsb, dtype=torch.uint8, device="cuda") if wsb else None
+        tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, perm_out=perm, state_out=state, workspace=ws,
+                     flags=tk.TK_OPT_STRAIGHT_THROUGH)
+        tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, state=state, workspace=ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(out.cpu().numpy().astype(np.float64), tko.hard(x, k, mode)), (n, k, mode)
+        gref = tko.vjp(x, g, k, p, lam, mode)
+        assert rel_err(grad.cpu().numpy(), gref).max() <= TOL, (n, k, mode)
+    th = torch.zeros((2, 16), device="cuda")
+    with pytest.raises(tk.TkError) as e:            # the hard output is read off the permutation
+        tk.tk_fwd_ex(th, 2, 16, 3, 2.0, 1.0, mode, torch.empty_like(th), flags=tk.TK_OPT_STRAIGHT_THROUGH)
+    assert e.value.status == tk.TK_ERR_INVALID_ARG
+
+
 def test_dykstra_default_sweeps_and_limits():
     from oracle import tko
     x = rows_of(64, 16, 77)
