@@ -332,6 +332,9 @@ def main():
                         if name == "class_logit":
                             # the loss the paper trains that classifier with (k = 3), on the same logits
                             entry["smooth_topk_loss_k3"] = time_topk_loss(name, dev, tk, torch, k=3, peak=peak)
+                        if name == "expert_choice":
+                            # the same scores stored [tokens, experts]: the operator along the slow axis
+                            entry["slow_axis_fwd_vjp"] = time_cols(name, dev, tk, torch, peak)
                         if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
                             entry["dykstra_forward_10_sweeps"] = time_solver_forward(
                                 name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
@@ -391,6 +394,34 @@ def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, 
         out.append({"p": round(c.p, 6), "avg_us": us, "elements_per_s": c.elements / (us * 1e-6)})
         del th, y, ws
     return out
+
+
+def time_cols(workload, dev, tk, torch, peak, launches=10):
+    """tk_fwd_cols (state saved) + tk_vjp_cols (from state, transposed theta reused) on the workload's
+    matrix stored [n, rows]: two transposes around each pass."""
+    c = workload_cases(workload)[0]
+    x = np.ascontiguousarray(c.theta().T)
+    th = torch.from_numpy(x).to(dev)
+    gt = torch.from_numpy(np.ascontiguousarray(c.cotangent(c.theta()).T)).to(dev)
+    out, grad = torch.empty_like(th), torch.empty_like(th)
+    ws = torch.empty(tk.tk_cols_workspace_bytes(c.n, c.rows), dtype=torch.uint8, device=dev)
+    st = tk.new_state(c.rows, dev)
+
+    def run():
+        tk.tk_fwd_cols(th, c.n, c.rows, c.rows, c.k, c.p, c.lam, c.mode, out, workspace=ws, state_out=st)
+        tk.tk_vjp_cols(None, gt, c.n, c.rows, c.rows, c.k, c.p, c.lam, c.mode, grad, workspace=ws, state=st)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(launches):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / launches
+    return {"avg_us": us, "elements_per_s": c.elements / (us * 1e-6),
+            "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * c.elements / (us * 1e-6) / 1e9 / peak}
 
 
 def time_topk_loss(workload, dev, tk, torch, k, peak, launches=10):

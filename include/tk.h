@@ -163,6 +163,25 @@ tk_status tk_topk_loss(const float *theta, const int32_t *target, int64_t rows, 
                        double p, double lambda, float *loss, float *grad, const tk_opts *opts,
                        tk_stream stream);
 
+/* The operator along the slow axis of a matrix (Sec. 6, sparse MoE with expert-choice routing:
+ * every expert takes its top-k over the tokens, from a [tokens, experts] score matrix).
+ * theta, out (and grad_out, grad_theta): device, n rows of `cols` fp32 values, row i starting at
+ * element i * ld (ld >= cols, the same for every array of a call); problem c is column c:
+ *   out[:, c] = operator(theta[:, c]),   grad_theta[:, c] = J(theta[:, c])^T grad_out[:, c].
+ * The columns are transposed into opts->workspace (tk_cols_workspace_bytes, 256-byte aligned;
+ * TK_ERR_WORKSPACE without it), the row kernels run there, and the result is transposed back:
+ * one extra read and write of every array.  n <= 16384; cols <= 2^21; opts otherwise as for
+ * tk_fwd_ex / tk_vjp with rows = cols (state_out: one record per column; perm_out: [cols*n],
+ * contiguous per column).  tk_vjp_cols reads the workspace copy of theta that tk_fwd_cols left
+ * there when opts->state_out is given and theta == NULL is passed; with theta given it is
+ * transposed again.                                                                          */
+size_t tk_cols_workspace_bytes(int64_t n, int64_t cols);
+tk_status tk_fwd_cols(const float *theta, int64_t n, int64_t cols, int64_t ld, int64_t k, double p,
+                      double lambda, int mode, float *out, const tk_opts *opts, tk_stream stream);
+tk_status tk_vjp_cols(const float *theta, const float *grad_out, int64_t n, int64_t cols, int64_t ld,
+                      int64_t k, double p, double lambda, int mode, float *grad_theta,
+                      const tk_opts *opts, tk_stream stream);
+
 /* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
  * perm_out[i] = index of the i-th largest key (theta, or |theta| for
  * TK_TOPKMAG), equal keys in ascending index, -0 == +0.  sorted_out (may be

@@ -25,7 +25,8 @@ TK_OPT_STRAIGHT_THROUGH = 1
 ROWSTATE_BYTES = 16
 
 EXPORTS = ("tk_version", "tk_status_string", "tk_workspace_bytes", "tk_fwd", "tk_fwd_ex", "tk_vjp",
-           "tk_jvp", "tk_argsort", "tk_fwd_noalloc", "tk_topk_loss")
+           "tk_jvp", "tk_argsort", "tk_fwd_noalloc", "tk_topk_loss",
+           "tk_cols_workspace_bytes", "tk_fwd_cols", "tk_vjp_cols")
 TK_NOALLOC_MAX_ELEMENTS = 1 << 18
 
 
@@ -78,6 +79,12 @@ def load() -> ctypes.CDLL:
     lib.tk_jvp.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_topk_loss.restype = ci
     lib.tk_topk_loss.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, vp, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_cols_workspace_bytes.restype = ctypes.c_size_t
+    lib.tk_cols_workspace_bytes.argtypes = [i64, i64]
+    lib.tk_fwd_cols.restype = ci
+    lib.tk_fwd_cols.argtypes = [vp, i64, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_vjp_cols.restype = ci
+    lib.tk_vjp_cols.argtypes = [vp, vp, i64, i64, i64, i64, dbl, dbl, ci, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_argsort.restype = ci
     lib.tk_argsort.argtypes = [vp, i64, i64, ci, vp, vp, ctypes.POINTER(TkOpts), vp]
     _lib = lib
@@ -181,6 +188,29 @@ def tk_topk_loss(theta, target, rows, n, k, p, lam, loss, grad, *, solver=TK_SOL
                              _dev(grad, torch.float32, "grad"), ctypes.byref(o), _stream())
     if rc != TK_OK:
         raise TkError(rc, "tk_topk_loss")
+
+
+def tk_cols_workspace_bytes(n: int, cols: int) -> int:
+    return int(load().tk_cols_workspace_bytes(n, cols))
+
+
+def tk_fwd_cols(theta, n, cols, ld, k, p, lam, mode, out, *, workspace, solver=TK_SOLVER_AUTO, sweeps=0,
+                perm_out=None, state_out=None, status_out=None, flags=0) -> None:
+    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out, flags)
+    rc = load().tk_fwd_cols(_dev(theta, torch.float32, "theta"), n, cols, ld, k, p, lam, mode,
+                            _dev(out, torch.float32, "out"), ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_fwd_cols")
+
+
+def tk_vjp_cols(theta, grad_out, n, cols, ld, k, p, lam, mode, grad_theta, *, workspace, state=None,
+                status_out=None) -> None:
+    o = _opts(state=state, workspace=workspace, status_out=status_out)
+    rc = load().tk_vjp_cols(_dev(theta, torch.float32, "theta"), _dev(grad_out, torch.float32, "grad_out"),
+                            n, cols, ld, k, p, lam, mode, _dev(grad_theta, torch.float32, "grad_theta"),
+                            ctypes.byref(o), _stream())
+    if rc != TK_OK:
+        raise TkError(rc, "tk_vjp_cols")
 
 
 def tk_argsort(theta, rows, n, mode, perm_out, sorted_out=None, *, workspace=None,

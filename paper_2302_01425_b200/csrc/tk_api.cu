@@ -27,6 +27,9 @@ cudaError_t launch_loss(const float* theta, const int32_t* target, float* grad, 
 // hard operators from the permutation (tk_hard.cu)
 cudaError_t launch_hard(const float* theta, const int32_t* perm, float* out, long long rows, int n, int k,
                         int mode, cudaStream_t stream);
+// [n, cols] with leading dimension <-> contiguous [cols, n] (tk_transpose.cu)
+cudaError_t launch_transpose(const float* in, long long in_rows, long long in_cols, long long in_ld, float* out,
+                             long long out_ld, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
 cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream);
@@ -305,6 +308,69 @@ tk_status tk_topk_loss(const float* theta, const int32_t* target, int64_t rows, 
   cudaError_t e = tk::launch_loss(theta, target, grad, loss, rows, (int)n, p, lambda, q4, qm1, vec4,
                                   (cudaStream_t)stream);
   return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+// ---- the operator along the slow axis: transpose into the workspace, row kernels, transpose back
+static size_t cols_slab_bytes(int64_t n, int64_t cols) {
+  return ((size_t)n * (size_t)cols * sizeof(float) + 255) & ~size_t(255);
+}
+
+size_t tk_cols_workspace_bytes(int64_t n, int64_t cols) {
+  if (n < 1 || cols < 1 || n > tk::kMaxOnChipN || cols > (int64_t(1) << 21)) return 0;
+  return 3 * cols_slab_bytes(n, cols);
+}
+
+static tk_status check_cols(int64_t n, int64_t cols, int64_t ld, const tk_opts* opts, float** slab) {
+  if (cols < 0 || n < 1 || ld < cols) return TK_ERR_INVALID_ARG;
+  if (n > tk::kMaxOnChipN || cols > (int64_t(1) << 21)) return TK_ERR_UNSUPPORTED;
+  if (cols == 0) return TK_OK;
+  if (!opts || !opts->workspace || (reinterpret_cast<uintptr_t>(opts->workspace) & 255u)) return TK_ERR_WORKSPACE;
+  if (opts->workspace_bytes < tk_cols_workspace_bytes(n, cols)) return TK_ERR_WORKSPACE;
+  const size_t slab_bytes = cols_slab_bytes(n, cols);
+  for (int i = 0; i < 3; ++i) slab[i] = reinterpret_cast<float*>(static_cast<char*>(opts->workspace) + i * slab_bytes);
+  return TK_OK;
+}
+
+tk_status tk_fwd_cols(const float* theta, int64_t n, int64_t cols, int64_t ld, int64_t k, double p,
+                      double lambda, int mode, float* out, const tk_opts* opts, tk_stream stream) {
+  float* slab[3] = {nullptr, nullptr, nullptr};
+  tk_status s = check_cols(n, cols, ld, opts, slab);
+  if (s != TK_OK) return s;
+  int q4 = 0; double qm1 = 0.0;
+  s = check_common(theta, cols, n, k, p, lambda, mode, &q4, &qm1);
+  if (s != TK_OK) return s;
+  if (cols == 0) return TK_OK;
+  if (out == nullptr) return TK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (tk::launch_transpose(theta, n, cols, ld, slab[0], n, st) != cudaSuccess) return TK_ERR_CUDA;
+  tk_opts inner = *opts;
+  inner.workspace = nullptr; inner.workspace_bytes = 0;
+  s = tk_fwd_ex(slab[0], cols, n, k, p, lambda, mode, slab[1], &inner, stream);
+  if (s != TK_OK) return s;
+  return tk::launch_transpose(slab[1], cols, n, n, out, ld, st) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_vjp_cols(const float* theta, const float* grad_out, int64_t n, int64_t cols, int64_t ld,
+                      int64_t k, double p, double lambda, int mode, float* grad_theta,
+                      const tk_opts* opts, tk_stream stream) {
+  float* slab[3] = {nullptr, nullptr, nullptr};
+  tk_status s = check_cols(n, cols, ld, opts, slab);
+  if (s != TK_OK) return s;
+  // theta == NULL: the transposed copy a forward call left in the workspace (needs its row state too)
+  const bool reuse = theta == nullptr && opts && opts->state_out != nullptr;
+  int q4 = 0; double qm1 = 0.0;
+  s = check_common(reuse ? (const void*)slab : (const void*)theta, cols, n, k, p, lambda, mode, &q4, &qm1);
+  if (s != TK_OK) return s;
+  if (cols == 0) return TK_OK;
+  if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!reuse && tk::launch_transpose(theta, n, cols, ld, slab[0], n, st) != cudaSuccess) return TK_ERR_CUDA;
+  if (tk::launch_transpose(grad_out, n, cols, ld, slab[1], n, st) != cudaSuccess) return TK_ERR_CUDA;
+  tk_opts inner = *opts;
+  inner.workspace = nullptr; inner.workspace_bytes = 0;
+  s = tk_vjp(slab[0], slab[1], cols, n, k, p, lambda, mode, slab[2], &inner, stream);
+  if (s != TK_OK) return s;
+  return tk::launch_transpose(slab[2], cols, n, n, grad_theta, ld, st) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
 }
 
 tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int32_t* perm_out,

@@ -430,6 +430,48 @@ def test_straight_through_hard_forward_relaxed_backward(mode):
     assert e.value.status == tk.TK_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+def test_operator_along_the_slow_axis(mode):
+    """tk_fwd_cols / tk_vjp_cols on [n, cols] matrices with a leading dimension: every column against
+    the oracle on that column; ragged tiles (neither n nor cols a multiple of 32), ld > cols, the
+    padding columns left untouched; the VJP with theta given and with the workspace copy reused."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    for n, cols, ld, k, lam, p in [(1, 1, 1, 1, 1.0, 2.0), (5, 3, 3, 2, 0.5, 2.0), (33, 70, 77, 7, 0.3, P43),
+                                   (400, 32, 32, 28, 1.0, 2.0), (64, 1000, 1024, 2, 0.1, 2.0), (1500, 37, 40, 150, 1.0, P43)]:
+        if mode == tk.TK_TOPKMAG and p != 2.0 and n > 1000:
+            continue
+        rng = np.random.default_rng(n * 1000 + cols)
+        x = rng.standard_normal((n, ld)).astype(np.float32)
+        g = rng.standard_normal((n, ld)).astype(np.float32)
+        th, gt = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+        out = torch.full_like(th, -7.0)
+        grad = torch.full_like(th, -7.0)
+        grad2 = torch.full_like(th, -7.0)
+        ws = torch.empty(tk.tk_cols_workspace_bytes(n, cols), dtype=torch.uint8, device="cuda")
+        state = tk.new_state(cols)
+        tk.tk_fwd_cols(th, n, cols, ld, k, p, lam, mode, out, workspace=ws, state_out=state)
+        tk.tk_vjp_cols(None, gt, n, cols, ld, k, p, lam, mode, grad, workspace=ws, state=state)   # reuses theta^T
+        tk.tk_vjp_cols(th, gt, n, cols, ld, k, p, lam, mode, grad2, workspace=ws)                 # recomputes
+        torch.cuda.synchronize()
+        xt, gtt = np.ascontiguousarray(x[:, :cols].T), np.ascontiguousarray(g[:, :cols].T)
+        ref = tko.fwd(xt, k, p, lam, mode).T
+        gref = tko.vjp(xt, gtt, k, p, lam, mode).T
+        o, gr, gr2 = out.cpu().numpy(), grad.cpu().numpy(), grad2.cpu().numpy()
+        assert rel_err(o[:, :cols], ref).max() <= TOL, (n, cols, mode)
+        assert rel_err(gr[:, :cols], gref).max() <= TOL, (n, cols, mode)
+        assert rel_err(gr2[:, :cols], gref).max() <= TOL, (n, cols, mode)
+        assert (o[:, cols:] == -7.0).all() and (gr[:, cols:] == -7.0).all()
+    th = torch.zeros((8, 8), device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_cols(th, 8, 8, 8, 2, 2.0, 1.0, mode, torch.empty_like(th), workspace=None)
+    assert e.value.status == tk.TK_ERR_WORKSPACE
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_cols(th, 8, 8, 4, 2, 2.0, 1.0, mode, torch.empty_like(th),
+                       workspace=torch.empty(4096, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == tk.TK_ERR_INVALID_ARG
+
+
 def test_dykstra_default_sweeps_and_limits():
     from oracle import tko
     x = rows_of(64, 16, 77)
