@@ -38,11 +38,9 @@ __device__ __forceinline__ void sort_registers_f(float (&r)[E]) {   // bitonic n
 
 // The warp's 32 E keys, each lane's E already descending -> descending across the warp (lane l
 // ends with ranks [l E, l E + E) of the warp's keys): bitonic merges through shuffles.
-// The rounds and the lane stages are loops, not unrolled copies: a round is a few hundred
-// instructions, the unrolled network was several thousand that every warp fetched once per row.
 template <int E>
 __device__ __forceinline__ void warp_sort_keys(float (&r)[E], int lane) {
-#pragma unroll 1
+#pragma unroll
   for (int size = 2; size <= 32; size <<= 1) {
     {
       const bool keepmax = (lane & (size >> 1)) == 0;
@@ -54,7 +52,7 @@ __device__ __forceinline__ void warp_sort_keys(float (&r)[E], int lane) {
         r[E - 1 - i] = keepmax ? fmaxf(r[E - 1 - i], ob) : fminf(r[E - 1 - i], ob);
       }
     }
-#pragma unroll 1
+#pragma unroll
     for (int st = size >> 2; st >= 1; st >>= 1) {
       const bool keepmax = (lane & st) == 0;
 #pragma unroll

@@ -70,9 +70,11 @@ __device__ __forceinline__ void lane_sort_f<32>(float (&r)[32]) {
 template <int G, int E>
 __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned mask) {
   lane_sort_f<E>(r);
-  // wide groups: the rounds and lane stages are loops (a round is a few hundred instructions; the
-  // unrolled network was thousands that every warp fetched once per row)
-#pragma unroll (G >= 16 ? 1 : 5)
+  // 16 or 32 keys per lane: the rounds and lane stages are loops (a round is a few hundred
+  // instructions; unrolled, the network is thousands that every warp fetches once per row).
+  // Measured per 2^25 elements: n = 512 324 -> 313 us (p = 4/3: 392 -> 365), n = 1024 422 -> 411;
+  // with 8 keys per lane the loops lose (n = 128: 175 -> 203 us), so those stay unrolled.
+#pragma unroll (E >= 16 ? 1 : 5)
   for (int size = 2; size <= G; size <<= 1) {
     {
       const bool keepmax = (lig & (size >> 1)) == 0;
@@ -92,7 +94,7 @@ __device__ __forceinline__ void group_sort_keys(float (&r)[E], int lig, unsigned
         }
       }
     }
-#pragma unroll (G >= 16 ? 1 : 5)
+#pragma unroll (E >= 16 ? 1 : 5)
     for (int st = size >> 2; st >= 1; st >>= 1) {
       const bool keepmax = (lig & st) == 0;
 #pragma unroll
