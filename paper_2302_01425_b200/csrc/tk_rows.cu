@@ -314,8 +314,11 @@ struct RowsGeom {
 };
 
 // QM: 0 for q = 2, 1 for q = 4, 2 for any other q (short rows, mask and top-k modes)
+// Resident blocks asked of the compiler: 6 with 8 or 16 keys per lane (16 keys: 76 registers instead
+// of 82, no spills, and n = 300..512 runs 6 % faster than at 5 blocks; 8 keys: 8 blocks of half the
+// batches were measured 3-17 % slower), 3 with 32.
 template <int G, int E, int B, int QM, bool MAG>
-__global__ void __launch_bounds__(kRowsThreads, E == 8 ? 6 : (E == 16 ? 4 : 3)) tk_rows_kernel(const Problem P) {
+__global__ void __launch_bounds__(kRowsThreads, E <= 16 ? 6 : 3) tk_rows_kernel(const Problem P) {
   constexpr bool Q4 = QM == 1, GEN = QM == 2;
   constexpr int RPB = RowsGeom<G, E, B>::RPB, R = RowsGeom<G, E, B>::R, BATCHES = B;
   constexpr int STRIDE = RowsGeom<G, E, B>::STRIDE;
