@@ -49,6 +49,9 @@ __device__ __forceinline__ void dyk_pair(float& a, float& b, float& delta, float
 __device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w2, float a_prev,
                                            float a_next, const Math& M) {
   const float c1 = w1 + a_prev, c2 = w2 - a_next;
+  // s1 >= s2, so the separate minimisers s_i - lam cbrt(c_i) are in order whenever c1 <= c2: most
+  // pairs (equal weights, no active neighbour) end here without a cube root
+  if (c1 <= c2) return 0.0f;
   const float v1 = s1 - M.lam * cbrtf(c1), v2 = s2 - M.lam * cbrtf(c2);
   if (v1 >= v2) return 0.0f;
   const float d = 0.5f * (s1 - s2), m = 0.5f * (s1 + s2);
@@ -68,8 +71,10 @@ __device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w
 // The solver on E consecutive ranks per thread.  Exchange with the neighbouring threads goes
 // through the two callables: next0(x) returns the NEXT thread's x, prev_last(x) the PREVIOUS thread's.
 // On return y[i] = rho(s_i - v_i).
-template <int E, typename NextF, typename PrevF, typename SyncF>
-__device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
+// MAG (phi even) is a template flag: for phi = x every metric weight is the constant 1, the pair
+// projection loses its division and the weights their registers.
+template <int E, bool MAG, typename NextF, typename PrevF, typename SyncF>
+__device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, const float (&s)[E], int rank0,
                                             bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
                                             SyncF sync, float (&y)[E]) {
   const int n = P.n, k = P.k;
@@ -83,12 +88,12 @@ __device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, con
 #pragma unroll
     for (int i = 0; i < E; ++i) {
       const float w = wgt(rank0 + i);
-      c[i] = M.mag ? 1.0f + M.lam * w : 1.0f;
-      v[i] = M.mag ? s[i] / c[i] : s[i] - M.lam * w;
+      c[i] = MAG ? 1.0f + M.lam * w : 1.0f;
+      v[i] = MAG ? s[i] / c[i] : s[i] - M.lam * w;
     }
 #pragma unroll
     for (int j = 0; j < E / 2; ++j) { pd[j] = 0.0f; qd[j] = 0.0f; }
-    const float c_next = M.mag ? 1.0f + M.lam * wgt(rank0 + E) : 1.0f;
+    const float c_next = MAG ? 1.0f + M.lam * wgt(rank0 + E) : 1.0f;
 #pragma unroll 1
     for (int it = 0; it < sweeps; ++it) {
 #pragma unroll
@@ -109,7 +114,7 @@ __device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, con
     }
 #pragma unroll
     for (int i = 0; i < E; ++i) {
-      const float vi = M.mag ? fmaxf(v[i], 0.0f) : v[i];
+      const float vi = MAG ? fmaxf(v[i], 0.0f) : v[i];
       y[i] = (s[i] - vi) * M.inv_lam;
     }
   } else {
@@ -151,6 +156,14 @@ __device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, con
       y[i] = wgt(rank0 + i) - a_i + a_im1;
     }
   }
+}
+
+template <int E, typename NextF, typename PrevF, typename SyncF>
+__device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
+                                            bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
+                                            SyncF sync, float (&y)[E]) {
+  if (M.mag) solve_pairs_m<E, true>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
+  else solve_pairs_m<E, false>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
 }
 
 // ------------------------------------------------------------------ rows of up to 256 elements
@@ -211,7 +224,8 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   const Math M = make_math_q24(P);
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
   float* stage = reinterpret_cast<float*>(smem_raw);
-  float* xch = reinterpret_cast<float*>(keys + pad(N) + 1);   // T + 2 floats
+  float* xch_a = reinterpret_cast<float*>(keys + pad(N) + 1);   // 2 x (T + 2) floats
+  float* xch_b = xch_a + (T + 2);
   const float* x_row = P.theta + row * (long long)n;
   unsigned long long r[E];
   bool bad = false;
@@ -223,11 +237,15 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   float s[E], y[E];
 #pragma unroll
   for (int i = 0; i < E; ++i) s[i] = un_key(r[i]);
-  // neighbour exchange through xch[]: write own value, barrier, read the neighbour's slot.  The
-  // solver calls sync() after every exchange before the next one overwrites the buffer.
-  auto next_of = [&](float x) -> float { xch[t] = x; __syncthreads(); return (t + 1 < T) ? xch[t + 1] : 0.0f; };
-  auto prev_of = [&](float x) -> float { xch[t] = x; __syncthreads(); return (t > 0) ? xch[t - 1] : 0.0f; };
-  auto sync = [&]() { __syncthreads(); };
+  // Neighbour exchange: write own value, barrier, read the neighbour's slot.  The solver alternates
+  // the two kinds of exchange and each has its own array, so a slot is overwritten only after the
+  // barrier of the other kind's exchange, which every thread passes after its read: the solver's
+  // sync() between exchanges needs a barrier only after the one exchange that precedes the sweeps
+  // (it is followed by another of its kind).  Two block barriers per sweep.
+  auto next_of = [&](float x) -> float { xch_a[t] = x; __syncthreads(); return (t + 1 < T) ? xch_a[t + 1] : 0.0f; };
+  auto prev_of = [&](float x) -> float { xch_b[t] = x; __syncthreads(); return (t > 0) ? xch_b[t - 1] : 0.0f; };
+  bool before_sweeps = true;
+  auto sync = [&]() { if (before_sweeps) { __syncthreads(); before_sweeps = false; } };
   solve_pairs<E>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, y);
 
   __syncthreads();
@@ -255,7 +273,7 @@ __global__ void __launch_bounds__(kClusterT, 1) tk_cluster_dykstra_kernel(const 
   namespace cg = cooperative_groups;
   constexpr int E = kClusterE, T = kClusterT;
   cg::cluster_group cluster = cg::this_cluster();
-  __shared__ float xch[T];
+  __shared__ float xch_a[T], xch_b[T];
   const int t = threadIdx.x, n = P.n;
   const int C = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
   const long long row = blockIdx.x / C;
@@ -266,22 +284,28 @@ __global__ void __launch_bounds__(kClusterT, 1) tk_cluster_dykstra_kernel(const 
 #pragma unroll
   for (int i = 0; i < E; ++i) s[i] = (rank0 + i < n) ? key2f(~__ldg(k_row + rank0 + i)) : 0.0f;
   // The neighbour's slot is in this block's array, or in the adjacent block's through the cluster's
-  // shared-memory window.  Every exchange is write, cluster barrier, read; the solver calls sync()
-  // (a cluster barrier too) before the next exchange overwrites the slots, and ends on one, so no
-  // block leaves while a neighbour still reads its array.
-  const float* xch_next = (c + 1 < C) ? cluster.map_shared_rank(xch, c + 1) : xch;
-  const float* xch_prev = (c > 0) ? cluster.map_shared_rank(xch, c - 1) : xch;
+  // shared-memory window.  Every exchange is write, cluster barrier, read.  The solver alternates
+  // the two kinds of exchange, and each has its own array: a thread overwrites its slot of one
+  // array only after the barrier of the other kind's exchange, which every thread passes after
+  // its read of the first.  So the solver's sync() between exchanges needs no barrier of its own
+  // (two cluster barriers per sweep instead of four), except after the one exchange that precedes
+  // the sweeps, which is followed by another of its kind.  A last barrier keeps every block
+  // resident until its neighbours have read its arrays.
+  const float* nxt_a = (c + 1 < C) ? cluster.map_shared_rank(xch_a, c + 1) : xch_a;
+  const float* prv_b = (c > 0) ? cluster.map_shared_rank(xch_b, c - 1) : xch_b;
   const bool has_next = !(c == C - 1 && t == T - 1), has_prev = !(c == 0 && t == 0);
   auto next_of = [&](float x) -> float {
-    xch[t] = x; cluster.sync();
-    return (t + 1 < T) ? xch[t + 1] : (has_next ? xch_next[0] : 0.0f);
+    xch_a[t] = x; cluster.sync();
+    return (t + 1 < T) ? xch_a[t + 1] : (has_next ? nxt_a[0] : 0.0f);
   };
   auto prev_of = [&](float x) -> float {
-    xch[t] = x; cluster.sync();
-    return (t > 0) ? xch[t - 1] : (has_prev ? xch_prev[T - 1] : 0.0f);
+    xch_b[t] = x; cluster.sync();
+    return (t > 0) ? xch_b[t - 1] : (has_prev ? prv_b[T - 1] : 0.0f);
   };
-  auto sync = [&]() { cluster.sync(); };
+  bool before_sweeps = true;
+  auto sync = [&]() { if (before_sweeps) { cluster.sync(); before_sweeps = false; } };
   solve_pairs<E>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
+  cluster.sync();
 
   // un-permute: out[sigma_i] = y_i (times the sign of theta for the magnitude mode, times theta for
   // topk).  The row was just read by the sort, so these scattered accesses are served by L2.
@@ -348,7 +372,7 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
   P.N = cta_padded_length(P.n);
   const int E = P.N >= 4096 ? 16 : (P.N >= 1024 ? 8 : 4);
   const int T = P.N / E;
-  const size_t smem = (size_t)(P.N + (P.N >> PAD_SHIFT) + 1) * 8 + (size_t)(T + 2) * 4 + 16;
+  const size_t smem = (size_t)(P.N + (P.N >> PAD_SHIFT) + 1) * 8 + (size_t)(T + 2) * 8 + 16;
   void (*kern)(const Problem) = nullptr;
   int slot;
   switch (E) {
@@ -364,7 +388,7 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
-    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 1) * 8 + (1024 + 2) * 4 + 16;
+    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 1) * 8 + (1024 + 2) * 8 + 16;
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (err != cudaSuccess) return err;
     if (dev >= 0 && dev < 64) configured[slot][dev] = true;
