@@ -73,10 +73,12 @@ __device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w
 // On return y[i] = rho(s_i - v_i).
 // MAG (phi even) is a template flag: for phi = x every metric weight is the constant 1, the pair
 // projection loses its division and the weights their registers.
-template <int E, bool MAG, typename NextF, typename PrevF, typename SyncF>
+// key_again(i): the key s[i] once more, for the output map of the p = 2 iteration, which does not
+// touch s between its first line and its last: a kernel short of registers reads it from memory there.
+template <int E, bool MAG, typename NextF, typename PrevF, typename SyncF, typename KeyF>
 __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, const float (&s)[E], int rank0,
                                             bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
-                                            SyncF sync, float (&y)[E]) {
+                                            SyncF sync, KeyF key_again, float (&y)[E]) {
   const int n = P.n, k = P.k;
   const int sweeps = P.sweeps > 0 ? P.sweeps : 100;
   const float s_next = next_of(s[0]);                      // key of the next thread's first rank
@@ -115,7 +117,7 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
 #pragma unroll
     for (int i = 0; i < E; ++i) {
       const float vi = MAG ? fmaxf(v[i], 0.0f) : v[i];
-      y[i] = (s[i] - vi) * M.inv_lam;
+      y[i] = (key_again(i) - vi) * M.inv_lam;
     }
   } else {
     // alpha of constraint (rank0 + i, rank0 + i + 1): i even -> ao[i/2], i odd -> ae[i/2]
@@ -158,12 +160,12 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
   }
 }
 
-template <int E, typename NextF, typename PrevF, typename SyncF>
+template <int E, typename NextF, typename PrevF, typename SyncF, typename KeyF>
 __device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
                                             bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
-                                            SyncF sync, float (&y)[E]) {
-  if (M.mag) solve_pairs_m<E, true>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
-  else solve_pairs_m<E, false>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
+                                            SyncF sync, KeyF key_again, float (&y)[E]) {
+  if (M.mag) solve_pairs_m<E, true>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
+  else solve_pairs_m<E, false>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
 }
 
 // ------------------------------------------------------------------ rows of up to 256 elements
@@ -197,7 +199,8 @@ __global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) 
   auto next_of = [&](float x) -> float { return __shfl_down_sync(mask, x, 1, G); };
   auto prev_of = [&](float x) -> float { return __shfl_up_sync(mask, x, 1, G); };
   auto sync = [&]() {};
-  solve_pairs<EPL>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync, y);
+  solve_pairs<EPL>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync,
+                   [&](int i) -> float { return s[i]; }, y);
 
   float* stage = stage_all[grp];
 #pragma unroll
@@ -246,7 +249,7 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   auto prev_of = [&](float x) -> float { xch_b[t] = x; __syncthreads(); return (t > 0) ? xch_b[t - 1] : 0.0f; };
   bool before_sweeps = true;
   auto sync = [&]() { if (before_sweeps) { __syncthreads(); before_sweeps = false; } };
-  solve_pairs<E>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, y);
+  solve_pairs<E>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, [&](int i) -> float { return s[i]; }, y);
 
   __syncthreads();
 #pragma unroll
@@ -304,7 +307,11 @@ __global__ void __launch_bounds__(kClusterT, 1) tk_cluster_dykstra_kernel(const 
   };
   bool before_sweeps = true;
   auto sync = [&]() { if (before_sweeps) { cluster.sync(); before_sweeps = false; } };
-  solve_pairs<E>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, y);
+  // 1024 threads leave 64 registers each: the keys are read again (L2) for the output map instead
+  // of living through the sweeps, which keeps the iterate and its corrections out of local memory
+  // (spill traffic was also what every cluster barrier's fence waited for)
+  auto key_again = [&](int i) -> float { return (rank0 + i < n) ? key2f(~__ldg(k_row + rank0 + i)) : 0.0f; };
+  solve_pairs<E>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
   cluster.sync();
 
   // un-permute: out[sigma_i] = y_i (times the sign of theta for the magnitude mode, times theta for
