@@ -77,23 +77,29 @@ def hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def kernel_source_hash() -> str:
+def kernel_source_hash(sources=None) -> str:
+    """Hash of the kernel sources a traffic record depends on: the listed files (paths relative to the
+    repository root: the kernel's translation unit and every header it includes), or all of csrc/."""
     h = hashlib.sha256()
-    csrc = os.path.join(ROOT, "paper_2302_01425_b200", "csrc")
-    for f in sorted(os.listdir(csrc)):
-        with open(os.path.join(csrc, f), "rb") as fh:
+    if sources:
+        paths = [os.path.join(ROOT, f) for f in sources]
+    else:
+        csrc = os.path.join(ROOT, "paper_2302_01425_b200", "csrc")
+        paths = [os.path.join(csrc, f) for f in sorted(os.listdir(csrc))]
+    for path in paths:
+        with open(path, "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
 
 
 def recorded_traffic(workload: str, kernel: str):
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary; None when
-    absent or taken on different kernel sources."""
+    absent or taken on different sources of that kernel."""
     try:
         with open(os.path.join(ROOT, "profiles", "traffic.json")) as fh:
             rec = json.load(fh)
         e = rec[workload][kernel]
-        if e.get("source_hash") != kernel_source_hash():
+        if e.get("source_hash") != kernel_source_hash(e.get("sources")):
             return None
         return e["dram_bytes_per_launch"]
     except Exception:
