@@ -69,11 +69,12 @@ typedef enum {
   TK_ERR_INVALID_ARG = 1,   /* null pointer, k out of range, lambda <= 0, p <= 1, ...        */
   TK_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for                    */
   TK_ERR_WORKSPACE = 3,     /* workspace missing or smaller than tk_workspace_bytes          */
-  TK_ERR_CUDA = 4,          /* a CUDA runtime call (launch, attribute) failed                */
-  TK_ERR_NOT_CONVERGED = 5
+  TK_ERR_CUDA = 4           /* a CUDA runtime call (launch, attribute) failed                */
 } tk_status;
 
-/* bits OR-ed into *tk_opts.status_out by the kernels */
+/* bits OR-ed into *tk_opts.status_out by the kernels.  An iteration that stops at its cap is
+ * reported here and nowhere else: the host never waits for the device, so no entry point can
+ * return it as a status.                                                                       */
 #define TK_FLAG_NONFINITE 1      /* some input was NaN or Inf                                */
 #define TK_FLAG_NOT_CONVERGED 2  /* an iterative solve stopped at its iteration cap          */
 
@@ -194,23 +195,29 @@ tk_status tk_argsort(const float *theta, int64_t rows, int64_t n, int mode, int3
  * when they need the operator: a plugin inside an application that owns the
  * allocator, a real-time loop that must not hit cudaMalloc's implicit device
  * synchronisation, a process whose memory pool is fully committed.  Such callers
- * can use tk_fwd for rows of up to 16384 elements (which needs no scratch), but
+ * can use tk_fwd for rows of up to 32768 elements (which needs no scratch), but
  * tk_fwd_ex wants a workspace for longer rows; this call does not.
  *
  * Arguments, layout and results are those of tk_fwd (all pointers device
  * pointers owned by the caller; out[r, :] = operator(theta[r, :]); work is
- * enqueued on `stream`).  Rows of up to 16384 elements are passed straight to
+ * enqueued on `stream`).  Rows of up to 32768 elements are passed straight to
  * tk_fwd.  Longer rows run the global-memory pipeline of tk_fwd_ex on a scratch
  * array compiled into the library: TK_NOALLOC_SCRATCH_BYTES of device memory
- * that every GPU holds from the moment it loads the library until the process
- * exits.  The call itself performs no allocation of any kind.
+ * that a GPU holds from the moment the CUDA runtime loads the library's module
+ * on it until the process exits.  The call never asks an allocator for memory
+ * (no cudaMalloc, cudaFree or allocating library routine).
  *
  *  - Limit: rows * n <= TK_NOALLOC_MAX_ELEMENTS (and the scratch the shape needs
  *    must fit the array); anything larger returns TK_ERR_WORKSPACE before any
  *    launch.  Use tk_fwd_ex with your own workspace for bigger problems.
  *  - The first call on a device looks up the array's device address
- *    (cudaGetSymbolAddress) with that device current; make that first call
- *    outside of any stream capture.
+ *    (cudaGetSymbolAddress) with that device current.  With CUDA's default lazy
+ *    module loading that lookup is also what loads the module, and with it
+ *    reserves the array, on that device: it is the one call that can fail with
+ *    TK_ERR_CUDA when the device has no room left.  Make it once at start-up,
+ *    before the memory pool is committed and outside of any stream capture.
+ *    The address is not looked up again: after cudaDeviceReset it is stale and
+ *    this entry point must not be used in that process any more.
  *  - All calls on a device share the one array.  It keeps whatever the previous
  *    call left in it, which is harmless (every word is written before it is read
  *    within a call), but two calls whose kernels overlap on the GPU -- different

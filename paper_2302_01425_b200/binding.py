@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libtk.so")
 TK_MASK, TK_TOPK, TK_TOPKMAG = 0, 1, 2
 TK_SOLVER_AUTO, TK_SOLVER_PAV, TK_SOLVER_DYKSTRA, TK_SOLVER_THRESHOLD = 0, 1, 2, 3
 TK_OK = 0
-TK_ERR_INVALID_ARG, TK_ERR_UNSUPPORTED, TK_ERR_WORKSPACE, TK_ERR_CUDA, TK_ERR_NOT_CONVERGED = 1, 2, 3, 4, 5
+TK_ERR_INVALID_ARG, TK_ERR_UNSUPPORTED, TK_ERR_WORKSPACE, TK_ERR_CUDA = 1, 2, 3, 4
 TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
 TK_OPT_STRAIGHT_THROUGH = 1
 ROWSTATE_BYTES = 16

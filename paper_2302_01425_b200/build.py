@@ -16,7 +16,7 @@ LIB = os.path.join(_PKG, "libtk.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-    "--use_fast_math=false", "-Xcompiler", "-fPIC", "-shared", "--threads", "0",
+    "-Xcompiler", "-fPIC", "-shared", "--threads", "0",
 ]
 
 
@@ -38,7 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc] + [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+    cmd = [nvcc] + NVCC_FLAGS
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()

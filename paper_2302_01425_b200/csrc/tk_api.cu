@@ -14,8 +14,10 @@ cudaError_t launch_group(const Problem& P, cudaStream_t stream);
 cudaError_t launch_rows(const Problem& P, cudaStream_t stream);
 // block-per-row kernel with a key-only sort and results by value (tk_ctav.cu)
 cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
-// exact forward pass without a sort (tk_thr.cu)
+// exact forward pass without a sort (tk_thr.cu); the same for phi(x) = x with rows in registers (tk_newton.cu)
 cudaError_t launch_thr(const Problem& P, cudaStream_t stream);
+cudaError_t launch_newton(const Problem& P, cudaStream_t stream);
+int newton_max_n();
 // alternating-projection solver path (tk_dykstra.cu)
 cudaError_t launch_dykstra(const Problem& P, cudaStream_t stream);
 int dykstra_cluster_max_n();
@@ -56,20 +58,6 @@ inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
   }
   return P.n <= kMaxGroupN ? launch_group(P, stream) : launch_cta(P, stream);
 }
-}  // namespace tk
-
-namespace {
-
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
-
-// Long rows need the caller's scratch: present, 256-byte aligned and large enough.
-tk_status check_workspace(const tk_opts* opts, int64_t rows, int64_t n) {
-  if (rows > 65535) return TK_ERR_UNSUPPORTED;            // rows ride on gridDim.y there
-  if (!opts || !opts->workspace) return TK_ERR_WORKSPACE;
-  if (reinterpret_cast<uintptr_t>(opts->workspace) & 255u) return TK_ERR_WORKSPACE;
-  if (opts->workspace_bytes < tk::long_workspace_bytes(rows, (int)n)) return TK_ERR_WORKSPACE;
-  return TK_OK;
-}
 
 // q = p/(p-1): 2 and 4 (p = 2, p = 4/3) have closed-form block solves and run everywhere.  Any
 // other 1 < p <= 1.5 (q >= 3) is *qm1 = q - 1 > 0: forward pass by the sort-free solver, VJP from
@@ -92,10 +80,28 @@ tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, do
   if (mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
   if (!(lambda > 0.0) || !isfinite(lambda)) return TK_ERR_INVALID_ARG;
   tk_status s = classify_p(p, q4, qm1);
-  if (s == TK_OK && *qm1 > 0.0 && (mode == TK_TOPKMAG || n > tk::kMaxOnChipN)) s = TK_ERR_UNSUPPORTED;
+  if (s == TK_OK && *qm1 > 0.0 && (mode == TK_TOPKMAG || n > kMaxOnChipN)) s = TK_ERR_UNSUPPORTED;
   if (s != TK_OK) return s;
   if (rows > 0 && theta == nullptr) return TK_ERR_INVALID_ARG;
   if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
+  return TK_OK;
+}
+
+int max_key_only_n() { return kMaxKeyOnlyN; }
+}  // namespace tk
+
+namespace {
+
+using tk::check_common;
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Long rows need the caller's scratch: present, 256-byte aligned and large enough.
+tk_status check_workspace(const tk_opts* opts, int64_t rows, int64_t n) {
+  if (rows > 65535) return TK_ERR_UNSUPPORTED;            // rows ride on gridDim.y there
+  if (!opts || !opts->workspace) return TK_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(opts->workspace) & 255u) return TK_ERR_WORKSPACE;
+  if (opts->workspace_bytes < tk::long_workspace_bytes(rows, (int)n)) return TK_ERR_WORKSPACE;
   return TK_OK;
 }
 
@@ -122,7 +128,6 @@ const char* tk_status_string(int status) {
     case TK_ERR_UNSUPPORTED: return "unsupported configuration";
     case TK_ERR_WORKSPACE: return "workspace missing or too small";
     case TK_ERR_CUDA: return "CUDA runtime error";
-    case TK_ERR_NOT_CONVERGED: return "iteration cap reached";
     default: return "unknown status";
   }
 }
@@ -157,6 +162,14 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
   P.what = tk::W_FWD;
   if (opts) { P.perm_out = opts->perm_out; P.state_out = opts->state_out; P.status = opts->status_out; }
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
+  // phi(x) = x with a closed-form block solve, nothing but values asked for: the threshold form needs no
+  // order at all (TK_SOLVER_PAV keeps the sort)
+  const bool by_threshold = (solver == TK_SOLVER_AUTO || solver == TK_SOLVER_THRESHOLD) && mode != TK_TOPKMAG &&
+                            qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
+  if (by_threshold) {
+    cudaError_t en = tk::launch_newton(P, (cudaStream_t)stream);
+    return en == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+  }
   if (solver == TK_SOLVER_THRESHOLD) {
     // no sort, hence no permutation to return; rows held on chip only
     if (n > tk::kMaxOnChipN || (opts && opts->perm_out)) return TK_ERR_UNSUPPORTED;

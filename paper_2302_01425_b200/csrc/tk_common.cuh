@@ -40,6 +40,20 @@ struct Problem {
   int jvp;                  // tk_vjp_state kernels: the tangent goes through J instead of the cotangent through J^T
 };
 
+// ---------------------------------------------------------------- host helpers
+// Number of SMs of the current device, asked once per device (148, a B200, if the query fails).
+inline int sm_count() {
+  static int cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  if (cached[dev] == 0) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    cached[dev] = v;
+  }
+  return cached[dev];
+}
+
 // ---------------------------------------------------------------- keys
 // Order-preserving map float -> uint32 (larger float, larger integer).
 __device__ __forceinline__ uint32_t f2key(float x) {

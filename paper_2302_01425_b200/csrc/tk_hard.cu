@@ -30,7 +30,8 @@ cudaError_t launch_hard(const float* theta, const int32_t* perm, float* out, lon
                         int mode, cudaStream_t stream) {
   const long long total = rows * (long long)n;
   long long blocks = (total + 255) / 256;
-  if (blocks > 148LL * 64) blocks = 148LL * 64;      // grid-stride beyond a few waves
+  const long long cap = (long long)sm_count() * 64;  // grid-stride beyond a few waves
+  if (blocks > cap) blocks = cap;
   tk_hard_kernel<<<(unsigned)blocks, 256, 0, stream>>>(theta, perm, out, total, n, k, mode);
   return cudaGetLastError();
 }

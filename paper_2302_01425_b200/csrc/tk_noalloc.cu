@@ -9,18 +9,26 @@
 // points make such callers size and pass a workspace for rows longer than
 // 16384 elements; this one does not.
 //
-// How: the scratch is a file-scope __device__ array.  It is part of the loaded
-// module, so every GPU that loads the library carries TK_NOALLOC_SCRATCH_BYTES
-// of it until the process exits, whether or not this entry point is ever used.
-// In host code the array's name only stands for the symbol; its device address
-// is looked up with cudaGetSymbolAddress, once per device, on the first call
-// made with that device current.
+// How: the scratch is a file-scope __device__ array.  It belongs to the library's
+// module: a GPU carries TK_NOALLOC_SCRATCH_BYTES of it from the moment the CUDA
+// runtime loads that module on it (with lazy loading: this file's first lookup or
+// launch on that GPU) until the process exits or resets the device.  In host code
+// the array's name only stands for the symbol; its device address is looked up
+// with cudaGetSymbolAddress, once per device, on the first call made with that
+// device current -- which is therefore the call that can still fail for lack of
+// memory, and the one to make at start-up.
+#include <atomic>
+
 #include "tk_common.cuh"
 
 namespace tk {
 size_t long_workspace_bytes(long long rows, int n);
 cudaError_t launch_long(const Problem& P, void* workspace, tk_rowstate* state_dst, bool skip_map,
                         cudaStream_t stream);
+// the argument checks of the regular entry points, and the longest row they serve without scratch (tk_api.cu)
+tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, double p, double lambda,
+                       int mode, int* q4, double* qm1);
+int max_key_only_n();
 }  // namespace tk
 
 namespace {
@@ -29,7 +37,11 @@ constexpr size_t kScratchBytes = TK_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {};   // device address of g_scratch, per device ordinal
+// Device address of g_scratch, per device ordinal.  Host threads that make the first call on a
+// device at the same time each look the address up and store the same value: the atomic makes
+// that store and the later loads well defined.  The address is that of the module instance loaded
+// when it was looked up: after cudaDeviceReset it is stale and this entry point must not be used.
+std::atomic<void*> g_scratch_addr[kMaxDevices];
 
 // Device address of the scratch array on the current device (looked up once).
 cudaError_t scratch_address(void** out) {
@@ -37,13 +49,13 @@ cudaError_t scratch_address(void** out) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-  if (g_scratch_addr[dev] == nullptr) {
-    void* p = nullptr;
+  void* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (p == nullptr) {
     e = cudaGetSymbolAddress(&p, g_scratch);
     if (e != cudaSuccess) return e;
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return cudaSuccess;
 }
 
@@ -52,20 +64,16 @@ cudaError_t scratch_address(void** out) {
 extern "C" tk_status tk_fwd_noalloc(const float* theta, int64_t rows, int64_t n, int64_t k, double p,
                                     double lambda, int mode, float* out, tk_stream stream) {
   // shapes that need no scratch go through the regular entry point unchanged
-  if (n <= 16384) return tk_fwd(theta, rows, n, k, p, lambda, mode, out, stream);
-  // the same argument checks as tk_fwd_ex, before anything touches the device
-  if (rows < 0 || k < 1 || k > n) return TK_ERR_INVALID_ARG;
-  if (mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
-  if (!(lambda > 0.0) || !isfinite(lambda)) return TK_ERR_INVALID_ARG;
-  if (!(p > 1.0) || !isfinite(p)) return TK_ERR_INVALID_ARG;
-  const double q = p / (p - 1.0);
-  int q4;
-  if (fabs(q - 2.0) <= 1e-6) q4 = 0;
-  else if (fabs(q - 4.0) <= 1e-6) q4 = 1;
-  else return TK_ERR_UNSUPPORTED;
+  if (n <= tk::max_key_only_n()) return tk_fwd(theta, rows, n, k, p, lambda, mode, out, stream);
+  // the argument checks of tk_fwd_ex, before anything touches the device
+  int q4 = 0;
+  double qm1 = 0.0;
+  const tk_status cs = tk::check_common(theta, rows, n, k, p, lambda, mode, &q4, &qm1);
+  if (cs != TK_OK) return cs;
+  if (qm1 > 0.0) return TK_ERR_UNSUPPORTED;
   if (rows == 0) return TK_OK;
-  if (theta == nullptr || out == nullptr) return TK_ERR_INVALID_ARG;
-  if (rows > 65535 || n > 0x7fffffff) return TK_ERR_UNSUPPORTED;
+  if (out == nullptr) return TK_ERR_INVALID_ARG;
+  if (rows > 65535) return TK_ERR_UNSUPPORTED;
   // the built-in scratch has a fixed size: larger problems are refused, never truncated
   if ((double)rows * (double)n > (double)TK_NOALLOC_MAX_ELEMENTS) return TK_ERR_WORKSPACE;
   if (tk::long_workspace_bytes(rows, (int)n) > kScratchBytes) return TK_ERR_WORKSPACE;

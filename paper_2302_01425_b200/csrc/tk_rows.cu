@@ -598,14 +598,15 @@ cudaError_t launch_rows_gb(const Problem& P, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-constexpr long long kWarpsToFill = 148 * 24;   // warps below which a launch leaves SMs short of work
+// warps below which a launch leaves SMs short of work: 24 per SM
+inline long long warps_to_fill() { return (long long)sm_count() * 24; }
 
-// 8 keys per lane.  The most batches per warp that still leave kWarpsToFill warps, out of {1, 2, BMAX}.
+// 8 keys per lane.  The most batches per warp that still leave warps_to_fill() warps, out of {1, 2, BMAX}.
 template <int G, int BMAX>
 cudaError_t launch_rows_g(const Problem& P, cudaStream_t stream) {
   constexpr int RPB = 32 / G;
-  if (BMAX > 2 && P.rows / (RPB * BMAX) >= kWarpsToFill) return launch_rows_gb<G, 8, BMAX>(P, stream);
-  if (BMAX >= 2 && P.rows / (RPB * 2) >= kWarpsToFill) return launch_rows_gb<G, 8, (BMAX >= 2 ? 2 : 1)>(P, stream);
+  if (BMAX > 2 && P.rows / (RPB * BMAX) >= warps_to_fill()) return launch_rows_gb<G, 8, BMAX>(P, stream);
+  if (BMAX >= 2 && P.rows / (RPB * 2) >= warps_to_fill()) return launch_rows_gb<G, 8, (BMAX >= 2 ? 2 : 1)>(P, stream);
   return launch_rows_gb<G, 8, 1>(P, stream);
 }
 
@@ -620,13 +621,13 @@ cudaError_t launch_rows(const Problem& P0, cudaStream_t stream) {
   }
   if (P.n > 512) {                             // one warp per row, 32 keys per lane, up to 2 rows per warp
     P.N = 1024;
-    if (P.rows / 2 >= kWarpsToFill) return launch_rows_gb<32, 32, 2>(P, stream);
+    if (P.rows / 2 >= warps_to_fill()) return launch_rows_gb<32, 32, 2>(P, stream);
     return launch_rows_gb<32, 32, 1>(P, stream);
   }
   if (P.n > 256) {                             // one warp per row, 16 keys per lane, up to 4 rows per warp
     P.N = 512;
-    if (P.rows / 4 >= kWarpsToFill) return launch_rows_gb<32, 16, 4>(P, stream);
-    if (P.rows / 2 >= kWarpsToFill) return launch_rows_gb<32, 16, 2>(P, stream);
+    if (P.rows / 4 >= warps_to_fill()) return launch_rows_gb<32, 16, 4>(P, stream);
+    if (P.rows / 2 >= warps_to_fill()) return launch_rows_gb<32, 16, 2>(P, stream);
     return launch_rows_gb<32, 16, 1>(P, stream);
   }
   int G = 1;

@@ -13,7 +13,9 @@ __global__ void __launch_bounds__(256) tk_transpose_kernel(const float* __restri
                                                            long long in_cols, long long in_ld,
                                                            float* __restrict__ out, long long out_ld) {
   __shared__ float tile[32][33];
-  const long long c0 = (long long)blockIdx.x * 32, r0 = (long long)blockIdx.y * 32;
+  // tiles are numbered along a 1-D grid (either side of the matrix can exceed the 65535 blocks of gridDim.y)
+  const long long tiles_c = (in_cols + 31) / 32;
+  const long long c0 = ((long long)blockIdx.x % tiles_c) * 32, r0 = ((long long)blockIdx.x / tiles_c) * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;        // 32 x 8 threads
 #pragma unroll
   for (int j = 0; j < 32; j += 8) {
@@ -32,8 +34,9 @@ __global__ void __launch_bounds__(256) tk_transpose_kernel(const float* __restri
 
 cudaError_t launch_transpose(const float* in, long long in_rows, long long in_cols, long long in_ld, float* out,
                              long long out_ld, cudaStream_t stream) {
-  const dim3 grid((unsigned)((in_cols + 31) / 32), (unsigned)((in_rows + 31) / 32));
-  tk_transpose_kernel<<<grid, 256, 0, stream>>>(in, in_rows, in_cols, in_ld, out, out_ld);
+  const long long tiles = ((in_cols + 31) / 32) * ((in_rows + 31) / 32);
+  if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+  tk_transpose_kernel<<<(unsigned)tiles, 256, 0, stream>>>(in, in_rows, in_cols, in_ld, out, out_ld);
   return cudaGetLastError();
 }
 

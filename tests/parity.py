@@ -2,13 +2,17 @@
 
 Tolerances (written here once, used by every GPU test):
   * permutations: bit-exact;
-  * forward values: |gpu - ref| <= 1e-5 * max(1, |ref|);
+  * forward values: |gpu - ref| <= 1e-5 * max(1, |ref|).  Mask values lie in [0, 1], so for
+    them this is the absolute 1e-5 of the benchmark spec; topk and topkmag values grow with
+    theta (fp32 spacing exceeds 1e-5 above 128), hence the relative form there, with the raw
+    maximum printed whenever it is above 1e-5;
   * VJP: |gpu - ref| <= 1e-5 * max(1, |ref|) on rows where the fp32 path and
     the fp64 oracle found the same pooled block.  The VJP is discontinuous
     where an element enters or leaves the pooled block, so a row where the two
     disagree is accepted only when every disputed rank sits within
     1e-5 * max(1, |s_j|) of the block's edge in the oracle; such rows are
-    counted, reported and left out of the VJP maximum.
+    counted, reported, left out of the VJP maximum, and may not be more than
+    max(2, 1e-3 * rows) of a case.
 """
 from __future__ import annotations
 
@@ -23,6 +27,20 @@ TOL = 1e-5
 
 def rel_err(gpu: np.ndarray, ref: np.ndarray) -> np.ndarray:
     return np.abs(gpu.astype(np.float64) - ref) / np.maximum(1.0, np.abs(ref))
+
+
+def fwd_err(gpu: np.ndarray, ref: np.ndarray, mode: int) -> float:
+    """The gated forward error; for the mask (values in [0, 1]) it is the absolute error."""
+    if mode == tko.MASK:
+        assert np.abs(ref).max() <= 1.0 + 1e-9
+    return float(rel_err(gpu, ref).max())
+
+
+def check_disputed(count: int, rows: int, label: str):
+    cap = max(2, int(1e-3 * rows))
+    if count:
+        print(f"{label}: {count} of {rows} rows with a near-tie at the block edge (cap {cap})")
+    assert count <= cap, f"{label}: {count} disputed rows of {rows} (cap {cap})"
 
 
 def oracle_blocks(det, k):
@@ -96,10 +114,13 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         assert np.array_equal(perm.cpu().numpy(), det["perm"]), f"{label}: permutation differs"
     gout = out.cpu().numpy()
     assert np.isfinite(gout).all(), f"{label}: non-finite output"
-    res["fwd_max_rel"] = float(rel_err(gout, ref).max())
+    res["fwd_max_rel"] = fwd_err(gout, ref, mode)
     res["fwd_max_abs"] = float(np.abs(gout - ref).max())
+    if res["fwd_max_abs"] > TOL:
+        print(f"{label}: forward max-abs {res['fwd_max_abs']:.3g} on values above 1 (relative {res['fwd_max_rel']:.3g})")
     assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
     bad_noperm = np.zeros(0, np.int64)
+    bad_keysort = bad_noperm
     # the call without a permutation output takes its own path for short rows (keys sorted alone,
     # results placed by value): same tolerance against the oracle, same pooled blocks
     if sorts:
@@ -114,18 +135,39 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         assert int(status.item()) == 0
         g2 = out2.cpu().numpy()
         assert np.isfinite(g2).all(), f"{label}: non-finite output (no permutation)"
-        res["fwd_noperm_max_rel"] = float(rel_err(g2, ref).max())
+        res["fwd_noperm_max_rel"] = fwd_err(g2, ref, mode)
         assert res["fwd_noperm_max_rel"] <= TOL, f"{label}: forward error without permutation {res}"
         assert torch.equal(out2, out3), f"{label}: tk_fwd differs from tk_fwd_ex"
         st2 = read_state(state2, rows)
         ab2 = np.stack([st2["a"], st2["b"]], axis=1).astype(np.int64)
         bad_noperm = disputed_rows_ok(theta, k, p, lam, mode, det, ab2, oracle_blocks(det, k))
         res["rows_block_disputed_noperm"] = int(len(bad_noperm))
+        check_disputed(len(bad_noperm), rows, label + " (no permutation)")
+        # TK_SOLVER_PAV without a permutation: the keys are sorted alone and results placed by
+        # value (the default solver may skip the sort altogether); the recomputing VJP runs this
+        # solve, so its near-tie rows are the ones left out there
+        bad_keysort = bad_noperm
+        if solver == tk.TK_SOLVER_AUTO:
+            out4 = torch.full_like(out, float("nan"))
+            state4 = tk.new_state(rows)
+            tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out4, state_out=state4, status_out=status, workspace=ws,
+                         solver=tk.TK_SOLVER_PAV)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+            g4 = out4.cpu().numpy()
+            assert np.isfinite(g4).all(), f"{label}: non-finite output (keys sorted alone)"
+            res["fwd_keysort_max_rel"] = fwd_err(g4, ref, mode)
+            assert res["fwd_keysort_max_rel"] <= TOL, f"{label}: forward error with the keys sorted alone {res}"
+            st4 = read_state(state4, rows)
+            ab4 = np.stack([st4["a"], st4["b"]], axis=1).astype(np.int64)
+            bad_keysort = disputed_rows_ok(theta, k, p, lam, mode, det, ab4, oracle_blocks(det, k))
+            check_disputed(len(bad_keysort), rows, label + " (keys sorted alone)")
     st = read_state(state, rows)
     gpu_ab = np.stack([st["a"], st["b"]], axis=1).astype(np.int64)
     ref_ab = oracle_blocks(det, k)
     bad = disputed_rows_ok(theta, k, p, lam, mode, det, gpu_ab, ref_ab)
     res["rows_block_disputed"] = int(len(bad))
+    check_disputed(len(bad), rows, label)
     if g is not None:
         g = np.ascontiguousarray(g, np.float32)
         gt = torch.from_numpy(g).to(dev)
@@ -140,14 +182,26 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
         if mode == tko.TOPKMAG:
             kth = np.sort(np.abs(theta), axis=1)[:, ::-1][:, k - 1]
             free = (theta == 0.0) & (kth == 0.0)[:, None]
-        for name, kwargs in (("vjp_state", {"state": state}), ("vjp_recompute", {})):
+        # slope of a top singleton at key 0 (phi even): 1/(1+lambda) for p = 2; for p = 4/3
+        # rho'(0) = 0, so the slope rho'/(rho'+1) vanishes
+        zero_slope = 1.0 / (1.0 + lam) if abs(q - 2.0) < 1e-6 else 0.0
+        variants = [("vjp_state", {"state": state}), ("vjp_recompute", {})]
+        if sorts:
+            # the row state of the call without a permutation (its own kernels) feeds the VJP too
+            variants.insert(1, ("vjp_state_noperm", {"state": state2}))
+        for name, kwargs in variants:
             recomputes = sorts or (general and solver == tk.TK_SOLVER_AUTO and n <= 128)
             if name == "vjp_recompute" and (ws_bytes or not recomputes):
                 continue
             # rows left out: near-ties at a block edge in the solve this VJP rests on (the saved
             # state of the first call; its own solve, the one of the second call, when it recomputes)
             keep = np.ones(rows, bool)
-            keep[bad if (name == "vjp_state" or not sorts) else bad_noperm] = False
+            if name == "vjp_state" or not sorts:
+                keep[bad] = False
+            elif name == "vjp_state_noperm":
+                keep[bad_noperm] = False
+            else:
+                keep[bad_keysort] = False
             grad = torch.full((rows, n), float("nan"), device=dev)
             tk.tk_vjp(th, gt, rows, n, k, p, lam, mode, grad, workspace=ws, **kwargs)
             torch.cuda.synchronize()
@@ -156,8 +210,9 @@ def run_case(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: np.n
             e = rel_err(gg, gref)
             e[free] = 0.0
             if free.any():
-                slope = np.abs(gg[free]) / np.maximum(np.abs(g[free]), 1e-30)
-                assert np.all((gg[free] == 0.0) | (slope <= 1.0 + 1e-5)), f"{label}: {name} at tied zeros"
+                want = zero_slope * g[free].astype(np.float64)
+                near = np.abs(gg[free] - want) <= TOL * np.maximum(1.0, np.abs(want))
+                assert np.all((gg[free] == 0.0) | near), f"{label}: {name} at tied zeros"
             res[name + "_max_rel"] = float(e[keep].max()) if keep.any() else 0.0
             res[name + "_max_abs"] = float((np.abs(gg - gref) * ~free)[keep].max()) if keep.any() else 0.0
             assert res[name + "_max_rel"] <= TOL, f"{label}: {name} error {res}"
@@ -189,7 +244,7 @@ def run_sampled(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: n
     idx = torch.from_numpy(sample).to(dev)
     sub = theta[sample]
     ref, det = tko.fwd(sub, k, p, lam, mode, details=True)
-    res = {"fwd_max_rel": float(rel_err(out[idx].cpu().numpy(), ref).max())}
+    res = {"fwd_max_rel": fwd_err(out[idx].cpu().numpy(), ref, mode)}
     assert res["fwd_max_rel"] <= TOL, f"{label}: forward error {res}"
     st = read_state(state, rows)[sample]
     gpu_ab = np.stack([st["a"], st["b"]], axis=1).astype(np.int64)
@@ -200,5 +255,6 @@ def run_sampled(theta: np.ndarray, k: int, p: float, lam: float, mode: int, g: n
     e = rel_err(grad[idx].cpu().numpy(), gref)
     res["vjp_max_rel"] = float(e[keep].max()) if keep.any() else 0.0
     res["rows_block_disputed"] = int(len(bad))
+    check_disputed(len(bad), len(sample), label)
     assert res["vjp_max_rel"] <= TOL, f"{label}: VJP error {res}"
     return res

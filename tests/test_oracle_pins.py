@@ -474,6 +474,60 @@ def test_dykstra_hundred_sweeps_small_block():
     assert np.max(np.abs(out - exact)) < 1e-6
 
 
+def test_dykstra_iterates_after_one_and_two_sweeps_by_hand():
+    """Algorithm 1 at a finite sweep count, worked by hand (fractions, no oracle value involved).
+
+    phi(x) = x, k = 1, lambda = 4, s = (4, 3, 2): z = s - lambda w = (0, 3, 2), p = q = 0.
+      sweep 1, C1 (pair 1,2): (0, 3) -> 3/2 each, p = (-3/2, 3/2, 0);
+               C2 (pair 2,3): (3/2, 2) -> 7/4 each, q = (0, -1/4, 1/4);      v = (3/2, 7/4, 7/4)
+      sweep 2, C1: v + p = (0, 13/4, 7/4) -> (13/8, 13/8, 7/4), p = (-13/8, 13/8, 0);
+               C2: y + q = (13/8, 11/8, 2) -> (13/8, 27/16, 27/16);          v = (13/8, 27/16, 27/16)
+    (C2 before C1, or a correction dropped on the pair that does not violate, gives other numbers;
+    the limit is the mean 5/3.)  Output y = (s - v)/lambda.
+    phi(x) = x^2/2, k = 1, lambda = 1, s = (4, 3, 5/2): metric c = (2, 1, 1), z = s/c = (2, 3, 5/2).
+      sweep 1, C1: (2, 3) -> (2*2 + 3)/3 = 7/3, p = (-1/3, 2/3, 0);
+               C2: (7/3, 5/2) -> 29/12, q = (0, -1/12, 1/12);                v = (7/3, 29/12, 29/12)
+      sweep 2, C1: v + p = (2, 37/12, 29/12) -> 85/36, p = (-13/36, 26/36, 0);
+               C2: y + q = (85/36, 82/36, 90/36) -> 43/18;                   v = (85/36, 43/18, 43/18)
+    """
+    from fractions import Fraction as Fr
+    theta = np.array([[3.0, 2.0, 4.0]], np.float32)            # unsorted on purpose: s = (4, 3, 2)
+    expect_v = {0: [Fr(0), Fr(3), Fr(2)], 1: [Fr(3, 2), Fr(7, 4), Fr(7, 4)], 2: [Fr(13, 8), Fr(27, 16), Fr(27, 16)]}
+    s = [Fr(4), Fr(3), Fr(2)]
+    for sweeps, ev in expect_v.items():
+        out, v = tko.dykstra(theta, 1, 2.0, 4.0, tko.MASK, sweeps=sweeps, return_v=True)
+        assert np.max(np.abs(v[0] - np.array([float(a) for a in ev]))) < 1e-14
+        y_sorted = [float((si - vi) / 4) for si, vi in zip(s, ev)]
+        assert np.max(np.abs(out[0] - np.array([y_sorted[1], y_sorted[2], y_sorted[0]]))) < 1e-14
+    theta = np.array([[-3.0, 2.5, 4.0]], np.float32)           # |theta| sorted: (4, 3, 5/2), signs (+, -, +)
+    expect_v = {1: [Fr(7, 3), Fr(29, 12), Fr(29, 12)], 2: [Fr(85, 36), Fr(43, 18), Fr(43, 18)]}
+    s = [Fr(4), Fr(3), Fr(5, 2)]
+    for sweeps, ev in expect_v.items():
+        out, v = tko.dykstra(theta, 1, 2.0, 1.0, tko.TOPKMAG, sweeps=sweeps, return_v=True)
+        assert np.max(np.abs(v[0] - np.array([float(a) for a in ev]))) < 1e-14
+        y_sorted = [float(si - vi) for si, vi in zip(s, ev)]    # rho(t) = t / lambda, lambda = 1
+        assert np.max(np.abs(out[0] - np.array([-y_sorted[1], y_sorted[2], y_sorted[0]]))) < 1e-14
+
+
+def test_dual_coordinate_ascent_first_updates_by_hand():
+    """App. A.8 for p = 4/3 (rho(t) = (t/lambda)^3), phi(x) = x, k = 1, lambda = 1, three equal keys s.
+
+    Sweep 1, odd coordinate alpha_1 (pair 1,2; alpha_0 = alpha_2 = 0): separate minimisers s - 1 < s,
+    so both take the common gamma with 2 (s - gamma)^3 = 1, and alpha_1 = 1 - (s - gamma)^3 = 1/2.
+    Even coordinate alpha_2 (pair 2,3; alpha_1 = 1/2, alpha_3 = 0): s - cbrt(1/2) < s, common gamma
+    with 2 (s - gamma)^3 = 1/2, alpha_2 = 1/2 - 1/4 = 1/4.  Primal iterate v_i = s - cbrt(w_i + alpha_{i-1}
+    - alpha_i): outputs y = (1/2, 1/4, 1/4).
+    Sweep 2: alpha_1 solves 2 a^3 = 1 - 1/4 -> alpha_1 = 1 - 3/8 = 5/8; alpha_2 solves 2 a^3 = 5/8 ->
+    alpha_2 = 5/8 - 5/16 = 5/16: y = (3/8, 5/16, 5/16).  (Even before odd would give (1/2, 1/2, 0) after
+    the first sweep; the limit is (1/3, 1/3, 1/3).)
+    """
+    theta = np.full((1, 3), 0.625, np.float32)
+    for sweeps, y in ((1, [0.5, 0.25, 0.25]), (2, [0.375, 0.3125, 0.3125])):
+        out, v = tko.dykstra(theta, 1, P43, 1.0, tko.MASK, sweeps=sweeps, return_v=True)
+        assert np.max(np.abs(out[0] - np.array(y))) < 1e-13
+        assert np.max(np.abs(v[0] - (0.625 - np.cbrt(np.array(y))))) < 1e-13
+
+
 # --------------------------------------------------------------------------
 # VJP
 # --------------------------------------------------------------------------
