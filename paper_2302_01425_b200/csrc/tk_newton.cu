@@ -1,5 +1,5 @@
 // tk_newton.cu -- the exact forward pass without a sort, for phi(x) = x (TK_MASK, TK_TOPK),
-// p = 2 and p = 4/3, rows of up to 4096 elements held in registers.
+// p = 2 and p = 4/3, rows of up to 32768 elements held in registers.
 //
 // With w = 1_k the relaxed mask is the maximiser of <y, x> - R(y) over the capped simplex
 // P(1_k) = {y in [0,1]^n, sum y = k} (Sec. 3), so y_i = clip(rho(x_i - tau), 0, 1) with tau the
@@ -26,10 +26,13 @@
 // cancellation; the row state stores exactly the pair the last pass classified with, and its
 // counts, so the VJP from state sees the same classes.
 //
-// Layout: G lanes of a warp per row (32/G rows per warp), E keys per lane.  The warp's rows are
-// contiguous in memory: they are staged through a shared-memory tile with coalesced 128-bit
-// accesses, every lane reads its own span from the tile (chunk order rotated per lane: no bank
-// conflicts), results go back through the tile the same way.
+// Layout: a row is held by G lanes of a warp (32/G rows per warp) or, above 2048 elements, by W whole
+// warps, 64 keys per lane (fewer for rows of up to 32); the only exchange between the lanes of a
+// row is the sum of the pass's counts and power sums (shuffles, plus one shared-memory slot per
+// warp and a named barrier when W > 1).  Rows are read and written with coalesced 128-bit
+// accesses straight from the registers; with one or two lanes per row through a shared-memory
+// tile instead.
+#include <float.h>
 #include <math.h>
 
 #include "tk_common.cuh"
@@ -84,21 +87,24 @@ __device__ __forceinline__ void nt_top3(float x, float& m1, float& m2, float& m3
 }
 
 // Root of g(u) = sum_i (t_i - u)^3 - rhs (rhs >= 0) over the cm inside keys, from their power sums.
-// g is decreasing; by Jensen g(mu - cbrt(rhs / cm)) >= 0 with mu the mean of the t_i, so that point is
-// left of the root, where g is convex: Newton from it increases monotonically to the root.  The
-// anchor of the sums is the current iterate, so u -> 0 as the outer iteration converges and fp32
-// is enough.  c0 = g(0).
+// g is decreasing.  The anchor of the sums is the current iterate, so once the outer iteration is
+// close the root is near 0 and Newton from 0 takes two steps; fp32 is enough there (u -> 0).  When
+// the first step is not small against the spread of the t_i, the start is mu - cbrt(rhs / cm)
+// instead, mu the mean of the t_i: by Jensen g >= 0 there, i.e. it is left of the root, where g is
+// convex and Newton increases monotonically to the root.  c0 = g(0).
 __device__ __forceinline__ float nt_cubic(int cm, float s1, float s2, float s3, float rhs, float c0) {
   const float fcm = (float)cm;
-  const float mu = s1 / fcm;
-  float u = mu - cbrtf(rhs / fcm);
-  const float spread = sqrtf(s2 / fcm);
+  const float inv_cm = __fdividef(1.0f, fcm);
+  const float spread2 = s2 * inv_cm;                       // mean of t^2
+  float u = __fdividef(c0, 3.0f * s2);                     // Newton step from 0
+  if (u * u > 0.01f * spread2) u = s1 * inv_cm - cbrtf(rhs * inv_cm);
+  const float spread = sqrtf(spread2);
 #pragma unroll 1
   for (int it = 0; it < 8; ++it) {
     const float g = ((-fcm * u + 3.0f * s1) * u - 3.0f * s2) * u + c0;
     const float gp = -3.0f * ((fcm * u - 2.0f * s1) * u + s2);
     if (!(gp < 0.0f)) break;
-    const float st = -g / gp;
+    const float st = -__fdividef(g, gp);
     u += st;
     if (fabsf(st) <= 1e-7f * (fabsf(u) + spread)) break;
   }
@@ -135,12 +141,12 @@ __device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, floa
     float c0;
     if (!Q4) {
       c0 = s1 - lam * (float)m;
-      du = c0 / (float)cm;
+      du = __fdividef(c0, (float)cm);
     } else {
       const float rhs = lam3 * (float)m;
       c0 = s3 - rhs;
       du = nt_cubic(cm, s1, s2, s3, rhs, c0);
-      if ((du > 0.0f) != (c0 > 0.0f)) du = c0 / (3.0f * s2);
+      if ((du > 0.0f) != (c0 > 0.0f)) du = __fdividef(c0, 3.0f * s2);
     }
     fpos = c0 > 0.0f;
     const float adu = fabsf(du);
@@ -213,27 +219,155 @@ __device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, floa
   S.off = nxt;
 }
 
-// G lanes per row, E keys per lane (E / 4 a power of two).  KSEL: 0 = moment start, 1 / 2 = k is 1 / 2.
-template <int G, int E, bool Q4, int KSEL>
-__global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))) tk_newton_kernel(const Problem P, const float zq) {
+// threads per block, and the blocks per SM the register budget is set for: 24 warps of 80 registers with
+// up to 32 keys per lane, 16 warps of 128 registers with 64
+constexpr int nt_threads(int W) { return W * 32 > kNtThreads ? W * 32 : kNtThreads; }
+constexpr int nt_min_blocks(int E, int W) {
+  const int warps = E >= 128 ? 8 : (E >= 64 ? 16 : 24);
+  const int b = warps * 32 / nt_threads(W);
+  return b < 1 ? 1 : b;
+}
+
+// ---------------------------------------------------------------- row access
+// A row is spread over a team of T = G * W lanes (G lanes of one warp, or W whole warps), E keys per
+// lane in E / 4 chunks of four.  DIRECT: chunk c of team lane tl is float4 number c * T + tl of the
+// row, read from and written to global memory with coalesced 128-bit accesses (T * 16 contiguous
+// bytes per row and instruction).  STAGED (one or two lanes per row, where that would be 16 or 32
+// bytes): the warp's rows, contiguous in memory, go through a shared-memory tile with coalesced
+// accesses, and every lane owns a contiguous span of the tile (chunk order rotated per lane: no
+// bank conflicts).
+template <int G, int E, int W, bool STAGED>
+struct NtIO {
+  static constexpr int CH = E / 4;
+  static constexpr int T = G * W;
+  const float* src;      // DIRECT: the row in global memory
+  float* dst;
+  float4* span4;         // STAGED: this lane's span of the tile
+  int n, tl, rot, vec4;
+  bool row_ok;
+
+  // index in the row of the first key of chunk c
+  __device__ __forceinline__ int pos(int c) const {
+    return STAGED ? tl * E + 4 * ((c + rot) & (CH - 1)) : 4 * (c * T + tl);
+  }
+  // the four words of chunk c as they are in memory (a chunk past the row re-reads the row's start:
+  // no load depends on a test, so the loads of a lane are all in flight at once)
+  __device__ __forceinline__ void load_raw(int c, float (&x)[4]) const {
+    const int p0 = pos(c);
+    if (STAGED) {
+      const float4 v = span4[(c + rot) & (CH - 1)];
+      x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else if (vec4) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(src + (p0 < n ? p0 : 0)));
+      x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) x[j] = __ldg(src + (p0 + j < n ? p0 + j : 0));
+    }
+  }
+  // slots past the end of the row become -infinity, which never takes part.
+  // ninf (may be null): set when a key of the row is itself -infinity
+  __device__ __forceinline__ void mask(int c, float (&x)[4], bool* ninf = nullptr) const {
+    const int p0 = pos(c);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const bool in = p0 + j < n;
+      if (ninf && in && x[j] == -INFINITY) *ninf = true;
+      if (!in) x[j] = -INFINITY;
+    }
+  }
+  __device__ __forceinline__ void load(int c, float (&x)[4]) const {
+    load_raw(c, x);
+    mask(c, x);
+  }
+  __device__ __forceinline__ void store(int c, const float (&y)[4]) const {
+    const int p0 = pos(c);
+    if (STAGED) {
+      span4[(c + rot) & (CH - 1)] = make_float4(y[0], y[1], y[2], y[3]);
+    } else if (vec4) {
+      if (row_ok && p0 < n) *reinterpret_cast<float4*>(dst + p0) = make_float4(y[0], y[1], y[2], y[3]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (row_ok && p0 + j < n) dst[p0 + j] = y[j];
+    }
+  }
+};
+
+// Keeps the loads of later chunks behind this point: the second passes over a row (new pivot, top-k
+// values, smallest capped key) run while the row's registers are live, and E more words in flight would spill.
+__device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
+
+// Sum of NV values over the lanes of a row: shuffles inside the warp, then (W > 1) one slot per warp in
+// shared memory and a named barrier over the team's W warps.  red: the team's W * 4 words for this
+// phase (the caller alternates two such buffers, so one barrier per sum is enough).  Every warp adds the
+// slots in the same order: all lanes of the team hold identical results.
+template <int G, int W, int NV>
+__device__ __forceinline__ void nt_allsum(float (&v)[NV], uint32_t& packed, float* red, int wit, int lane, int bar) {
+#pragma unroll
+  for (int i = 0; i < NV; ++i) v[i] = nt_gsum<G>(v[i]);
+  packed = (uint32_t)nt_gsum<G>((int)packed);
+  if (W > 1) {
+    if (lane == 0) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) red[wit * 4 + i] = v[i];
+      red[wit * 4 + 3] = __uint_as_float(packed);
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(W * 32) : "memory");
+#pragma unroll
+    for (int i = 0; i < NV; ++i) v[i] = 0.0f;
+    packed = 0;
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+#pragma unroll
+      for (int i = 0; i < NV; ++i) v[i] += red[w * 4 + i];
+      packed += __float_as_uint(red[w * 4 + 3]);
+    }
+  }
+}
+
+// G lanes per row (W == 1) or W warps per row (G == 32), E keys per lane (E / 4 a power of two).
+// KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1 only).
+template <int G, int E, int W, bool Q4, int KSEL, bool STAGED>
+__global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_kernel(const Problem P, const float zq) {
   extern __shared__ float4 nt_smem4[];
-  constexpr int R = 32 / G;                    // rows per warp
-  constexpr int RS = G * E;                    // row stride in the tile
+  static_assert(W == 1 || G == 32, "several warps per row: every lane of them belongs to the row");
+  static_assert(!STAGED || W == 1, "the staging tile belongs to one warp");
+  constexpr int BW = kNtWarps > W ? kNtWarps : W;   // warps per block
+  constexpr int TEAMS = BW / W;                      // teams (of W warps) per block
+  constexpr int R = W > 1 ? 1 : 32 / G;              // rows per team
   constexpr int CH = E / 4;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float* tile = reinterpret_cast<float*>(nt_smem4) + warp * (32 * E);
-  const long long row0 = ((long long)blockIdx.x * kNtWarps + warp) * R;
-  if (row0 >= P.rows) return;                  // the whole warp
+  const int team = warp / W, wit = warp % W;
+  const long long row0 = ((long long)blockIdx.x * TEAMS + team) * R;
+  if (row0 >= P.rows) return;                  // the whole team
   const int n = P.n, k = P.k;
   const int rl = lane / G, lig = lane % G;
   const long long row = row0 + rl;
   const bool row_ok = row < P.rows;
-  const int rows_here = (int)(P.rows - row0 < (long long)R ? P.rows - row0 : (long long)R);
   const float lam = P.lam, inv_lam = P.inv_lam, lam3 = P.lam3, wid = P.lam;
   const float tol = (Q4 ? 3e-7f : 1e-6f) * wid;
+  float* smem = reinterpret_cast<float*>(nt_smem4);
+  // shared memory: [STAGED: one tile of 32 E floats per warp] [W > 1: two buffers of W * 4 words per team]
+  float* red = smem + (STAGED ? BW * 32 * E : 0) + team * (2 * W * 4);
+  const int bar = 1 + team;
+  int phase = 0;                               // which of the two buffers the next team sum uses
 
-  // ---- stage the warp's rows in the tile
-  {
+  NtIO<G, E, W, STAGED> io;
+  io.n = n; io.vec4 = P.vec4; io.row_ok = row_ok;
+  io.tl = W > 1 ? wit * 32 + lane : lig;
+  io.rot = nt_rot<E>(lane);
+  // a group past the last row works on the last row again and stores nothing
+  const long long row_c = row_ok ? row : P.rows - 1;
+  io.src = P.theta + row_c * (long long)n;
+  io.dst = P.out + row_c * (long long)n;
+  io.span4 = nullptr;
+  if (STAGED) {
+    // ---- stage the warp's rows (contiguous in memory) in its tile, row stride G * E
+    constexpr int RS = G * E;
+    float* tile = smem + warp * (32 * E);
+    io.span4 = reinterpret_cast<float4*>(tile + lane * E);
+    const int rows_here = (int)(P.rows - row0 < (long long)R ? P.rows - row0 : (long long)R);
     const float* src = P.theta + row0 * (long long)n;
     if (n == RS) {
       const int total = rows_here * n;
@@ -255,63 +389,66 @@ __global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))
         }
       }
     }
+    // lanes whose row lies past the last one solve a row of zeros and store nothing
+    for (int i = rows_here * RS + lane; i < R * RS; i += 32) tile[i] = 0.0f;
+    __syncwarp();
   }
-  __syncwarp();
 
-  const int rot = nt_rot<E>(lane);
-  float4* span4 = reinterpret_cast<float4*>(tile + lane * E);   // this lane's E keys of its row
-  const int span_n = n - lig * E;              // keys of the span that exist (may be <= 0 or >= E)
   float d[E];
-  float fin = 0.0f;                            // becomes NaN when the row holds a NaN or an infinity
-  {
-    const bool full = row_ok && n == RS;       // every slot of the span is a key of the row
+  bool bad = false;                            // a NaN or an infinity among this lane's keys
 #pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const int cc = (c + rot) & (CH - 1);
-      const float4 v = span4[cc];
-      const float x4[4] = {v.x, v.y, v.z, v.w};
+  for (int c = 0; c < CH; ++c) {
+    float x4[4];
+    io.load_raw(c, x4);
+    d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
+  }
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const bool in = full || (row_ok && 4 * cc + j < span_n);
-        d[4 * c + j] = in ? x4[j] : -INFINITY;  // slots past the end of the row never take part
-        fin = fmaf(in ? x4[j] : 0.0f, 0.0f, fin);
-      }
-    }
+  for (int c = 0; c < CH; ++c) {
+    float x4[4] = {d[4 * c], d[4 * c + 1], d[4 * c + 2], d[4 * c + 3]};
+    io.mask(c, x4, &bad);
+    d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
   }
 
   // ---- start: bracket and first tau
   NtRow S;
-  S.done = !row_ok; S.noblock = false; S.repiv = false;
+  S.done = false; S.noblock = false; S.repiv = false;
   S.a0 = k; S.b0 = k; S.gallop = 0; S.nnewt = 0; S.prev_ct = -1; S.prev_cm = -1; S.edge_tried = false;
-  S.off = 0.0f;
-  float lo, hi;
+  S.off = 0.0f; S.piv = 0.0f;
+  float lo = -FLT_MAX, hi = FLT_MAX;
   if (KSEL == 0) {
-    const float x0 = tile[rl * RS];            // sums are taken about the row's first key
-    float sm = 0.f, ss = 0.f, mx = -INFINITY, mn = INFINITY;
+    // sums about the row's first key: mean and spread of the keys
+    const float x0 = __ldg(io.src);
+    float v[2] = {0.f, 0.f};
 #pragma unroll
     for (int i = 0; i < E; ++i) {
-      const bool in = !(d[i] == -INFINITY);
-      const float dd = in ? d[i] - x0 : 0.0f;
-      sm += dd; ss = fmaf(dd, dd, ss);
-      mx = fmaxf(mx, d[i]);
-      mn = fminf(mn, in ? d[i] : INFINITY);
+      const float dd = (d[i] == -INFINITY) ? 0.0f : d[i] - x0;
+      v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
     }
-    sm = nt_gsum<G>(sm); ss = nt_gsum<G>(ss); mx = nt_gmax<G>(mx); mn = nt_gmin<G>(mn);
+    uint32_t none = 0;
+    nt_allsum<G, W, 2>(v, none, red + (phase & 1) * (W * 4), wit, lane, bar);
+    ++phase;
+    if (!(v[1] < INFINITY)) {                  // overflow, an infinity or a NaN: look at the keys themselves
+#pragma unroll
+      for (int i = 0; i < E; ++i) bad |= !(fabsf(d[i]) < INFINITY) && d[i] != -INFINITY;
+    }
     const float inv_n = 1.0f / (float)n;
-    const float mean_d = sm * inv_n;
-    const float sd = sqrtf(fmaxf(ss * inv_n - mean_d * mean_d, 0.0f));
-    lo = mn - wid; hi = mx;
+    const float mean_d = v[0] * inv_n;
+    const float sd = sqrtf(fmaxf(v[1] * inv_n - mean_d * mean_d, 0.0f));
     if (k == n) {                              // everything is selected
-      S.piv = mn; S.off = -wid; S.done = true; S.noblock = true;
+      S.piv = -FLT_MAX; S.off = -wid; S.done = true; S.noblock = true;
     } else {
       float tau0 = (x0 + mean_d) + zq * sd - (Q4 ? 0.75f : 0.5f) * lam;
-      if (!(tau0 > lo && tau0 < hi)) tau0 = 0.5f * (lo + hi);
+      if (!(fabsf(tau0) < FLT_MAX)) tau0 = x0;
       S.piv = tau0;
     }
   } else {
-    float m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY;
+    float m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY, fin = 0.0f;
 #pragma unroll
-    for (int i = 0; i < E; ++i) nt_top3(d[i], m1, m2, m3);
+    for (int i = 0; i < E; ++i) {
+      nt_top3(d[i], m1, m2, m3);
+      fin = fmaf(d[i] == -INFINITY ? 0.0f : d[i], 0.0f, fin);
+    }
+    bad |= fin != fin;
 #pragma unroll
     for (int o = G >> 1; o > 0; o >>= 1) {
       const float p1 = __shfl_xor_sync(0xffffffffu, m1, o), p2 = __shfl_xor_sync(0xffffffffu, m2, o),
@@ -326,11 +463,10 @@ __global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))
       S.piv = 0.5f * (lo + hi);
     }
   }
-  fin = nt_gsum<G>(fin);
-  const bool bad = row_ok && fin != fin;
-  if (!row_ok) { S.piv = 0.0f; lo = 0.0f; hi = 0.0f; }
   const bool early = S.done && S.noblock;      // pivot already exact
-  S.lo_a = lo; S.hi_a = hi; S.lo_o = lo - S.piv; S.hi_o = hi - S.piv;
+  S.lo_a = lo; S.hi_a = hi;
+  S.lo_o = KSEL == 0 ? -INFINITY : lo - S.piv;
+  S.hi_o = KSEL == 0 ? INFINITY : hi - S.piv;
 #pragma unroll
   for (int i = 0; i < E; ++i) d[i] -= S.piv;
 
@@ -361,22 +497,23 @@ __global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))
         if (Q4) { const float t2 = tm * tm; b1 += t2; e1 = fmaf(t2, tm, e1); }
       }
     }
-    const int packed = nt_gsum<G>((ct0 + ct1) | ((cm0 + cm1) << 16));
-    const float s1 = nt_gsum<G>(a0 + a1);
-    float s2 = 0.f, s3 = 0.f;
-    if (Q4) { s2 = nt_gsum<G>(b0 + b1); s3 = nt_gsum<G>(e0 + e1); }
+    float v[Q4 ? 3 : 1];
+    v[0] = a0 + a1;
+    if (Q4) { v[1] = b0 + b1; v[2] = e0 + e1; }
+    uint32_t packed = (uint32_t)(ct0 + ct1) | ((uint32_t)(cm0 + cm1) << 16);
+    nt_allsum<G, W, Q4 ? 3 : 1>(v, packed, red + (phase & 1) * (W * 4), wit, lane, bar);
+    ++phase;
     if (!S.done) {
-      nt_step<Q4>(S, packed & 0xffff, packed >> 16, s1, s2, s3, k, lam, lam3, tol);
+      nt_step<Q4>(S, (int)(packed & 0xffffu), (int)(packed >> 16), v[0], Q4 ? v[1] : 0.0f, Q4 ? v[Q4 ? 2 : 0] : 0.0f,
+                  k, lam, lam3, tol);
       if (S.repiv) {
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
-          const int cc = (c + rot) & (CH - 1);
-          const float4 v = span4[cc];
-          // slots past the row stay at -infinity
-          d[4 * c] = (d[4 * c] > -INFINITY) ? v.x - S.piv : d[4 * c];
-          d[4 * c + 1] = (d[4 * c + 1] > -INFINITY) ? v.y - S.piv : d[4 * c + 1];
-          d[4 * c + 2] = (d[4 * c + 2] > -INFINITY) ? v.z - S.piv : d[4 * c + 2];
-          d[4 * c + 3] = (d[4 * c + 3] > -INFINITY) ? v.w - S.piv : d[4 * c + 3];
+          float x4[4];
+          io.load(c, x4);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) d[4 * c + j] = x4[j] - S.piv;
+          if ((c & 3) == 3) nt_fence();
         }
       }
     }
@@ -397,51 +534,65 @@ __global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))
     const bool want_p = row_ok && !block && !early;
     const bool safe = wid > 9.6e-7f * (fabsf(S.piv) + fabsf(S.off));
     const bool scan = want_p && !safe;
-    if (__any_sync(0xffffffffu, scan)) {
+    if (__any_sync(0xffffffffu, scan)) {       // uniform over the warps of a row: they hold the same S
       float cmin = INFINITY;
 #pragma unroll
       for (int c = 0; c < CH; ++c) {
-        const int cc = (c + rot) & (CH - 1);
-        const float4 v = span4[cc];
-        if (d[4 * c] - S.off >= wid) cmin = fminf(cmin, v.x);
-        if (d[4 * c + 1] - S.off >= wid) cmin = fminf(cmin, v.y);
-        if (d[4 * c + 2] - S.off >= wid) cmin = fminf(cmin, v.z);
-        if (d[4 * c + 3] - S.off >= wid) cmin = fminf(cmin, v.w);
+        float x4[4];
+        io.load(c, x4);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+          if (d[4 * c + j] - S.off >= wid) cmin = fminf(cmin, x4[j]);
+        if ((c & 3) == 3) nt_fence();
       }
       cmin = nt_gmin<G>(cmin);
+      if (W > 1) {
+        float* rb = red + (phase & 1) * (W * 4);
+        ++phase;
+        if (lane == 0) rb[wit * 4] = cmin;
+        asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(W * 32) : "memory");
+        cmin = rb[0];
+#pragma unroll
+        for (int w = 1; w < W; ++w) cmin = fminf(cmin, rb[w * 4]);
+      }
       if (scan) piv_state = cmin;
     }
     if (want_p && safe) piv_state = (S.piv + S.off) + 0.5f * wid;
     if (!block) off_state = 0.0f;
   }
-  if (P.state_out && row_ok && lig == 0) {
+  if (P.state_out && row_ok && lig == 0 && wit == 0) {
     tk_rowstate st;
     st.pivot = piv_state; st.offset = off_state; st.a = S.a0; st.b = S.b0;
     P.state_out[row] = st;
   }
 
-  // ---- dual map, back through the tile
+  // ---- dual map y = rho(clamp(x - tau)), in the order the keys were read
   {
-    const float off = S.off;
+    const float shift = -S.off * inv_lam;
     const bool times_x = P.mode == TK_TOPK;
 #pragma unroll
     for (int c = 0; c < CH; ++c) {
-      const int cc = (c + rot) & (CH - 1);
       float y[4];
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        const float a = __saturatef((d[4 * c + j] - off) * inv_lam);
+        const float a = __saturatef(fmaf(d[4 * c + j], inv_lam, shift));
         y[j] = Q4 ? a * a * a : a;
       }
       if (times_x) {
-        const float4 v = span4[cc];
-        y[0] *= v.x; y[1] *= v.y; y[2] *= v.z; y[3] *= v.w;
+        float x4[4];
+        io.load(c, x4);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) y[j] = (x4[j] == -INFINITY) ? 0.0f : y[j] * x4[j];
       }
-      span4[cc] = make_float4(y[0], y[1], y[2], y[3]);
+      io.store(c, y);
+      if (times_x && (c & 3) == 3) nt_fence();
     }
   }
-  __syncwarp();
-  {
+  if (STAGED) {
+    constexpr int RS = G * E;
+    __syncwarp();
+    const float* tile = smem + warp * (32 * E);
+    const int rows_here = (int)(P.rows - row0 < (long long)R ? P.rows - row0 : (long long)R);
     float* dst = P.out + row0 * (long long)n;
     if (n == RS) {
       const int total = rows_here * n;
@@ -466,7 +617,7 @@ __global__ void __launch_bounds__(kNtThreads, (E >= 128 ? 2 : (E >= 32 ? 4 : 6))
   }
   if (P.status) {
     if (bad) flags |= TK_FLAG_NONFINITE;
-    if (flags && lig == 0) atomicOr(P.status, flags);
+    if (flags) atomicOr(P.status, flags);
   }
 }
 
@@ -480,10 +631,12 @@ float upper_normal_quantile(double tail) {
   return (float)(0.5 * (lo + hi));
 }
 
-template <int G, int E, bool Q4, int KSEL>
+template <int G, int E, int W, bool Q4, int KSEL, bool STAGED>
 cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
-  constexpr int smem = kNtWarps * 32 * E * (int)sizeof(float);
-  auto kern = tk_newton_kernel<G, E, Q4, KSEL>;
+  constexpr int BW = kNtWarps > W ? kNtWarps : W;
+  constexpr int TEAMS = BW / W;
+  constexpr int smem = (STAGED ? BW * 32 * E * (int)sizeof(float) : 0) + (W > 1 ? TEAMS * 2 * W * 4 * (int)sizeof(float) : 0);
+  auto kern = tk_newton_kernel<G, E, W, Q4, KSEL, STAGED>;
   if (smem > 48 * 1024) {
     static bool configured[64];
     int dev = 0;
@@ -495,39 +648,49 @@ cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
       if (dev >= 0 && dev < 64) configured[dev] = true;
     }
   }
-  constexpr long long rows_per_block = (long long)kNtWarps * (32 / G);
+  constexpr long long rows_per_block = (long long)TEAMS * (W > 1 ? 1 : 32 / G);
   const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
-  kern<<<blocks, kNtThreads, smem, stream>>>(P, zq);
+  kern<<<blocks, BW * 32, smem, stream>>>(P, zq);
   return cudaGetLastError();
 }
 
-template <int G, int E, bool KS>
+// KS: the shape also has the variants that track the k + 1 largest keys (k <= 2)
+template <int G, int E, int W, bool KS, bool STAGED>
 cudaError_t nt_launch_q(const Problem& P, float zq, cudaStream_t stream) {
   const bool q4 = P.q4 != 0;
-  if (KS && P.k == 1) return q4 ? nt_launch<G, E, true, 1>(P, zq, stream) : nt_launch<G, E, false, 1>(P, zq, stream);
-  if (KS && P.k == 2) return q4 ? nt_launch<G, E, true, 2>(P, zq, stream) : nt_launch<G, E, false, 2>(P, zq, stream);
-  return q4 ? nt_launch<G, E, true, 0>(P, zq, stream) : nt_launch<G, E, false, 0>(P, zq, stream);
+  if (KS && P.k == 1)
+    return q4 ? nt_launch<G, E, W, true, KS ? 1 : 0, STAGED>(P, zq, stream)
+              : nt_launch<G, E, W, false, KS ? 1 : 0, STAGED>(P, zq, stream);
+  if (KS && P.k == 2)
+    return q4 ? nt_launch<G, E, W, true, KS ? 2 : 0, STAGED>(P, zq, stream)
+              : nt_launch<G, E, W, false, KS ? 2 : 0, STAGED>(P, zq, stream);
+  return q4 ? nt_launch<G, E, W, true, 0, STAGED>(P, zq, stream) : nt_launch<G, E, W, false, 0, STAGED>(P, zq, stream);
 }
 
 }  // namespace
 
-int newton_max_n() { return 4096; }
+int newton_max_n() { return 32768; }
 
 // Forward pass of TK_MASK / TK_TOPK with p = 2 or 4/3, rows of up to newton_max_n() elements,
 // no permutation output.
 cudaError_t launch_newton(const Problem& P, cudaStream_t stream) {
   const int n = P.n;
   const float zq = upper_normal_quantile(((double)P.k - 0.5) / (double)n);
-  if (n <= 8) return nt_launch_q<1, 8, true>(P, zq, stream);
-  if (n <= 16) return nt_launch_q<1, 16, true>(P, zq, stream);
-  if (n <= 32) return nt_launch_q<1, 32, true>(P, zq, stream);
-  if (n <= 64) return nt_launch_q<1, 64, true>(P, zq, stream);
-  if (n <= 128) return nt_launch_q<2, 64, true>(P, zq, stream);
-  if (n <= 256) return nt_launch_q<4, 64, true>(P, zq, stream);
-  if (n <= 512) return nt_launch_q<8, 64, false>(P, zq, stream);
-  if (n <= 1024) return nt_launch_q<16, 64, false>(P, zq, stream);
-  if (n <= 2048) return nt_launch_q<32, 64, false>(P, zq, stream);
-  return nt_launch_q<32, 128, false>(P, zq, stream);
+  // 32 keys per lane (more lanes per row and more rows in flight beat longer register rows); one or
+  // two lanes per row go through the staging tile
+  if (n <= 8) return nt_launch_q<1, 8, 1, true, true>(P, zq, stream);
+  if (n <= 16) return nt_launch_q<1, 16, 1, true, true>(P, zq, stream);
+  if (n <= 32) return nt_launch_q<1, 32, 1, true, true>(P, zq, stream);
+  if (n <= 64) return nt_launch_q<2, 32, 1, true, true>(P, zq, stream);
+  if (n <= 128) return nt_launch_q<4, 32, 1, true, false>(P, zq, stream);
+  if (n <= 256) return nt_launch_q<8, 32, 1, false, false>(P, zq, stream);
+  if (n <= 512) return nt_launch_q<16, 32, 1, false, false>(P, zq, stream);
+  if (n <= 1024) return nt_launch_q<32, 32, 1, false, false>(P, zq, stream);
+  if (n <= 2048) return nt_launch_q<32, 32, 2, false, false>(P, zq, stream);
+  if (n <= 4096) return nt_launch_q<32, 32, 4, false, false>(P, zq, stream);
+  if (n <= 8192) return nt_launch_q<32, 32, 8, false, false>(P, zq, stream);
+  if (n <= 16384) return nt_launch_q<32, 32, 16, false, false>(P, zq, stream);
+  return nt_launch_q<32, 64, 16, false, false>(P, zq, stream);
 }
 
 }  // namespace tk
