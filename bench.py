@@ -6,8 +6,12 @@
 One step = one pass of the whole path over one batch of the workload: for every
 (p, lambda) variant of the workload, tk_fwd_ex (sort, isotonic solve, dual map,
 un-permute; row state saved) followed by tk_vjp from that state.  The default
-workload is the MoE-router configuration (16384 tokens x 64 experts, k = 2,
-p in {2, 4/3}, lambda in {0.1, 1}).  Inputs are seeded synthetic data, resident
+workload is the n = 4096 shape of the 2^26-element sweep (16384 rows, k = 512,
+lambda = 1, p in {2, 4/3}): the largest row length the 50 %-of-HBM target is
+stated for.  The other workloads (the remaining sweep shapes, MoE router,
+class-logit, expert-choice, pruning) are timed after it and reported under
+"other_workloads", each with its own roofline fractions and oracle timing.
+Inputs are seeded synthetic data, resident
 in HBM before the timed region; each (variant, step) uses the next of a ring of
 input/output buffer sets whose total size exceeds the L2 cache, so no step
 finds its inputs in L2.  The step's launches are captured once per buffer set in
@@ -160,10 +164,21 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------ CPU oracle legs
-def time_oracle(cases, min_seconds: float, max_rows_elements: int = 1 << 22):
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except Exception:
+        pass
+    return "unknown"
+
+
+def time_oracle(cases, min_seconds: float, max_rows_elements: int = 1 << 22, single_thread: bool = False):
     """Times the oracle (forward + VJP) on a bounded sample of the workload: for each variant
     the leading rows up to max_rows_elements elements; repeated until min_seconds have passed."""
     from oracle import tko
+    flags = tko.FLAG_SINGLE_THREAD if single_thread else 0
     inputs = []
     for c in cases:
         rows = max(1, min(c.rows, max_rows_elements // c.n))
@@ -174,14 +189,23 @@ def time_oracle(cases, min_seconds: float, max_rows_elements: int = 1 << 22):
     reps, t0 = 0, time.perf_counter()
     while True:
         for c, x, g in inputs:
-            tko.fwd(x, c.k, c.p, c.lam, c.mode)
-            tko.vjp(x, g, c.k, c.p, c.lam, c.mode)
+            tko.fwd(x, c.k, c.p, c.lam, c.mode, flags=flags)
+            tko.vjp(x, g, c.k, c.p, c.lam, c.mode, flags=flags)
         reps += 1
         dt = time.perf_counter() - t0
         if dt >= min_seconds or reps >= 1000:
             break
     sample = "; ".join(f"{c.name}: first {x.shape[0]} of {c.rows} rows" for c, x, _ in inputs)
-    return elements * reps / dt, dt / reps, tko.num_threads(), f"{reps} pass(es) over [{sample}]"
+    threads = 1 if single_thread else tko.num_threads()
+    return elements * reps / dt, dt / reps, threads, f"{reps} pass(es) over [{sample}]"
+
+
+def oracle_baseline(cases, seconds: float, max_rows_elements: int = 1 << 22):
+    """The cpu_baseline object: the oracle on all host cores and on one, on the same bounded sample."""
+    v, sec, threads, sample = time_oracle(cases, seconds, max_rows_elements)
+    v1, sec1, _, _ = time_oracle(cases, max(0.2 * seconds, 0.5), max_rows_elements // 8, single_thread=True)
+    return {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+            "ms_per_pass": sec * 1e3, "single_thread_value": v1, "cpu_model": cpu_model()}
 
 
 def run_reference(args):
@@ -204,7 +228,7 @@ def run_reference(args):
         "config": {"workload": args.workload, "step": "oracle forward + VJP on a bounded sample",
                    "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                         "sample": sample},
+                         "sample": sample, "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -235,7 +259,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="moe_router")
+    ap.add_argument("--workload", default="sweep_n4096")
     ap.add_argument("--impl", default="tk", choices=["tk", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="plain launches instead of CUDA graphs")
     ap.add_argument("--no-extra", action="store_true", help="skip the other workloads' summary")
@@ -314,54 +338,39 @@ def main():
         if ROWS_LIMIT:
             line["config"]["rows_limit"] = ROWS_LIMIT
         if world == 1 and args.cpu_seconds > 0:
-            v, sec, threads, sample = time_oracle(workload_cases(args.workload), args.cpu_seconds)
-            line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle",
-                                    "sample": sample, "ms_per_pass": sec * 1e3}
+            line["cpu_baseline"] = oracle_baseline(workload_cases(args.workload), args.cpu_seconds)
         if world == 1:
+            line["solver_paths"] = solver_paths(args.workload, res, dev, tk, torch, peak)
             if not args.no_extra:
                 extra = []
-                names = ["class_logit", "expert_choice", "pruning"] + [f"sweep_n{n}" for n in (8, 64, 512, 4096, 32768)]
+                names = ["moe_router", "class_logit", "expert_choice", "pruning"] + \
+                        [f"sweep_n{n}" for n in (8, 64, 512, 4096, 32768)]
                 for name in names:
                     if name == args.workload:
                         continue
                     try:
-                        r = measure(name, 10, 3, dev, tk, torch, graph=False, barrier=barrier,
+                        r = measure(name, 10, 3, dev, tk, torch, graph=(name == "moe_router"), barrier=barrier,
                                     sample_clocks=False, e2e=False)
                         v2 = r["elements_per_step"] * r["steps"] / (r["ms_total"] * 1e-3)
+                        d2 = r["dominant"]
+                        a2 = d2["alg_bytes_per_launch"] / (d2["avg_us"] * 1e-6) / 1e9
                         entry = {"workload": name, "value": v2, "unit": UNIT,
                                  "ms_per_step": r["ms_total"] / r["steps"],
                                  "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
+                                 "roofline": {"bound": "hbm", "kernel": d2["name"], "achieved": a2, "peak": peak,
+                                              "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": a2 / peak,
+                                              "avg_launch_us": d2["avg_us"],
+                                              "alg_bytes_per_launch": d2["alg_bytes_per_launch"]},
                                  "kernels": r["kernels"], "config": r["config"]}
-                        if name.startswith("sweep_n"):
-                            entry["dykstra_forward_100_sweeps"] = time_solver_forward(
-                                name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
+                        entry.update(solver_paths(name, r, dev, tk, torch, peak))
                         if name == "class_logit":
                             # the loss the paper trains that classifier with (k = 3), on the same logits
                             entry["smooth_topk_loss_k3"] = time_topk_loss(name, dev, tk, torch, k=3, peak=peak)
                         if name == "expert_choice":
                             # the same scores stored [tokens, experts]: the operator along the slow axis
                             entry["slow_axis_fwd_vjp"] = time_cols(name, dev, tk, torch, peak)
-                        if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
-                            entry["dykstra_forward_10_sweeps"] = time_solver_forward(
-                                name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
-                        if name in ("sweep_n64", "sweep_n4096"):
-                            # p = 1.5 (q = 3): no closed-form block solve; the library picks the path
-                            # (n = 64: sorting kernel + per-row Newton; n = 4096: sort-free solver)
-                            entry["general_p_1.5_forward"] = time_solver_forward(
-                                name, dev, tk, torch, tk.TK_SOLVER_AUTO, p_override=1.5)
-                        ncase = workload_cases(name)[0].n
-                        if 512 <= ncase <= 16384:
-                            # the same exact result without the sort (solver = TK_SOLVER_THRESHOLD),
-                            # reported beside the sorted path, never instead of it
-                            sf = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_THRESHOLD)
-                            vj = {round(kx["p"], 6): kx for kx in sf}
-                            fwd_us = sum(x["avg_us"] for x in sf)
-                            vjp_us = r["kernels"][1]["avg_us"] * r["kernels"][1]["launches_per_step"]
-                            el = r["elements_per_step"]
-                            entry["sort_free"] = {
-                                "forward": sf,
-                                "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * el / ((fwd_us + vjp_us) * 1e-6) / 1e9 / peak,
-                                "note": "tk_fwd_ex(solver=TK_SOLVER_THRESHOLD, state saved) + tk_vjp(from state)"}
+                        if args.cpu_seconds > 0:
+                            entry["cpu_baseline"] = oracle_baseline(workload_cases(name), min(3.0, args.cpu_seconds))
                         extra.append(entry)
                     except tk.TkError as e:
                         extra.append({"workload": name, "unavailable": str(e)})
@@ -370,6 +379,32 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def solver_paths(name, r, dev, tk, torch, peak):
+    """The forward pass of a workload through the other solver paths, reported beside the timed one
+    (tk_fwd_ex with the default solver: for phi(x) = x the threshold form, which needs no sort)."""
+    out = {}
+    cases = workload_cases(name)
+    ncase, mode = cases[0].n, cases[0].mode
+    vjp_us = r["kernels"][1]["avg_us"] * r["kernels"][1]["launches_per_step"]
+    el = r["elements_per_step"]
+    if mode != wl.MODE_TOPKMAG and ncase <= 32768:
+        # TK_SOLVER_PAV: the keys are sorted (no permutation asked for: keys alone), then the same block solve
+        sf = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_PAV)
+        fwd_us = sum(x["avg_us"] for x in sf)
+        out["sorted_path"] = {
+            "forward": sf,
+            "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * el / ((fwd_us + vjp_us) * 1e-6) / 1e9 / peak,
+            "note": "tk_fwd_ex(solver=TK_SOLVER_PAV, state saved) + tk_vjp(from state)"}
+    if name.startswith("sweep_n"):
+        out["dykstra_forward_100_sweeps"] = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=100)
+    if name == "expert_choice":     # that experiment ran 10 sweeps of Dykstra
+        out["dykstra_forward_10_sweeps"] = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_DYKSTRA, sweeps=10)
+    if name in ("sweep_n64", "sweep_n4096"):
+        # p = 1.5 (q = 3): no closed-form block solve; the library picks the path
+        out["general_p_1.5_forward"] = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_AUTO, p_override=1.5)
+    return out
 
 
 def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, p_override=None):
@@ -383,7 +418,7 @@ def time_solver_forward(workload, dev, tk, torch, solver, sweeps=0, launches=3, 
     for c in cases:
         th = torch.from_numpy(c.theta()).to(dev)
         y = torch.empty_like(th)
-        st = tk.new_state(c.rows, dev) if solver == tk.TK_SOLVER_THRESHOLD else None
+        st = tk.new_state(c.rows, dev) if solver != tk.TK_SOLVER_DYKSTRA else None
         wsb = tk.tk_workspace_bytes(c.rows, c.n, c.k, c.p, c.mode, solver) if solver == tk.TK_SOLVER_DYKSTRA else 0
         ws = torch.empty(wsb, dtype=torch.uint8, device=dev) if wsb else None
         run = lambda: tk.tk_fwd_ex(th, c.rows, c.n, c.k, c.p, c.lam, c.mode, y, solver=solver, sweeps=sweeps,

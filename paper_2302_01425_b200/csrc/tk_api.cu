@@ -164,8 +164,9 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
   // phi(x) = x with a closed-form block solve, nothing but values asked for: the threshold form needs no
   // order at all (TK_SOLVER_PAV keeps the sort)
-  const bool by_threshold = (solver == TK_SOLVER_AUTO || solver == TK_SOLVER_THRESHOLD) && mode != TK_TOPKMAG &&
-                            qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
+  // (rows of up to 16 elements sort faster than they iterate: AUTO keeps the sort there)
+  const bool by_threshold = (solver == TK_SOLVER_THRESHOLD || (solver == TK_SOLVER_AUTO && n > 16)) &&
+                            mode != TK_TOPKMAG && qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
   if (by_threshold) {
     cudaError_t en = tk::launch_newton(P, (cudaStream_t)stream);
     return en == cudaSuccess ? TK_OK : TK_ERR_CUDA;
