@@ -35,14 +35,13 @@
 #include <float.h>
 #include <math.h>
 
-#include "tk_common.cuh"
+#include "tk_team.cuh"
 
 namespace tk {
 
 namespace {
 
-constexpr int kNtWarps = 4;               // warps per thread block
-constexpr int kNtThreads = kNtWarps * 32;
+constexpr int kNtWarps = kTeamWarps;      // warps per thread block (more when a row takes more)
 constexpr int kNtMaxPasses = 200;
 
 // rotation of the chunk order that makes the per-lane float4 reads of a quarter warp hit 8 bank groups
@@ -50,31 +49,6 @@ template <int E>
 __device__ __forceinline__ int nt_rot(int lane) {
   constexpr int CH = E / 4;
   return CH >= 8 ? lane : (lane * CH) >> 3;
-}
-
-template <int G>
-__device__ __forceinline__ float nt_gsum(float v) {
-#pragma unroll
-  for (int o = G >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-template <int G>
-__device__ __forceinline__ int nt_gsum(int v) {
-#pragma unroll
-  for (int o = G >> 1; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-template <int G>
-__device__ __forceinline__ float nt_gmax(float v) {
-#pragma unroll
-  for (int o = G >> 1; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
-}
-template <int G>
-__device__ __forceinline__ float nt_gmin(float v) {
-#pragma unroll
-  for (int o = G >> 1; o > 0; o >>= 1) v = fminf(v, __shfl_xor_sync(0xffffffffu, v, o));
-  return v;
 }
 
 // keeps (m1 >= m2 >= m3) the three largest values seen
@@ -122,45 +96,11 @@ struct NtRow {
   bool done, noblock, repiv;
 };
 
-// What one pass found at S.off -> the next offset, or the end of the iteration.
-template <bool Q4>
-__device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, float s2, float s3, int k,
-                                        float lam, float lam3, float tol) {
-  const float wid = lam;
-  S.repiv = false;
-  const int m = k - ct;                        // weight the inside keys have to carry
-  if (cm == 0 && ct == k) {                    // F = 0 on a flat piece: no pooled block
-    S.noblock = true; S.done = true; S.a0 = k; S.b0 = k;
-    return;
-  }
-  // more than k keys capped: no piece to solve, the root is further right by an unknown amount
-  const bool have = cm > 0 && m >= 0;
-  float du = 0.0f;
-  bool fpos;                                   // F(tau) > 0: the root is to the right
-  if (have) {
-    float c0;
-    if (!Q4) {
-      c0 = s1 - lam * (float)m;
-      du = __fdividef(c0, (float)cm);
-    } else {
-      const float rhs = lam3 * (float)m;
-      c0 = s3 - rhs;
-      du = nt_cubic(cm, s1, s2, s3, rhs, c0);
-      if ((du > 0.0f) != (c0 > 0.0f)) du = __fdividef(c0, 3.0f * s2);
-    }
-    fpos = c0 > 0.0f;
-    const float adu = fabsf(du);
-    // a pooled block has members of both weights: 1 <= m < cm
-    if (adu <= tol && m >= 1 && m < cm &&
-        ((ct == S.prev_ct && cm == S.prev_cm) || (float)cm * adu <= tol)) {
-      S.done = true; S.a0 = ct; S.b0 = ct + cm;
-      return;
-    }
-  } else {
-    fpos = ct >= k;                            // ct == k here means cm > 0: F > 0
-  }
-  S.prev_ct = ct; S.prev_cm = cm;
-  if (fpos) { S.lo_o = S.off; S.lo_a = S.piv + S.off; } else { S.hi_o = S.off; S.hi_a = S.piv + S.off; }
+// The next offset when the piece's own solution cannot be taken as it is: it left the bracket, there was
+// no piece to solve, six Newton steps have gone by, or the offset has grown large against lambda.  Out
+// of line: the common pass never comes here, and its code stays short.
+__device__ __noinline__ NtRow nt_step_slow(NtRow S, int ct, int cm, int m, float du, bool have, bool fpos,
+                                           float wid, float tol) {
   bool ok = false;
   float nxt = S.off;
   float cand = S.off;
@@ -206,7 +146,7 @@ __device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, floa
   }
   if (nxt == S.off || !(nxt > S.lo_o && nxt < S.hi_o)) {   // bracket exhausted at the resolution of the offset
     S.done = true; S.a0 = ct; S.b0 = ct + cm;
-    return;
+    return S;
   }
   if (fabsf(nxt) > 8.0f * wid) {               // keep the offset small against the keys it is subtracted from
     const float np = S.piv + nxt;
@@ -217,16 +157,61 @@ __device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, floa
     }
   }
   S.off = nxt;
+  return S;
+}
+
+// What one pass found at S.off -> the next offset, or the end of the iteration.
+template <bool Q4>
+__device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, float s2, float s3, int k,
+                                        float lam, float lam3, float tol) {
+  const float wid = lam;
+  S.repiv = false;
+  const int m = k - ct;                        // weight the inside keys have to carry
+  if (cm == 0 && ct == k) {                    // F = 0 on a flat piece: no pooled block
+    S.noblock = true; S.done = true; S.a0 = k; S.b0 = k;
+    return;
+  }
+  // more than k keys capped: no piece to solve, the root is further right by an unknown amount
+  const bool have = cm > 0 && m >= 0;
+  float du = 0.0f;
+  bool fpos;                                   // F(tau) > 0: the root is to the right
+  if (have) {
+    float c0;
+    if (!Q4) {
+      c0 = s1 - lam * (float)m;
+      du = __fdividef(c0, (float)cm);
+    } else {
+      const float rhs = lam3 * (float)m;
+      c0 = s3 - rhs;
+      du = nt_cubic(cm, s1, s2, s3, rhs, c0);
+      if ((du > 0.0f) != (c0 > 0.0f)) du = __fdividef(c0, 3.0f * s2);
+    }
+    fpos = c0 > 0.0f;
+    const float adu = fabsf(du);
+    // a pooled block has members of both weights: 1 <= m < cm
+    if (adu <= tol && m >= 1 && m < cm &&
+        ((ct == S.prev_ct && cm == S.prev_cm) || (float)cm * adu <= tol)) {
+      S.done = true; S.a0 = ct; S.b0 = ct + cm;
+      return;
+    }
+  } else {
+    fpos = ct >= k;                            // ct == k here means cm > 0: F > 0
+  }
+  S.prev_ct = ct; S.prev_cm = cm;
+  if (fpos) { S.lo_o = S.off; S.lo_a = S.piv + S.off; } else { S.hi_o = S.off; S.hi_a = S.piv + S.off; }
+  // the common case: the piece's solution lies inside the bracket and near the pivot
+  const float cand = S.off + du;
+  if (have && m != cm && cand > S.lo_o && cand < S.hi_o && S.nnewt < 6 && fabsf(cand) <= 8.0f * wid) {
+    S.gallop = 0; S.nnewt++; S.off = cand;
+    return;
+  }
+  S = nt_step_slow(S, ct, cm, m, du, have, fpos, wid, tol);
 }
 
 // threads per block, and the blocks per SM the register budget is set for: 24 warps of 80 registers with
 // up to 32 keys per lane, 16 warps of 128 registers with 64
-constexpr int nt_threads(int W) { return W * 32 > kNtThreads ? W * 32 : kNtThreads; }
-constexpr int nt_min_blocks(int E, int W) {
-  const int warps = E >= 128 ? 8 : (E >= 64 ? 16 : 24);
-  const int b = warps * 32 / nt_threads(W);
-  return b < 1 ? 1 : b;
-}
+constexpr int nt_threads(int W) { return team_threads(W); }
+constexpr int nt_min_blocks(int E, int W) { return team_min_blocks(E >= 128 ? 8 : (E >= 64 ? 16 : 24), W); }
 
 // ---------------------------------------------------------------- row access
 // A row is spread over a team of T = G * W lanes (G lanes of one warp, or W whole warps), E keys per
@@ -298,33 +283,6 @@ struct NtIO {
 // values, smallest capped key) run while the row's registers are live, and E more words in flight would spill.
 __device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
 
-// Sum of NV values over the lanes of a row: shuffles inside the warp, then (W > 1) one slot per warp in
-// shared memory and a named barrier over the team's W warps.  red: the team's W * 4 words for this
-// phase (the caller alternates two such buffers, so one barrier per sum is enough).  Every warp adds the
-// slots in the same order: all lanes of the team hold identical results.
-template <int G, int W, int NV>
-__device__ __forceinline__ void nt_allsum(float (&v)[NV], uint32_t& packed, float* red, int wit, int lane, int bar) {
-#pragma unroll
-  for (int i = 0; i < NV; ++i) v[i] = nt_gsum<G>(v[i]);
-  packed = (uint32_t)nt_gsum<G>((int)packed);
-  if (W > 1) {
-    if (lane == 0) {
-#pragma unroll
-      for (int i = 0; i < NV; ++i) red[wit * 4 + i] = v[i];
-      red[wit * 4 + 3] = __uint_as_float(packed);
-    }
-    asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(W * 32) : "memory");
-#pragma unroll
-    for (int i = 0; i < NV; ++i) v[i] = 0.0f;
-    packed = 0;
-#pragma unroll
-    for (int w = 0; w < W; ++w) {
-#pragma unroll
-      for (int i = 0; i < NV; ++i) v[i] += red[w * 4 + i];
-      packed += __float_as_uint(red[w * 4 + 3]);
-    }
-  }
-}
 
 // G lanes per row (W == 1) or W warps per row (G == 32), E keys per lane (E / 4 a power of two).
 // KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1 only).
@@ -425,7 +383,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
     }
     uint32_t none = 0;
-    nt_allsum<G, W, 2>(v, none, red + (phase & 1) * (W * 4), wit, lane, bar);
+    team_allsum<G, W, 2>(v, none, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!(v[1] < INFINITY)) {                  // overflow, an infinity or a NaN: look at the keys themselves
 #pragma unroll
@@ -501,7 +459,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     v[0] = a0 + a1;
     if (Q4) { v[1] = b0 + b1; v[2] = e0 + e1; }
     uint32_t packed = (uint32_t)(ct0 + ct1) | ((uint32_t)(cm0 + cm1) << 16);
-    nt_allsum<G, W, Q4 ? 3 : 1>(v, packed, red + (phase & 1) * (W * 4), wit, lane, bar);
+    team_allsum<G, W, Q4 ? 3 : 1>(v, packed, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!S.done) {
       nt_step<Q4>(S, (int)(packed & 0xffffu), (int)(packed >> 16), v[0], Q4 ? v[1] : 0.0f, Q4 ? v[Q4 ? 2 : 0] : 0.0f,
@@ -545,12 +503,12 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
           if (d[4 * c + j] - S.off >= wid) cmin = fminf(cmin, x4[j]);
         if ((c & 3) == 3) nt_fence();
       }
-      cmin = nt_gmin<G>(cmin);
+      cmin = team_gmin<G>(cmin);
       if (W > 1) {
         float* rb = red + (phase & 1) * (W * 4);
         ++phase;
         if (lane == 0) rb[wit * 4] = cmin;
-        asm volatile("bar.sync %0, %1;" ::"r"(bar), "r"(W * 32) : "memory");
+        team_barrier(bar, W * 32);
         cmin = rb[0];
 #pragma unroll
         for (int w = 1; w < W; ++w) cmin = fminf(cmin, rb[w * 4]);

@@ -1,4 +1,4 @@
-// tk_vjp_state.cu -- VJP from the row state saved by the forward pass.
+// tk_vjp_state.cu -- VJP from the row state saved by the forward pass: rows too long for registers.
 //
 // Prop. 7 makes the Jacobian of the isotonic solution block diagonal with one
 // rank-one block per pooled block; with w = 1_k there is at most one pooled
@@ -10,6 +10,10 @@
 #include "tk_common.cuh"
 
 namespace tk {
+
+// rows held in registers (tk_vjp_team.cu)
+int vjp_team_max_n();
+cudaError_t launch_vjp_team(const Problem& P, cudaStream_t stream);
 
 namespace {
 
@@ -80,110 +84,6 @@ __device__ __forceinline__ float finish(const Problem& P, const Math& M, const R
     o += g * y;
   }
   return o;
-}
-
-// G lanes of a warp per row (G = 1..32, power of two), 32/G rows per warp.  Every lane keeps its
-// CH float4 chunks of theta and g in registers, so the row is read from memory once (n <= 4 G CH).
-// GEN: q is neither 2 nor 4 (rho' through powf); a template flag so that the usual kernels carry no
-// trace of that branch.
-template <int G, int CH, bool GEN>
-__global__ void __launch_bounds__(256) tk_vjp_state_group(const Problem P) {
-  Math M = make_math(P);
-  M.gen = GEN;
-  const int lane = threadIdx.x & 31;
-  const int lig = lane % G;
-  const long long row = ((long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * (32 / G) + lane / G;
-  if (row >= P.rows) return;          // whole groups leave together
-  constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
-  const unsigned mask = kGroupBits << (lane / G * G);
-  const int n = P.n;
-  const float* x_row = P.theta + row * (long long)n;
-  const float* g_row = P.gout + row * (long long)n;
-  float* o_row = P.out + row * (long long)n;
-  float x[CH][4], g[CH][4];
-  if (P.vec4) {
-#pragma unroll
-    for (int c = 0; c < CH; ++c) {
-      const int v = c * G + lig;
-      float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), gv = xv;
-      if (4 * v < n) { xv = __ldg(reinterpret_cast<const float4*>(x_row) + v); gv = __ldg(reinterpret_cast<const float4*>(g_row) + v); }
-      x[c][0] = xv.x; x[c][1] = xv.y; x[c][2] = xv.z; x[c][3] = xv.w;
-      g[c][0] = gv.x; g[c][1] = gv.y; g[c][2] = gv.z; g[c][3] = gv.w;
-    }
-  } else {
-#pragma unroll
-    for (int c = 0; c < CH; ++c)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int i = 4 * (c * G + lig) + j;
-        x[c][j] = (i < n) ? __ldg(x_row + i) : 0.0f;
-        g[c][j] = (i < n) ? __ldg(g_row + i) : 0.0f;
-      }
-  }
-  const RowCtx c = load_ctx(P, M, row);
-  // One classification per element: w = sign * rho' on the pooled block (else 0) and the part of
-  // the result that does not depend on the block mean; then
-  //   o = w ((chi g - r0) - delta) + fixed,   r0 = fl(A / D),   delta = (sum w' (chi g - r0) - m r0) / D.
-  const bool jt = P.mode == TK_TOPK && P.jvp;          // topk JVP: theta multiplies outside the block mean
-  auto chi_of = [&](float xv) -> float {
-    return M.mag ? (signbit(xv) ? -1.0f : 1.0f) : ((P.mode == TK_TOPK && !jt) ? xv : 1.0f);
-  };
-  float w[CH][4], fixed[CH][4];
-  float A = 0.f, D = 0.f;
-#pragma unroll
-  for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const float xv = x[ch][j], gv = g[ch][j];
-      const bool in = 4 * (ch * G + lig) + j < n;
-      float tt = 0.0f;
-      const float key = sort_key(xv, M.mag);
-      const int cls = in ? classify(c, key, tt) : 0;
-      const float sgn = (M.mag && signbit(xv)) ? -1.0f : 1.0f;
-      const float chi = chi_of(xv);
-      const float dr = cls == 1 ? M.drho(tt) : 0.0f;
-      float f = (cls == 2 && M.mag) ? gv * M.top_slope(key) : 0.0f;          // sgn chi = 1 there
-      if (P.mode == TK_TOPK) f += gv * (cls == 2 ? 1.0f : (cls == 1 ? M.rho(tt) : 0.0f));
-      w[ch][j] = sgn * dr;
-      fixed[ch][j] = f;
-      D += dr;
-      A += dr * chi * gv;
-    }
-  float ratio = 0.0f, delta = 0.0f;
-  if (c.has_block) {
-#pragma unroll
-    for (int o = G >> 1; o > 0; o >>= 1) {
-      A += __shfl_xor_sync(mask, A, o);
-      D += __shfl_xor_sync(mask, D, o);
-    }
-    if (M.mag) D += (float)c.m;
-    ratio = D > 0.0f ? A / D : 0.0f;
-    float A2 = 0.f;
-#pragma unroll
-    for (int ch = 0; ch < CH; ++ch)
-#pragma unroll
-      for (int j = 0; j < 4; ++j)
-        A2 = fmaf(fabsf(w[ch][j]), fmaf(chi_of(x[ch][j]), g[ch][j], -ratio), A2);   // |w| = rho'
-#pragma unroll
-    for (int o = G >> 1; o > 0; o >>= 1) A2 += __shfl_xor_sync(mask, A2, o);
-    if (M.mag) A2 -= (float)c.m * ratio;
-    delta = D > 0.0f ? A2 / D : 0.0f;
-  }
-#pragma unroll
-  for (int ch = 0; ch < CH; ++ch) {
-    const int v = ch * G + lig;
-    float o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      o[j] = fmaf(w[ch][j] * (jt ? x[ch][j] : 1.0f), fmaf(chi_of(x[ch][j]), g[ch][j], -ratio) - delta, fixed[ch][j]);
-    }
-    if (P.vec4) {
-      if (4 * v < n) reinterpret_cast<float4*>(o_row)[v] = make_float4(o[0], o[1], o[2], o[3]);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) if (4 * v + j < n) o_row[4 * v + j] = o[j];
-    }
-  }
 }
 
 // one thread block per row
@@ -305,32 +205,10 @@ cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t 
 }
 
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream) {
+  // rows of up to 16384 elements are held in registers (tk_vjp_team.cu); longer ones are streamed twice
+  if (P.n <= vjp_team_max_n()) return launch_vjp_team(P, stream);
   const bool gen = P.qm1 > 0.0f;
-  if (P.n <= 512) {
-    // lanes per row: two float4 per lane (one for n <= 4), four for 256 < n <= 512
-    if (P.n > 256) {
-      const unsigned blocks = (unsigned)((P.rows + 7) / 8);
-      (gen ? tk_vjp_state_group<32, 4, true> : tk_vjp_state_group<32, 4, false>)<<<blocks, 256, 0, stream>>>(P);
-      return cudaGetLastError();
-    }
-    int G = 1;
-    while (G < 32 && G * 8 < P.n) G <<= 1;
-    const long long rows_per_block = 8 * (32 / G);
-    const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
-    switch (G) {
-      case 1:
-        if (P.n <= 4) (gen ? tk_vjp_state_group<1, 1, true> : tk_vjp_state_group<1, 1, false>)<<<blocks, 256, 0, stream>>>(P);
-        else (gen ? tk_vjp_state_group<1, 2, true> : tk_vjp_state_group<1, 2, false>)<<<blocks, 256, 0, stream>>>(P);
-        break;
-      case 2: (gen ? tk_vjp_state_group<2, 2, true> : tk_vjp_state_group<2, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
-      case 4: (gen ? tk_vjp_state_group<4, 2, true> : tk_vjp_state_group<4, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
-      case 8: (gen ? tk_vjp_state_group<8, 2, true> : tk_vjp_state_group<8, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
-      case 16: (gen ? tk_vjp_state_group<16, 2, true> : tk_vjp_state_group<16, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
-      default: (gen ? tk_vjp_state_group<32, 2, true> : tk_vjp_state_group<32, 2, false>)<<<blocks, 256, 0, stream>>>(P); break;
-    }
-  } else {
-    (gen ? tk_vjp_state_cta<true> : tk_vjp_state_cta<false>)<<<(unsigned)P.rows, 256, 0, stream>>>(P);
-  }
+  (gen ? tk_vjp_state_cta<true> : tk_vjp_state_cta<false>)<<<(unsigned)P.rows, 256, 0, stream>>>(P);
   return cudaGetLastError();
 }
 
