@@ -360,11 +360,15 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     io.load_raw(c, x4);
     d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
   }
+  // a row that fills its lanes exactly has no slot to mark (and a -infinity in it shows in the sums below)
+  const bool full = n == (STAGED ? G : G * W) * E;
+  if (!full) {
 #pragma unroll
-  for (int c = 0; c < CH; ++c) {
-    float x4[4] = {d[4 * c], d[4 * c + 1], d[4 * c + 2], d[4 * c + 3]};
-    io.mask(c, x4, &bad);
-    d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
+    for (int c = 0; c < CH; ++c) {
+      float x4[4] = {d[4 * c], d[4 * c + 1], d[4 * c + 2], d[4 * c + 3]};
+      io.mask(c, x4, &bad);
+      d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
+    }
   }
 
   // ---- start: bracket and first tau
@@ -377,17 +381,25 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     // sums about the row's first key: mean and spread of the keys
     const float x0 = __ldg(io.src);
     float v[2] = {0.f, 0.f};
+    if (full) {
 #pragma unroll
-    for (int i = 0; i < E; ++i) {
-      const float dd = (d[i] == -INFINITY) ? 0.0f : d[i] - x0;
-      v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
+      for (int i = 0; i < E; ++i) {
+        const float dd = d[i] - x0;
+        v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < E; ++i) {
+        const float dd = (d[i] == -INFINITY) ? 0.0f : d[i] - x0;
+        v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
+      }
     }
     uint32_t none = 0;
     team_allsum<G, W, 2>(v, none, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!(v[1] < INFINITY)) {                  // overflow, an infinity or a NaN: look at the keys themselves
 #pragma unroll
-      for (int i = 0; i < E; ++i) bad |= !(fabsf(d[i]) < INFINITY) && d[i] != -INFINITY;
+      for (int i = 0; i < E; ++i) bad |= !(fabsf(d[i]) < INFINITY) && (full || d[i] != -INFINITY);
     }
     const float inv_n = 1.0f / (float)n;
     const float mean_d = v[0] * inv_n;
@@ -404,7 +416,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
 #pragma unroll
     for (int i = 0; i < E; ++i) {
       nt_top3(d[i], m1, m2, m3);
-      fin = fmaf(d[i] == -INFINITY ? 0.0f : d[i], 0.0f, fin);
+      fin = fmaf((!full && d[i] == -INFINITY) ? 0.0f : d[i], 0.0f, fin);
     }
     bad |= fin != fin;
 #pragma unroll
