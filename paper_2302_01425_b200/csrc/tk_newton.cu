@@ -375,7 +375,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   NtRow S;
   S.done = false; S.noblock = false; S.repiv = false;
   S.a0 = k; S.b0 = k; S.gallop = 0; S.nnewt = 0; S.prev_ct = -1; S.prev_cm = -1; S.edge_tried = false;
-  S.off = 0.0f; S.piv = 0.0f;
+  S.off = 0.0f; S.piv = 0.0f; S.lo_o = -INFINITY; S.hi_o = INFINITY;
   float lo = -FLT_MAX, hi = FLT_MAX;
   if (KSEL == 0) {
     // sums about the row's first key: mean and spread of the keys
@@ -426,17 +426,18 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       nt_top3(p1, m1, m2, m3); nt_top3(p2, m1, m2, m3); nt_top3(p3, m1, m2, m3);
     }
     const float c = KSEL == 1 ? m1 : m2, sk = KSEL == 1 ? m2 : m3;   // k-th and (k+1)-th largest key
+    // The bracket (s_k - lambda, s_{k+1}) is kept relative to the pivot s_{k+1}: the gap s_k - s_{k+1}
+    // is exact there, and so is the end s_k - lambda the root may sit a hair inside of.
+    const float dc = c - sk;
     lo = c - wid; hi = sk;
-    if (!(lo < sk)) {                          // vtop(s_k) >= s_{k+1}: no violation, no block
+    if (!(dc < wid)) {                         // vtop(s_k) >= s_{k+1}: no violation, no block
       S.piv = c; S.off = -wid; S.done = true; S.noblock = true;
     } else {
-      S.piv = 0.5f * (lo + hi);
+      S.piv = sk; S.lo_o = dc - wid; S.hi_o = 0.0f; S.off = 0.5f * S.lo_o;
     }
   }
   const bool early = S.done && S.noblock;      // pivot already exact
   S.lo_a = lo; S.hi_a = hi;
-  S.lo_o = KSEL == 0 ? -INFINITY : lo - S.piv;
-  S.hi_o = KSEL == 0 ? INFINITY : hi - S.piv;
 #pragma unroll
   for (int i = 0; i < E; ++i) d[i] -= S.piv;
 
@@ -651,7 +652,11 @@ cudaError_t launch_newton(const Problem& P, cudaStream_t stream) {
   if (n <= 8) return nt_launch_q<1, 8, 1, true, true>(P, zq, stream);
   if (n <= 16) return nt_launch_q<1, 16, 1, true, true>(P, zq, stream);
   if (n <= 32) return nt_launch_q<1, 32, 1, true, true>(P, zq, stream);
-  if (n <= 64) return nt_launch_q<2, 32, 1, true, true>(P, zq, stream);
+  if (n <= 64) {
+    // a router-sized batch leaves the SMs short of warps at 16 rows per warp: 8 rows per warp then
+    if (P.rows < (long long)sm_count() * 24 * 16) return nt_launch_q<4, 16, 1, true, false>(P, zq, stream);
+    return nt_launch_q<2, 32, 1, true, true>(P, zq, stream);
+  }
   if (n <= 128) return nt_launch_q<4, 32, 1, true, false>(P, zq, stream);
   if (n <= 256) return nt_launch_q<8, 32, 1, false, false>(P, zq, stream);
   if (n <= 512) return nt_launch_q<16, 32, 1, false, false>(P, zq, stream);

@@ -272,6 +272,49 @@ def test_sweep_n32768_sampled_rows():
         run_case(x, case.k, case.p, case.lam, case.mode, g, label=case.name)
 
 
+def test_sweep_n32768_full_launch_sampled_rows():
+    """The 2048 x 32768 launches the benchmark times (both p), 32 rows of each checked by the oracle."""
+    from parity import run_sampled
+    for case in wl.shape_sweep_cases():
+        if case.n != 32768:
+            continue
+        x = case.theta()
+        g = case.cotangent(x)
+        sample = np.random.Generator(np.random.PCG64(32768)).choice(case.rows, 32, replace=False)
+        run_sampled(x, case.k, case.p, case.lam, case.mode, g, np.sort(sample), label=case.name + " full launch")
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_threshold_form_small_k_and_layout_edges(p):
+    """The sort-free default path: k = 1 and k = 2 (the k + 1 largest keys tracked exactly), ties and
+    near-ties at the top, row lengths on both sides of every lane layout, row counts that leave the
+    last warp partly empty, and the cases where the root sits at the end of its bracket."""
+    from parity import run_case
+    for n in (17, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 511, 512, 513, 1023, 1024, 1025,
+              2047, 2048, 2049, 4095, 4096, 4097, 8193, 16385):
+        rows = 5 if n > 2048 else 43
+        x = rows_of(n, rows, 700 + n)
+        g = wl.cotangent_like(x, 700 + n)
+        for k, lam in ((1, 1.0), (2, 0.1), (2, 1.0), (max(1, n // 8), 1.0), (n - 1, 0.3), (n, 1.0)):
+            if k > n:
+                continue
+            run_case(x, k, p, lam, tk.TK_MASK, g, check_perm=False, label=f"n={n} k={k} lam={lam} p={p}")
+        run_case(x, 2, p, 0.5, tk.TK_TOPK, g, check_perm=False, label=f"topk n={n} k=2 p={p}")
+    # ties and near-ties across rank k for k = 1, 2: equal top keys, a runner-up one ulp below,
+    # a gap of exactly lambda (no block), a gap a hair below lambda (block with rho = 1 - 1e-7)
+    y = rows_of(64, 64, 811)
+    y[:, 0] = 3.0; y[:, 1] = 3.0
+    y[8:16, 1] = np.nextafter(np.float32(3.0), np.float32(0.0))
+    y[16:24, 2] = 3.0
+    y[24:32, 1] = 2.5; y[24:32, 2] = 2.0
+    y[32:40, 1] = 2.5; y[32:40, 2] = np.nextafter(np.float32(2.0), np.float32(3.0))
+    y[40:48, 1] = 2.0
+    y[48:56, 1] = np.nextafter(np.float32(2.0), np.float32(3.0))
+    gy = wl.cotangent_like(y, 811)
+    for k, lam in ((1, 1.0), (2, 0.5), (2, 1.0), (1, 0.5), (3, 0.5)):
+        run_case(y, k, p, lam, tk.TK_MASK, gy, check_perm=False, label=f"top ties k={k} lam={lam} p={p}")
+
+
 @pytest.mark.parametrize("p", [2.0, P43])
 def test_dykstra_path_matches_oracle_sweeps(p):
     """Alternating projections with a fixed sweep count: same count in the oracle, <= 1e-5."""
