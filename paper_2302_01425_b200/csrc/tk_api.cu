@@ -18,6 +18,9 @@ cudaError_t launch_ctav(const Problem& P, cudaStream_t stream);
 cudaError_t launch_thr(const Problem& P, cudaStream_t stream);
 cudaError_t launch_newton(const Problem& P, cudaStream_t stream);
 int newton_max_n();
+// the same for a few rows of any length, the row in global memory (tk_long_newton.cu)
+size_t long_newton_scratch_bytes();
+cudaError_t launch_long_newton(const Problem& P, void* scratch, cudaStream_t stream);
 // alternating-projection solver path (tk_dykstra.cu)
 cudaError_t launch_dykstra(const Problem& P, cudaStream_t stream);
 int dykstra_cluster_max_n();
@@ -166,10 +169,20 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
   // order at all (TK_SOLVER_PAV keeps the sort)
   // (rows of up to 16 elements sort faster than they iterate: AUTO keeps the sort there)
   const bool by_threshold = (solver == TK_SOLVER_THRESHOLD || (solver == TK_SOLVER_AUTO && n > 16)) &&
-                            mode != TK_TOPKMAG && qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
+                            qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
   if (by_threshold) {
     cudaError_t en = tk::launch_newton(P, (cudaStream_t)stream);
     return en == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+  }
+  // A few very long rows (the pruning row): the same iteration with the row streamed from L2, all SMs on
+  // one row at a time.  Many long rows keep the sorting pipeline, which works on all of them at once.
+  if ((solver == TK_SOLVER_AUTO || solver == TK_SOLVER_THRESHOLD) && qm1 == 0.0 && P.perm_out == nullptr &&
+      n > tk::newton_max_n() && rows <= 16) {
+    s = check_workspace(opts, rows, n);
+    if (s != TK_OK) return s;
+    if (opts->workspace_bytes < tk::long_newton_scratch_bytes()) return TK_ERR_WORKSPACE;
+    cudaError_t eln = tk::launch_long_newton(P, opts->workspace, (cudaStream_t)stream);
+    return eln == cudaSuccess ? TK_OK : TK_ERR_CUDA;
   }
   if (solver == TK_SOLVER_THRESHOLD) {
     // no sort, hence no permutation to return; rows held on chip only

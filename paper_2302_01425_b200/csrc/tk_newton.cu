@@ -35,14 +35,24 @@
 #include <float.h>
 #include <math.h>
 
+#include "tk_newton_core.cuh"
 #include "tk_team.cuh"
 
 namespace tk {
 
+// z with P(N(0,1) > z) = tail, by bisection on erfc (a starting guess for the iteration: 1e-6 is plenty)
+float upper_normal_quantile(double tail) {
+  double lo = -8.0, hi = 8.0;
+  for (int i = 0; i < 28; ++i) {
+    const double mid = 0.5 * (lo + hi);
+    if (0.5 * erfc(mid * 0.70710678118654752440) > tail) lo = mid; else hi = mid;
+  }
+  return (float)(0.5 * (lo + hi));
+}
+
 namespace {
 
 constexpr int kNtWarps = kTeamWarps;      // warps per thread block (more when a row takes more)
-constexpr int kNtMaxPasses = 200;
 
 // rotation of the chunk order that makes the per-lane float4 reads of a quarter warp hit 8 bank groups
 template <int E>
@@ -58,154 +68,6 @@ __device__ __forceinline__ void nt_top3(float x, float& m1, float& m2, float& m3
   float r2 = fminf(m2, r);
   m2 = fmaxf(m2, r);
   m3 = fmaxf(m3, r2);
-}
-
-// Root of g(u) = sum_i (t_i - u)^3 - rhs (rhs >= 0) over the cm inside keys, from their power sums.
-// g is decreasing.  The anchor of the sums is the current iterate, so once the outer iteration is
-// close the root is near 0 and Newton from 0 takes two steps; fp32 is enough there (u -> 0).  When
-// the first step is not small against the spread of the t_i, the start is mu - cbrt(rhs / cm)
-// instead, mu the mean of the t_i: by Jensen g >= 0 there, i.e. it is left of the root, where g is
-// convex and Newton increases monotonically to the root.  c0 = g(0).
-__device__ __forceinline__ float nt_cubic(int cm, float s1, float s2, float s3, float rhs, float c0) {
-  const float fcm = (float)cm;
-  const float inv_cm = __fdividef(1.0f, fcm);
-  const float spread2 = s2 * inv_cm;                       // mean of t^2
-  float u = __fdividef(c0, 3.0f * s2);                     // Newton step from 0
-  if (u * u > 0.01f * spread2) u = s1 * inv_cm - cbrtf(rhs * inv_cm);
-  const float spread = sqrtf(spread2);
-#pragma unroll 1
-  for (int it = 0; it < 8; ++it) {
-    const float g = ((-fcm * u + 3.0f * s1) * u - 3.0f * s2) * u + c0;
-    const float gp = -3.0f * ((fcm * u - 2.0f * s1) * u + s2);
-    if (!(gp < 0.0f)) break;
-    const float st = -__fdividef(g, gp);
-    u += st;
-    if (fabsf(st) <= 1e-7f * (fabsf(u) + spread)) break;
-  }
-  return u;
-}
-
-struct NtRow {
-  float piv, off;            // tau = piv + off
-  float lo_o, hi_o;          // bracket of the offset: F > 0 at lo_o, F <= 0 at hi_o
-  float lo_a, hi_a;          // the same bracket as absolute values of tau
-  int prev_ct, prev_cm;      // classes of the pass before
-  int gallop, nnewt;
-  bool edge_tried;
-  int a0, b0;
-  bool done, noblock, repiv;
-};
-
-// The next offset when the piece's own solution cannot be taken as it is: it left the bracket, there was
-// no piece to solve, six Newton steps have gone by, or the offset has grown large against lambda.  Out
-// of line: the common pass never comes here, and its code stays short.
-__device__ __noinline__ NtRow nt_step_slow(NtRow S, int ct, int cm, int m, float du, bool have, bool fpos,
-                                           float wid, float tol) {
-  bool ok = false;
-  float nxt = S.off;
-  float cand = S.off;
-  if (have) {
-    cand = S.off + du;
-    // every inside key would have to reach the cap: aim just past it, so that they read as capped
-    if (m == cm) cand -= 0.5f * tol;
-    ok = cand > S.lo_o && cand < S.hi_o && S.nnewt < 6;
-    nxt = cand;
-  }
-  if (ok) {
-    S.gallop = 0; S.nnewt++;
-  } else {
-    S.nnewt = 0;
-    const float width = S.hi_o - S.lo_o;
-    if (have && !S.edge_tried && (cand <= S.lo_o || cand >= S.hi_o)) {
-      // The piece's root lies at the end of the bracket or a hair beyond it: the true root is
-      // closer to that end than the offset resolves (a key whose rho is 1 - 1e-9).  Look just inside.
-      const float near = fmaxf(tol, width * (1.0f / 64.0f));
-      float e = NAN;
-      if (cand <= S.lo_o && S.lo_o - cand <= near) e = S.lo_o + tol;
-      else if (cand >= S.hi_o && cand - S.hi_o <= near) e = S.hi_o - tol;
-      if (e > S.lo_o && e < S.hi_o) { nxt = e; ok = true; S.edge_tried = true; }
-    }
-    if (!ok && width > 2.0f * wid && S.gallop < 8) {
-      const float step = ldexpf(wid, S.gallop);
-      S.gallop++;
-      const float c2 = fpos ? S.off + step : S.off - step;
-      ok = c2 > S.lo_o && c2 < S.hi_o;
-      nxt = c2;
-    }
-    if (!ok) {
-      S.edge_tried = false;
-      nxt = 0.5f * (S.lo_o + S.hi_o);
-      if (!(width <= 4096.0f * wid)) {         // many binades (or not finite): halve the ordered integer keys
-        const uint32_t kl = f2key(S.lo_a), kh = f2key(S.hi_a);
-        if (kh > kl) {
-          const float c2 = key2f(kl + (kh - kl) / 2) - S.piv;
-          if (c2 > S.lo_o && c2 < S.hi_o) nxt = c2;
-        }
-      }
-    }
-  }
-  if (nxt == S.off || !(nxt > S.lo_o && nxt < S.hi_o)) {   // bracket exhausted at the resolution of the offset
-    S.done = true; S.a0 = ct; S.b0 = ct + cm;
-    return S;
-  }
-  if (fabsf(nxt) > 8.0f * wid) {               // keep the offset small against the keys it is subtracted from
-    const float np = S.piv + nxt;
-    if (np != S.piv) {
-      const float delta = np - S.piv;
-      S.lo_o -= delta; S.hi_o -= delta; nxt -= delta;
-      S.piv = np; S.repiv = true;
-    }
-  }
-  S.off = nxt;
-  return S;
-}
-
-// What one pass found at S.off -> the next offset, or the end of the iteration.
-template <bool Q4>
-__device__ __forceinline__ void nt_step(NtRow& S, int ct, int cm, float s1, float s2, float s3, int k,
-                                        float lam, float lam3, float tol) {
-  const float wid = lam;
-  S.repiv = false;
-  const int m = k - ct;                        // weight the inside keys have to carry
-  if (cm == 0 && ct == k) {                    // F = 0 on a flat piece: no pooled block
-    S.noblock = true; S.done = true; S.a0 = k; S.b0 = k;
-    return;
-  }
-  // more than k keys capped: no piece to solve, the root is further right by an unknown amount
-  const bool have = cm > 0 && m >= 0;
-  float du = 0.0f;
-  bool fpos;                                   // F(tau) > 0: the root is to the right
-  if (have) {
-    float c0;
-    if (!Q4) {
-      c0 = s1 - lam * (float)m;
-      du = __fdividef(c0, (float)cm);
-    } else {
-      const float rhs = lam3 * (float)m;
-      c0 = s3 - rhs;
-      du = nt_cubic(cm, s1, s2, s3, rhs, c0);
-      if ((du > 0.0f) != (c0 > 0.0f)) du = __fdividef(c0, 3.0f * s2);
-    }
-    fpos = c0 > 0.0f;
-    const float adu = fabsf(du);
-    // a pooled block has members of both weights: 1 <= m < cm
-    if (adu <= tol && m >= 1 && m < cm &&
-        ((ct == S.prev_ct && cm == S.prev_cm) || (float)cm * adu <= tol)) {
-      S.done = true; S.a0 = ct; S.b0 = ct + cm;
-      return;
-    }
-  } else {
-    fpos = ct >= k;                            // ct == k here means cm > 0: F > 0
-  }
-  S.prev_ct = ct; S.prev_cm = cm;
-  if (fpos) { S.lo_o = S.off; S.lo_a = S.piv + S.off; } else { S.hi_o = S.off; S.hi_a = S.piv + S.off; }
-  // the common case: the piece's solution lies inside the bracket and near the pivot
-  const float cand = S.off + du;
-  if (have && m != cm && cand > S.lo_o && cand < S.hi_o && S.nnewt < 6 && fabsf(cand) <= 8.0f * wid) {
-    S.gallop = 0; S.nnewt++; S.off = cand;
-    return;
-  }
-  S = nt_step_slow(S, ct, cm, m, du, have, fpos, wid, tol);
 }
 
 // threads per block, and the blocks per SM the register budget is set for: 24 warps of 80 registers with
@@ -285,12 +147,13 @@ __device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
 
 
 // G lanes per row (W == 1) or W warps per row (G == 32), E keys per lane (E / 4 a power of two).
-// KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1 only).
-template <int G, int E, int W, bool Q4, int KSEL, bool STAGED>
+// KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1, phi = x only).  MAG: phi(x) = x^2/2, keys |theta|.
+template <int G, int E, int W, bool Q4, int KSEL, bool STAGED, bool MAG>
 __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_kernel(const Problem P, const float zq) {
   extern __shared__ float4 nt_smem4[];
   static_assert(W == 1 || G == 32, "several warps per row: every lane of them belongs to the row");
   static_assert(!STAGED || W == 1, "the staging tile belongs to one warp");
+  static_assert(!MAG || KSEL == 0, "the magnitude mode starts from the moments");
   constexpr int BW = kNtWarps > W ? kNtWarps : W;   // warps per block
   constexpr int TEAMS = BW / W;                      // teams (of W warps) per block
   constexpr int R = W > 1 ? 1 : 32 / G;              // rows per team
@@ -303,8 +166,9 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   const int rl = lane / G, lig = lane % G;
   const long long row = row0 + rl;
   const bool row_ok = row < P.rows;
-  const float lam = P.lam, inv_lam = P.inv_lam, lam3 = P.lam3, wid = P.lam;
-  const float tol = (Q4 ? 3e-7f : 1e-6f) * wid;
+  const float lam = P.lam, inv_lam = P.inv_lam, lam3 = P.lam3;
+  float wid = P.lam;                           // phi = x: constant; phi even: follows tau
+  constexpr float kTolRel = Q4 ? 1e-7f : 3e-7f;
   float* smem = reinterpret_cast<float*>(nt_smem4);
   // shared memory: [STAGED: one tile of 32 E floats per warp] [W > 1: two buffers of W * 4 words per team]
   float* red = smem + (STAGED ? BW * 32 * E : 0) + team * (2 * W * 4);
@@ -358,7 +222,8 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   for (int c = 0; c < CH; ++c) {
     float x4[4];
     io.load_raw(c, x4);
-    d[4 * c] = x4[0]; d[4 * c + 1] = x4[1]; d[4 * c + 2] = x4[2]; d[4 * c + 3] = x4[3];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) d[4 * c + j] = MAG ? fabsf(x4[j]) : x4[j];
   }
   // a row that fills its lanes exactly has no slot to mark (and a -infinity in it shows in the sums below)
   const bool full = n == (STAGED ? G : G * W) * E;
@@ -373,14 +238,13 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
 
   // ---- start: bracket and first tau
   NtRow S;
-  S.done = false; S.noblock = false; S.repiv = false;
-  S.a0 = k; S.b0 = k; S.gallop = 0; S.nnewt = 0; S.prev_ct = -1; S.prev_cm = -1; S.edge_tried = false;
-  S.off = 0.0f; S.piv = 0.0f; S.lo_o = -INFINITY; S.hi_o = INFINITY;
+  nt_row_init(S, k);
   float lo = -FLT_MAX, hi = FLT_MAX;
   if (KSEL == 0) {
     // sums about the row's first key: mean and spread of the keys
-    const float x0 = __ldg(io.src);
+    const float x0 = MAG ? 0.0f : __ldg(io.src);
     float v[2] = {0.f, 0.f};
+    uint32_t nnz = 0;                          // phi even: keys above 0
     if (full) {
 #pragma unroll
       for (int i = 0; i < E; ++i) {
@@ -394,8 +258,11 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
         v[0] += dd; v[1] = fmaf(dd, dd, v[1]);
       }
     }
-    uint32_t none = 0;
-    team_allsum<G, W, 2>(v, none, red + (phase & 1) * (W * 4), wit, lane, bar);
+    if (MAG) {
+#pragma unroll
+      for (int i = 0; i < E; ++i) nnz += d[i] > 0.0f;
+    }
+    team_allsum<G, W, 2>(v, nnz, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!(v[1] < INFINITY)) {                  // overflow, an infinity or a NaN: look at the keys themselves
 #pragma unroll
@@ -404,12 +271,28 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     const float inv_n = 1.0f / (float)n;
     const float mean_d = v[0] * inv_n;
     const float sd = sqrtf(fmaxf(v[1] * inv_n - mean_d * mean_d, 0.0f));
-    if (k == n) {                              // everything is selected
-      S.piv = -FLT_MAX; S.off = -wid; S.done = true; S.noblock = true;
+    if (!MAG) {
+      if (k == n) {                            // everything is selected
+        S.piv = -FLT_MAX; S.off = -wid; S.done = true; S.noblock = true;
+      } else {
+        float tau0 = (x0 + mean_d) + zq * sd - (Q4 ? 0.75f : 0.5f) * lam;
+        if (!(fabsf(tau0) < FLT_MAX)) tau0 = x0;
+        S.piv = tau0;
+      }
     } else {
-      float tau0 = (x0 + mean_d) + zq * sd - (Q4 ? 0.75f : 0.5f) * lam;
-      if (!(fabsf(tau0) < FLT_MAX)) tau0 = x0;
-      S.piv = tau0;
+      if (k == n || (int)nnz < k) {
+        // the k-th largest |theta| is 0 (or everything is selected): every key is a top singleton
+        S.piv = 0.0f; S.off = 0.0f; S.done = true; S.noblock = true;
+      } else {
+        // zq: the upper k/(2n) quantile of N(0,1); the keys of a zero-mean row are its absolute values.
+        // About k keys lie above gamma + width/2 (q = 2) or gamma + 3 width/4 (q = 4).
+        const float t0 = zq * sqrtf(v[1] * inv_n);
+        float tau0 = Q4 ? t0 - 0.75f * lam * cbrtf(t0) : t0 / (1.0f + 0.5f * lam);
+        if (!(tau0 > 0.0f && tau0 < FLT_MAX)) tau0 = 0.5f * t0;
+        if (!(tau0 > 0.0f && tau0 < FLT_MAX)) tau0 = 1.0f;
+        S.piv = tau0;
+        lo = 0.0f; S.lo_o = -tau0;             // F(0) = n - k >= 0: every key is capped at tau = 0
+      }
     }
   } else {
     float m1 = -INFINITY, m2 = -INFINITY, m3 = -INFINITY, fin = 0.0f;
@@ -446,6 +329,9 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
 #pragma unroll 1
   for (; passes < kNtMaxPasses; ++passes) {
     if (__all_sync(0xffffffffu, S.done)) break;
+    if (MAG) wid = nt_width<Q4, true>(S.piv + S.off, lam);
+    // phi even: tau enters the width and the piece's equation itself, so a step is small against tau too
+    const float tol = kTolRel * (MAG ? fminf(wid, fmaxf(S.piv + S.off, 0.0f)) : wid);
     int ct0 = 0, ct1 = 0, cm0 = 0, cm1 = 0;
     float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, e0 = 0.f, e1 = 0.f;
     const float off = S.off;
@@ -475,15 +361,16 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     team_allsum<G, W, Q4 ? 3 : 1>(v, packed, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!S.done) {
-      nt_step<Q4>(S, (int)(packed & 0xffffu), (int)(packed >> 16), v[0], Q4 ? v[1] : 0.0f, Q4 ? v[Q4 ? 2 : 0] : 0.0f,
-                  k, lam, lam3, tol);
+      nt_step<Q4, MAG>(S, (int)(packed & 0xffffu), (int)(packed >> 16), v[0], Q4 ? v[1] : 0.0f,
+                       Q4 ? v[Q4 ? 2 : 0] : 0.0f, k, lam, lam3, wid, tol);
       if (S.repiv) {
 #pragma unroll
         for (int c = 0; c < CH; ++c) {
           float x4[4];
           io.load(c, x4);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) d[4 * c + j] = x4[j] - S.piv;
+          for (int j = 0; j < 4; ++j)      // (a slot past the row stays at -infinity)
+            d[4 * c + j] = ((MAG && x4[j] != -INFINITY) ? fabsf(x4[j]) : x4[j]) - S.piv;
           if ((c & 3) == 3) nt_fence();
         }
       }
@@ -496,6 +383,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   }
   if (S.b0 <= S.a0) { S.a0 = k; S.b0 = k; }
   const bool block = S.b0 > S.a0;
+  if (MAG) wid = nt_width<Q4, true>(S.piv + S.off, lam);   // of the point the last pass classified at
 
   // ---- row state.  Without a block the VJP classifies by key >= pivot: any value above the
   // (k+1)-th largest key and not above the k-th serves; tau + lambda/2 is one when lambda is
@@ -513,7 +401,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
         io.load(c, x4);
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-          if (d[4 * c + j] - S.off >= wid) cmin = fminf(cmin, x4[j]);
+          if (d[4 * c + j] - S.off >= wid) cmin = fminf(cmin, MAG ? fabsf(x4[j]) : x4[j]);
         if ((c & 3) == 3) nt_fence();
       }
       cmin = team_gmin<G>(cmin);
@@ -537,8 +425,9 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     P.state_out[row] = st;
   }
 
-  // ---- dual map y = rho(clamp(x - tau)), in the order the keys were read
-  {
+  // ---- dual map y = rho(clamp(key - tau)), in the order the keys were read.  phi even: a top singleton
+  // is its own minimiser vtop(key) (stationarity rho(key - v) = v), and the sign of theta comes back
+  if (!MAG) {
     const float shift = -S.off * inv_lam;
     const bool times_x = P.mode == TK_TOPK;
 #pragma unroll
@@ -557,6 +446,25 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       }
       io.store(c, y);
       if (times_x && (c & 3) == 3) nt_fence();
+    }
+  } else {
+    Math M = make_math(P);
+    M.q4 = Q4; M.mag = true; M.gen = false;
+    const float off = S.off;
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+      float x4[4], y[4];
+      io.load(c, x4);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float t = d[4 * c + j] - off;
+        float v = 0.0f;
+        if (t >= wid) v = M.vtop(fabsf(x4[j]));
+        else if (t > 0.0f) v = M.rho(t);
+        y[j] = signbit(x4[j]) ? -v : v;
+      }
+      io.store(c, y);
+      if ((c & 3) == 3) nt_fence();
     }
   }
   if (STAGED) {
@@ -592,22 +500,12 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   }
 }
 
-// z with P(N(0,1) > z) = tail, by bisection on erfc (a starting guess for the iteration: 1e-6 is plenty)
-float upper_normal_quantile(double tail) {
-  double lo = -8.0, hi = 8.0;
-  for (int i = 0; i < 28; ++i) {
-    const double mid = 0.5 * (lo + hi);
-    if (0.5 * erfc(mid * 0.70710678118654752440) > tail) lo = mid; else hi = mid;
-  }
-  return (float)(0.5 * (lo + hi));
-}
-
-template <int G, int E, int W, bool Q4, int KSEL, bool STAGED>
+template <int G, int E, int W, bool Q4, int KSEL, bool STAGED, bool MAG>
 cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
   constexpr int BW = kNtWarps > W ? kNtWarps : W;
   constexpr int TEAMS = BW / W;
   constexpr int smem = (STAGED ? BW * 32 * E * (int)sizeof(float) : 0) + (W > 1 ? TEAMS * 2 * W * 4 * (int)sizeof(float) : 0);
-  auto kern = tk_newton_kernel<G, E, W, Q4, KSEL, STAGED>;
+  auto kern = tk_newton_kernel<G, E, W, Q4, KSEL, STAGED, MAG>;
   if (smem > 48 * 1024) {
     static bool configured[64];
     int dev = 0;
@@ -625,28 +523,33 @@ cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
-// KS: the shape also has the variants that track the k + 1 largest keys (k <= 2)
+// KS: the shape also has the variants that track the k + 1 largest keys (k <= 2, phi = x)
 template <int G, int E, int W, bool KS, bool STAGED>
 cudaError_t nt_launch_q(const Problem& P, float zq, cudaStream_t stream) {
   const bool q4 = P.q4 != 0;
+  if (P.mode == TK_TOPKMAG)
+    return q4 ? nt_launch<G, E, W, true, 0, STAGED, true>(P, zq, stream)
+              : nt_launch<G, E, W, false, 0, STAGED, true>(P, zq, stream);
   if (KS && P.k == 1)
-    return q4 ? nt_launch<G, E, W, true, KS ? 1 : 0, STAGED>(P, zq, stream)
-              : nt_launch<G, E, W, false, KS ? 1 : 0, STAGED>(P, zq, stream);
+    return q4 ? nt_launch<G, E, W, true, KS ? 1 : 0, STAGED, false>(P, zq, stream)
+              : nt_launch<G, E, W, false, KS ? 1 : 0, STAGED, false>(P, zq, stream);
   if (KS && P.k == 2)
-    return q4 ? nt_launch<G, E, W, true, KS ? 2 : 0, STAGED>(P, zq, stream)
-              : nt_launch<G, E, W, false, KS ? 2 : 0, STAGED>(P, zq, stream);
-  return q4 ? nt_launch<G, E, W, true, 0, STAGED>(P, zq, stream) : nt_launch<G, E, W, false, 0, STAGED>(P, zq, stream);
+    return q4 ? nt_launch<G, E, W, true, KS ? 2 : 0, STAGED, false>(P, zq, stream)
+              : nt_launch<G, E, W, false, KS ? 2 : 0, STAGED, false>(P, zq, stream);
+  return q4 ? nt_launch<G, E, W, true, 0, STAGED, false>(P, zq, stream)
+            : nt_launch<G, E, W, false, 0, STAGED, false>(P, zq, stream);
 }
 
 }  // namespace
 
 int newton_max_n() { return 32768; }
 
-// Forward pass of TK_MASK / TK_TOPK with p = 2 or 4/3, rows of up to newton_max_n() elements,
-// no permutation output.
+// Forward pass with p = 2 or 4/3, rows of up to newton_max_n() elements, no permutation output.
 cudaError_t launch_newton(const Problem& P, cudaStream_t stream) {
   const int n = P.n;
-  const float zq = upper_normal_quantile(((double)P.k - 0.5) / (double)n);
+  // phi even: the keys are absolute values, k of n lie above the upper k/(2n) quantile of a zero-mean row
+  const double tail = ((double)P.k - 0.5) / (double)n;
+  const float zq = upper_normal_quantile(P.mode == TK_TOPKMAG ? 0.5 * tail : tail);
   // 32 keys per lane (more lanes per row and more rows in flight beat longer register rows); one or
   // two lanes per row go through the staging tile
   if (n <= 8) return nt_launch_q<1, 8, 1, true, true>(P, zq, stream);
