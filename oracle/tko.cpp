@@ -28,6 +28,12 @@
 //      even adjacent-pair constraints                   (Algorithm 1 and
 //      App. A.8), fixed number of sweeps.
 //
+//   8. General sorted w (Sec. 3, LP forms of sort and rank over the
+//      permutahedron P(w); Sec. 4, the relaxed operator for any w): tko_fwd_w /
+//      tko_vjp_w run steps 1, 3, 5, 6 with phi(x) = x and the caller's
+//      non-increasing w in place of 1_k; every pooled block is solved member by
+//      member (closed form for p = 2).
+//
 // Regulariser: R(y) = (lambda/p) sum |y_i|^p (the form used in the paper's
 // example after the PAV paragraph, in its Figure 3 and in its experiments),
 // hence r*(t) = |t|^q / (q lambda^(q-1)), q = p/(p-1), and
@@ -495,6 +501,148 @@ int tko_dykstra(const float* theta, int64_t rows, int64_t n, int64_t k, double p
         if (mode == TOPK) val *= (double)x[j];
         yo[j] = val;
         if (v_out) v_out[r * n + i] = vi;
+      }
+    }
+  }
+  return 0;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------- general sorted w
+// Relaxed linear maximisation over the permutahedron P(w) (Sec. 4 with phi(x) = x):
+//   y_R(x, w) = argmax_{y in P(w)} <x, y> - R(y) = grad R*(x - u*),   u* = v*_{sigma^-1},
+//   v* = argmin_{v_1 >= .. >= v_n} sum_i r*(s_i - v_i) + w_i v_i       (Prop. 5),
+// w_1 >= .. >= w_n any real numbers.  With w = 1_k this is the relaxed top-k mask; with
+// w = rho = (n, .., 1) and x -> -x the relaxed rank; with x = rho and w = sort(x) the relaxed sort
+// (Sec. 3, LP forms).
+namespace {
+
+struct WBlock {
+  int64_t lo, hi;
+  double gamma;
+};
+
+// d/dgamma of sum_{i in [lo,hi)} r*(s_i - gamma) + w_i gamma = sum -rho(s_i - gamma) + w_i
+double pooled_derivative_w(const Params& P, const double* s, const double* w, int64_t lo, int64_t hi,
+                           double gamma) {
+  double acc = 0.0;
+  for (int64_t i = lo; i < hi; ++i) acc += -rho(P, s[i] - gamma) + w[i];
+  return acc;
+}
+
+// Minimiser of the pooled objective: the derivative is increasing in gamma; each term vanishes at
+// s_i - rho^-1(w_i), so the root lies between the smallest and the largest of those.
+double solve_block_w(const Params& P, const double* s, const double* w, int64_t lo, int64_t hi) {
+  if (P.q_is_2) {
+    double ss = 0.0, ww = 0.0;
+    for (int64_t i = lo; i < hi; ++i) { ss += s[i]; ww += w[i]; }
+    return (ss - P.lambda * ww) / (double)(hi - lo);
+  }
+  double a = std::numeric_limits<double>::infinity(), b = -a;
+  for (int64_t i = lo; i < hi; ++i) {
+    double z = s[i] - rho_inv(P, w[i]);
+    a = std::min(a, z); b = std::max(b, z);
+  }
+  if (hi - lo == 1) return a;
+  for (int it = 0; it < 400; ++it) {
+    double m = 0.5 * (a + b);
+    if (m <= a || m >= b) break;
+    if (pooled_derivative_w(P, s, w, lo, hi, m) > 0.0) b = m; else a = m;
+  }
+  return 0.5 * (a + b);
+}
+
+// Pool adjacent violators (App. B.2) for general w: the same stack of blocks, merge while the
+// earlier of the two top blocks has a strictly smaller value, re-solve after each merge.
+void pav_w(const Params& P, const double* s, const double* w, int64_t n, std::vector<WBlock>& blocks) {
+  blocks.clear();
+  for (int64_t i = 0; i < n; ++i) {
+    WBlock b{i, i + 1, solve_block_w(P, s, w, i, i + 1)};
+    blocks.push_back(b);
+    while (blocks.size() >= 2) {
+      WBlock& prev = blocks[blocks.size() - 2];
+      WBlock& last = blocks[blocks.size() - 1];
+      if (!(prev.gamma < last.gamma)) break;
+      prev.hi = last.hi;
+      blocks.pop_back();
+      WBlock& merged = blocks.back();
+      merged.gamma = solve_block_w(P, s, w, merged.lo, merged.hi);
+    }
+  }
+}
+
+int check_args_w(int64_t rows, int64_t n, double p, double lambda, const double* w, int64_t w_rows) {
+  if (rows < 0 || n < 1 || !(p > 1.0) || !(lambda > 0.0) || w == nullptr) return 1;
+  if (w_rows != 1 && w_rows != rows) return 1;
+  for (int64_t r = 0; r < w_rows; ++r)
+    for (int64_t i = 0; i + 1 < n; ++i)
+      if (!(w[r * n + i] >= w[r * n + i + 1])) return 1;     // must be sorted (Prop. 1: "if not, sort w")
+  return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+// out[r, :] = y_R(theta[r, :], w[r or 0, :]).  w: [w_rows * n] doubles, w_rows = 1 (shared) or rows,
+// every row non-increasing.  Optional outputs as in tko_fwd.
+int tko_fwd_w(const float* theta, const double* w, int64_t rows, int64_t n, int64_t w_rows, double p,
+              double lambda, double* out, int32_t* perm, double* v, int32_t* block_lo, int32_t* block_hi) {
+  if (check_args_w(rows, n, p, lambda, w, w_rows)) return 1;
+  const Params P = make_params(p, lambda, MASK);
+#pragma omp parallel
+  {
+    std::vector<int32_t> pm(n);
+    std::vector<double> s(n);
+    std::vector<WBlock> blocks;
+#pragma omp for schedule(dynamic, 4)
+    for (int64_t r = 0; r < rows; ++r) {
+      const float* x = theta + r * n;
+      const double* wr = w + (w_rows == 1 ? 0 : r) * n;
+      argsort_row(x, n, false, pm.data(), s.data());
+      pav_w(P, s.data(), wr, n, blocks);
+      for (const WBlock& b : blocks)
+        for (int64_t i = b.lo; i < b.hi; ++i) {
+          out[r * n + pm[i]] = rho(P, s[i] - b.gamma);
+          if (v) v[r * n + i] = b.gamma;
+          if (block_lo) block_lo[r * n + i] = (int32_t)b.lo;
+          if (block_hi) block_hi[r * n + i] = (int32_t)b.hi;
+        }
+      if (perm) std::copy(pm.begin(), pm.end(), perm + r * n);
+    }
+  }
+  return 0;
+}
+
+// grad_theta = J^T g of y_R(., w) at theta (Prop. 7 with phi(x) = x: D_B = sum_B rho', no w term),
+// chained through y^s_i = rho(s_i - gamma_B): o_j = rho'_j (g^s_j - A_B / D_B), 0 where D_B = 0.
+int tko_vjp_w(const float* theta, const double* w, const float* gout, int64_t rows, int64_t n,
+              int64_t w_rows, double p, double lambda, double* grad) {
+  if (check_args_w(rows, n, p, lambda, w, w_rows)) return 1;
+  const Params P = make_params(p, lambda, MASK);
+#pragma omp parallel
+  {
+    std::vector<int32_t> pm(n);
+    std::vector<double> s(n);
+    std::vector<WBlock> blocks;
+#pragma omp for schedule(dynamic, 4)
+    for (int64_t r = 0; r < rows; ++r) {
+      const float* x = theta + r * n;
+      const float* g = gout + r * n;
+      const double* wr = w + (w_rows == 1 ? 0 : r) * n;
+      argsort_row(x, n, false, pm.data(), s.data());
+      pav_w(P, s.data(), wr, n, blocks);
+      for (const WBlock& b : blocks) {
+        double D = 0.0, A = 0.0;
+        for (int64_t i = b.lo; i < b.hi; ++i) {
+          double d = drho(P, s[i] - b.gamma);
+          D += d; A += d * (double)g[pm[i]];
+        }
+        for (int64_t i = b.lo; i < b.hi; ++i) {
+          double d = drho(P, s[i] - b.gamma);
+          grad[r * n + pm[i]] = (D > 0.0) ? d * ((double)g[pm[i]] - A / D) : 0.0;
+        }
       }
     }
   }

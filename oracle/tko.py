@@ -59,7 +59,9 @@ def _load() -> ctypes.CDLL:
                             ctypes.c_int, ctypes.c_int, f64p]
     lib.tko_dykstra.argtypes = [f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double,
                                 ctypes.c_int, ctypes.c_int, ctypes.c_int, f64p, f64p]
-    for fn in (lib.tko_argsort, lib.tko_fwd, lib.tko_vjp, lib.tko_dykstra):
+    lib.tko_fwd_w.argtypes = [f32p, f64p, i64, i64, i64, ctypes.c_double, ctypes.c_double, f64p, i32p, f64p, i32p, i32p]
+    lib.tko_vjp_w.argtypes = [f32p, f64p, f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double, f64p]
+    for fn in (lib.tko_argsort, lib.tko_fwd, lib.tko_vjp, lib.tko_dykstra, lib.tko_fwd_w, lib.tko_vjp_w):
         fn.restype = ctypes.c_int
     _lib = lib
     return lib
@@ -163,6 +165,67 @@ def dykstra(theta, k: int, p: float, lam: float, mode: int = MASK, sweeps: int =
     if rc:
         raise ValueError("tko_dykstra: invalid argument")
     return (out, v) if return_v else out
+
+
+def _w64(w, rows: int, n: int) -> np.ndarray:
+    a = np.ascontiguousarray(np.asarray(w, dtype=np.float64))
+    if a.ndim == 1:
+        a = a[None, :]
+    if a.shape not in ((1, n), (rows, n)):
+        raise ValueError("w must be (n,), (1, n) or (rows, n)")
+    return a
+
+
+def fwd_w(theta, w, p: float, lam: float, details: bool = False):
+    """Relaxed linear maximisation over the permutahedron P(w) (Sec. 3 LP forms, Sec. 4 with
+    phi(x) = x): y_R(theta, w), w non-increasing (one vector for all rows, or one per row).
+    (rows, n) float64; details=True also returns perm, v, block_lo, block_hi."""
+    x = _f32(theta)
+    rows, n = x.shape
+    ww = _w64(w, rows, n)
+    out = np.empty((rows, n), np.float64)
+    perm = v = blo = bhi = None
+    if details:
+        perm = np.empty((rows, n), np.int32); v = np.empty((rows, n), np.float64)
+        blo = np.empty((rows, n), np.int32); bhi = np.empty((rows, n), np.int32)
+    rc = _load().tko_fwd_w(_ptr(x, ctypes.c_float), _ptr(ww, ctypes.c_double), rows, n, ww.shape[0], p, lam,
+                           _ptr(out, ctypes.c_double), _ptr(perm, ctypes.c_int32), _ptr(v, ctypes.c_double),
+                           _ptr(blo, ctypes.c_int32), _ptr(bhi, ctypes.c_int32))
+    if rc:
+        raise ValueError("tko_fwd_w: invalid argument (w must be sorted in non-increasing order)")
+    if details:
+        return out, {"perm": perm, "v": v, "block_lo": blo, "block_hi": bhi}
+    return out
+
+
+def vjp_w(theta, w, gout, p: float, lam: float) -> np.ndarray:
+    """J^T g of y_R(., w) at theta (gradient in theta only)."""
+    x = _f32(theta)
+    g = _f32(gout)
+    rows, n = x.shape
+    ww = _w64(w, rows, n)
+    grad = np.empty((rows, n), np.float64)
+    rc = _load().tko_vjp_w(_ptr(x, ctypes.c_float), _ptr(ww, ctypes.c_double), _ptr(g, ctypes.c_float), rows, n,
+                           ww.shape[0], p, lam, _ptr(grad, ctypes.c_double))
+    if rc:
+        raise ValueError("tko_vjp_w: invalid argument")
+    return grad
+
+
+def soft_rank(theta, p: float, lam: float) -> np.ndarray:
+    """Relaxed rank (Sec. 3: rank(x) = y(-x, rho), rho = (n, .., 1); rank 1 = largest value)."""
+    x = _f32(theta)
+    n = x.shape[1]
+    return fwd_w(-x, np.arange(n, 0, -1, dtype=np.float64), p, lam)
+
+
+def soft_sort(theta, p: float, lam: float) -> np.ndarray:
+    """Relaxed descending sort (Sec. 3: sort(x) = y(rho, x) = argmax over P(x) of <rho, y>)."""
+    x = _f32(theta)
+    rows, n = x.shape
+    w = -np.sort(-x.astype(np.float64), axis=1)
+    rho_v = np.tile(np.arange(n, 0, -1, dtype=np.float32), (rows, 1))
+    return fwd_w(rho_v, w, p, lam)
 
 
 def topk_loss(theta, target, k: int, p: float, lam: float):

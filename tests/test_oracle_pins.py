@@ -529,6 +529,126 @@ def test_dual_coordinate_ascent_first_updates_by_hand():
 
 
 # --------------------------------------------------------------------------
+# general sorted w: relaxed linear maximisation over the permutahedron P(w)
+# --------------------------------------------------------------------------
+def lmo_by_vertex_hull(x, w, p, lam):
+    """max over the convex hull of all permutations of w of <y, x> - R(y), y = a^T V with a in the simplex
+    (Sec. 3, definition of the permutahedron); no sort, no isotonic solve."""
+    import itertools
+    x = np.asarray(x, np.float64)
+    V = np.array(sorted(set(itertools.permutations([float(a) for a in w]))))
+    m = len(V)
+
+    def neg(a):
+        y = a @ V
+        return -(y @ x) + lam / p * np.sum(np.abs(y) ** p)
+
+    def grad(a):
+        y = a @ V
+        return V @ (-x + lam * np.sign(y) * np.abs(y) ** (p - 1.0))
+
+    best = None
+    for start in range(3):
+        a0 = np.random.default_rng(start).dirichlet(np.ones(m))
+        res = minimize(neg, a0, jac=grad, method="SLSQP", bounds=[(0, 1)] * m,
+                       constraints=[{"type": "eq", "fun": lambda a: a.sum() - 1.0, "jac": lambda a: np.ones(m)}],
+                       options={"ftol": 1e-15, "maxiter": 800})
+        if best is None or res.fun < best.fun:
+            best = res
+    return best.x @ V
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_w_equals_maximiser_over_vertex_hull(p):
+    rng = np.random.default_rng(23)
+    for w in ([3.0, 2.0, 1.0], [4.0, 3.0, 2.0, 1.0], [2.0 / 3, 1.0 / 3, 0.0], [1.0, 1.0, 0.5, 0.0],
+              [5.0, 4.0, 3.0, 2.0, 1.0], [2.0, 0.5, 0.5, -1.0]):
+        for lam in (0.4, 1.5):
+            x = (rng.standard_normal(len(w)) * 1.5).astype(np.float32)
+            ref = lmo_by_vertex_hull(x, w, p, lam)
+            y = tko.fwd_w(x, w, p, lam)[0]
+            assert np.max(np.abs(y - ref)) < 5e-5, (w, lam, y, ref)
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_w_reduces_to_the_mask_and_to_the_hard_operators(p):
+    x = random_rows(20, 12, 29, scale=2.0)
+    for k in (1, 4, 11):
+        w = np.r_[np.ones(k), np.zeros(12 - k)]
+        assert np.max(np.abs(tko.fwd_w(x, w, p, 0.7) - tko.fwd(x, k, p, 0.7, tko.MASK))) < 1e-10
+    # lambda -> 0: the linear maximisation oracle y(x, w) = w_rank(x) (Prop. 1), hence sort and rank (Sec. 3)
+    w = np.linspace(3.0, -1.0, 12)
+    perm, _ = tko.argsort(x, tko.MASK)
+    y = tko.fwd_w(x, w, p, 1e-7)
+    for r in range(x.shape[0]):
+        want = np.empty(12); want[perm[r]] = w
+        assert np.max(np.abs(y[r] - want)) < 1e-5
+    ranks = tko.soft_rank(x, p, 1e-7)
+    srt = tko.soft_sort(x, p, 1e-7)
+    for r in range(x.shape[0]):
+        hard_rank = np.empty(12); hard_rank[perm[r]] = np.arange(1, 13)
+        assert np.max(np.abs(ranks[r] - hard_rank)) < 1e-5
+        assert np.max(np.abs(srt[r] - np.sort(x[r].astype(np.float64))[::-1])) < 1e-5
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_w_output_lies_in_the_permutahedron_and_is_optimal(p):
+    """y in P(w): same total, and the l largest entries of y sum to at most w_1 + .. + w_l (majorisation);
+    no point of P(w) (random convex combinations of permutations of w) does better in <x, y> - R(y)."""
+    rng = np.random.default_rng(31)
+    n = 9
+    x = random_rows(12, n, 33, scale=1.5)
+    w = np.array([4.0, 3.5, 3.5, 2.0, 1.0, 1.0, 0.5, 0.0, -1.0])
+    for lam in (0.2, 1.0, 5.0):
+        y = tko.fwd_w(x, w, p, lam)
+        assert np.max(np.abs(y.sum(axis=1) - w.sum())) < 1e-9
+        ys = -np.sort(-y, axis=1)
+        assert np.all(np.cumsum(ys, axis=1) <= np.cumsum(w)[None, :] + 1e-9)
+        for r in range(x.shape[0]):
+            xr = x[r].astype(np.float64)
+            best = y[r] @ xr - lam / p * np.sum(np.abs(y[r]) ** p)
+            for _ in range(200):
+                a = rng.dirichlet(np.ones(6) * 0.5)
+                z = sum(ai * w[rng.permutation(n)] for ai in a)
+                assert z @ xr - lam / p * np.sum(np.abs(z) ** p) <= best + 1e-10
+            # and towards y itself from those points the objective increases (concavity: a local check)
+            z = 0.9 * y[r] + 0.1 * w[rng.permutation(n)]
+            assert z @ xr - lam / p * np.sum(np.abs(z) ** p) <= best + 1e-10
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_w_vjp_matches_finite_differences(p):
+    rng = np.random.default_rng(37)
+    n = 7
+    w = np.array([3.0, 2.5, 2.0, 2.0, 1.0, 0.2, 0.0])
+    for lam in (0.5, 2.0):
+        x = (rng.standard_normal(n) * 1.2).astype(np.float32)
+        J = np.empty((n, n))
+        h = 1e-3
+        for j in range(n):
+            xp = x.copy(); xm = x.copy()
+            xp[j] = np.float32(x[j] + h); xm[j] = np.float32(x[j] - h)
+            J[:, j] = (tko.fwd_w(xp, w, p, lam)[0] - tko.fwd_w(xm, w, p, lam)[0]) / (float(xp[j]) - float(xm[j]))
+        Jv = np.empty((n, n))
+        for i in range(n):
+            e = np.zeros(n, np.float32); e[i] = 1.0
+            Jv[i, :] = tko.vjp_w(x, w, e, p, lam)[0]
+        # away from the kinks where a block forms or splits (a perturbation of 1e-3 must not change the partition)
+        _, d0 = tko.fwd_w(x, w, p, lam, details=True)
+        same = True
+        for j in range(n):
+            for sgn in (-1, 1):
+                xq = x.copy(); xq[j] = np.float32(x[j] + sgn * h)
+                _, d1 = tko.fwd_w(xq, w, p, lam, details=True)
+                same &= np.array_equal(d0["block_lo"], d1["block_lo"]) and np.array_equal(d0["perm"], d1["perm"])
+        if same:
+            assert np.max(np.abs(J - Jv)) < 2e-5, (lam, J, Jv)
+    # w sorted is required
+    with pytest.raises(ValueError):
+        tko.fwd_w(np.zeros((1, 3), np.float32), [1.0, 2.0, 0.0], 2.0, 1.0)
+
+
+# --------------------------------------------------------------------------
 # VJP
 # --------------------------------------------------------------------------
 def jacobian_fd(x, k, p, lam, mode, h=1e-3):
