@@ -183,6 +183,25 @@ tk_status tk_vjp_cols(const float *theta, const float *grad_out, int64_t n, int6
                       int64_t k, double p, double lambda, int mode, float *grad_theta,
                       const tk_opts *opts, tk_stream stream);
 
+/* Relaxed linear maximisation over the permutahedron P(w) of any sorted vector w (Sec. 3, LP forms
+ * of sort and rank; Sec. 4, the relaxed operator with phi(x) = x; Prop. 5 for its reduction to
+ * isotonic optimisation, solved here by pool-adjacent-violators with many blocks, App. B.2):
+ *   out[r, :] = argmax_{y in P(w_r)} <theta[r, :], y> - R(y).
+ * w_r = (1,..,1,0,..,0) gives the relaxed top-k mask of tk_fwd; w = (n, n-1, .., 1) applied to
+ * -x gives the relaxed rank of x (rank 1 = largest value); theta = (n, .., 1) with w_r = x_r
+ * sorted gives the relaxed descending sort of x_r.
+ * theta, out: device [rows*n] fp32.  w: device fp32, [n] shared by every row (w_rows = 1) or
+ * [rows*n] (w_rows = rows); every row of w must be in non-increasing order (it is not checked:
+ * an unsorted w gives an unspecified result).  p = 2 or p = 4/3, n <= 2048 (else
+ * TK_ERR_UNSUPPORTED).  opts may carry status_out; the other fields must be unset.
+ * tk_vjp_w: grad_theta[r, :] = J(theta[r, :])^T grad_out[r, :], the Jacobian of Prop. 7 (block
+ * diagonal over the pooled blocks) in theta, w held fixed; the row is sorted and solved again.  */
+tk_status tk_fwd_w(const float *theta, const float *w, int64_t rows, int64_t n, int64_t w_rows, double p,
+                   double lambda, float *out, const tk_opts *opts, tk_stream stream);
+tk_status tk_vjp_w(const float *theta, const float *w, const float *grad_out, int64_t rows, int64_t n,
+                   int64_t w_rows, double p, double lambda, float *grad_theta, const tk_opts *opts,
+                   tk_stream stream);
+
 /* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
  * perm_out[i] = index of the i-th largest key (theta, or |theta| for
  * TK_TOPKMAG), equal keys in ascending index, -0 == +0.  sorted_out (may be

@@ -35,6 +35,9 @@ cudaError_t launch_hard(const float* theta, const int32_t* perm, float* out, lon
 // [n, cols] with leading dimension <-> contiguous [cols, n] (tk_transpose.cu)
 cudaError_t launch_transpose(const float* in, long long in_rows, long long in_cols, long long in_ld, float* out,
                              long long out_ld, cudaStream_t stream);
+// relaxed operator over the permutahedron of any sorted w (tk_w.cu)
+int w_max_n();
+cudaError_t launch_w(const Problem& P, const float* w, long long w_rows, cudaStream_t stream);
 // VJP from saved row state (tk_vjp_state.cu)
 cudaError_t launch_vjp_state(const Problem& P, cudaStream_t stream);
 cudaError_t launch_vjp_state_long(const Problem& P, void* scratch, cudaStream_t stream);
@@ -63,16 +66,18 @@ inline cudaError_t launch_on_chip(const Problem& P, cudaStream_t stream) {
 }
 
 // q = p/(p-1): 2 and 4 (p = 2, p = 4/3) have closed-form block solves and run everywhere.  Any
-// other 1 < p <= 1.5 (q >= 3) is *qm1 = q - 1 > 0: forward pass by the sort-free solver, VJP from
-// saved state.  Not supported: q < 2 (p > 2: rho' unbounded at 0) and 2 < q < 3 (rho'' unbounded at
-// 0: an fp32 key difference cannot carry the VJP of a barely pooled element to 1e-5).
+// other 1 < p < 2 (q > 2) is *qm1 = q - 1 > 0: forward pass by the sort-free solver, VJP from
+// saved state for q >= 3.  Not supported: q < 2 (p > 2: rho' unbounded at 0); for 2 < q < 3
+// (1.5 < p < 2) rho'' is unbounded at 0 and an fp32 key difference cannot carry the VJP of a barely
+// pooled element to 1e-5, so only the forward pass (and the loss, whose gradient is the forward
+// output) is served there (vjp_supported).
 tk_status classify_p(double p, int* q4, double* qm1) {
   *q4 = 0; *qm1 = 0.0;
   if (!(p > 1.0) || !isfinite(p)) return TK_ERR_INVALID_ARG;
   double q = p / (p - 1.0);
   if (fabs(q - 2.0) <= 1e-6) return TK_OK;
   if (fabs(q - 4.0) <= 1e-6) { *q4 = 1; return TK_OK; }
-  if (!(q >= 3.0 - 1e-9) || q > 64.0) return TK_ERR_UNSUPPORTED;
+  if (!(q > 2.0) || q > 64.0) return TK_ERR_UNSUPPORTED;
   *qm1 = q - 1.0;
   return TK_OK;
 }
@@ -83,7 +88,7 @@ tk_status check_common(const void* theta, int64_t rows, int64_t n, int64_t k, do
   if (mode < TK_MASK || mode > TK_TOPKMAG) return TK_ERR_INVALID_ARG;
   if (!(lambda > 0.0) || !isfinite(lambda)) return TK_ERR_INVALID_ARG;
   tk_status s = classify_p(p, q4, qm1);
-  if (s == TK_OK && *qm1 > 0.0 && (mode == TK_TOPKMAG || n > kMaxOnChipN)) s = TK_ERR_UNSUPPORTED;
+  if (s == TK_OK && *qm1 > 0.0 && n > kMaxOnChipN) s = TK_ERR_UNSUPPORTED;
   if (s != TK_OK) return s;
   if (rows > 0 && theta == nullptr) return TK_ERR_INVALID_ARG;
   if (n > 0x7fffffff || rows > 0x7fffffffLL) return TK_ERR_UNSUPPORTED;
@@ -107,6 +112,9 @@ tk_status check_workspace(const tk_opts* opts, int64_t rows, int64_t n) {
   if (opts->workspace_bytes < tk::long_workspace_bytes(rows, (int)n)) return TK_ERR_WORKSPACE;
   return TK_OK;
 }
+
+// derivatives are served for q = 2, 4 and any q >= 3
+bool vjp_supported(double qm1) { return qm1 == 0.0 || qm1 >= 2.0 - 1e-9; }
 
 void fill(tk::Problem& P, const float* theta, int64_t rows, int64_t n, int64_t k, int q4,
           double qm1, double lambda, int mode) {
@@ -157,7 +165,7 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
     // for it): the sort-free solver.  No permutation output either way.
     if (solver == TK_SOLVER_PAV || solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
     if (opts && opts->perm_out) return TK_ERR_UNSUPPORTED;
-    if (n > tk::kMaxGeneralSortedN) solver = TK_SOLVER_THRESHOLD;
+    if (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG) solver = TK_SOLVER_THRESHOLD;
   }
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
@@ -252,8 +260,10 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
   if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
-  // general p: from saved state, or recomputed by the sorting kernel for rows of up to 128 elements
-  if (qm1 > 0.0 && !(opts && opts->state_out) && n > tk::kMaxGeneralSortedN) return TK_ERR_UNSUPPORTED;
+  if (!vjp_supported(qm1)) return TK_ERR_UNSUPPORTED;
+  // general p: from saved state, or recomputed by the sorting kernel for rows of up to 128 elements (phi = x)
+  if (qm1 > 0.0 && !(opts && opts->state_out) && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG))
+    return TK_ERR_UNSUPPORTED;
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.gout = grad_out;
@@ -297,7 +307,7 @@ tk_status tk_jvp(const float* theta, const float* tangent, int64_t rows, int64_t
   if (s != TK_OK) return s;
   if (rows == 0) return TK_OK;
   if (tangent == nullptr || out_tangent == nullptr) return TK_ERR_INVALID_ARG;
-  if (!(opts && opts->state_out)) return TK_ERR_UNSUPPORTED;       // from the forward pass's row state only
+  if (!(opts && opts->state_out) || !vjp_supported(qm1)) return TK_ERR_UNSUPPORTED;   // from the forward pass's row state only
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.gout = tangent;
@@ -398,6 +408,39 @@ tk_status tk_vjp_cols(const float* theta, const float* grad_out, int64_t n, int6
   s = tk_vjp(slab[0], slab[1], cols, n, k, p, lambda, mode, slab[2], &inner, stream);
   if (s != TK_OK) return s;
   return tk::launch_transpose(slab[2], cols, n, n, grad_theta, ld, st) == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+// ---- any sorted w: relaxed linear maximisation over the permutahedron P(w)
+static tk_status run_w(const float* theta, const float* w, const float* grad_out, int64_t rows, int64_t n,
+                       int64_t w_rows, double p, double lambda, float* out, const tk_opts* opts, tk_stream stream,
+                       int what) {
+  int q4 = 0;
+  double qm1 = 0.0;
+  tk_status s = check_common(theta, rows, n, 1, p, lambda, TK_MASK, &q4, &qm1);
+  if (s != TK_OK) return s;
+  if (w_rows != 1 && w_rows != rows) return TK_ERR_INVALID_ARG;
+  if (qm1 > 0.0 || n > tk::w_max_n() || (opts && (opts->flags || opts->perm_out))) return TK_ERR_UNSUPPORTED;
+  if (rows == 0) return TK_OK;
+  if (w == nullptr || out == nullptr || (what == tk::W_VJP && grad_out == nullptr)) return TK_ERR_INVALID_ARG;
+  tk::Problem P;
+  fill(P, theta, rows, n, 1, q4, 0.0, lambda, TK_MASK);
+  P.out = out;
+  P.gout = grad_out;
+  P.what = what;
+  if (opts) P.status = opts->status_out;
+  cudaError_t e = tk::launch_w(P, w, w_rows, (cudaStream_t)stream);
+  return e == cudaSuccess ? TK_OK : TK_ERR_CUDA;
+}
+
+tk_status tk_fwd_w(const float* theta, const float* w, int64_t rows, int64_t n, int64_t w_rows, double p,
+                   double lambda, float* out, const tk_opts* opts, tk_stream stream) {
+  return run_w(theta, w, nullptr, rows, n, w_rows, p, lambda, out, opts, stream, tk::W_FWD);
+}
+
+tk_status tk_vjp_w(const float* theta, const float* w, const float* grad_out, int64_t rows, int64_t n,
+                   int64_t w_rows, double p, double lambda, float* grad_theta, const tk_opts* opts,
+                   tk_stream stream) {
+  return run_w(theta, w, grad_out, rows, n, w_rows, p, lambda, grad_theta, opts, stream, tk::W_VJP);
 }
 
 tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int32_t* perm_out,

@@ -126,11 +126,24 @@ struct Math {
     if (gen) return qm1 * powf(a, qm1 - 1.0f) * inv_lam;
     return q4 ? 3.0f * a * a * inv_lam : inv_lam;
   }
-  // z >= 0 with z^3 + lam z = s (s >= 0): z = (s - v)/lam at the minimiser v of
-  // h(v) = v^2/2 + (s - v)^4 / (4 lam^3).  Newton from the right of the root on
-  // a convex increasing function: monotone convergence.
+  // z >= 0 with z^(q-1) + lam z = s (s >= 0): z = (s - v)/lam at the minimiser v of
+  // h(v) = v^2/2 + r*(s - v), i.e. the point where rho(s - v) = v.  Newton from the right of the
+  // root on a convex increasing function (q >= 3; for q < 3 it is concave and the same start is
+  // left of the root after one step): monotone convergence.
   __device__ __forceinline__ float cubic_z(float s) const {
     if (!(s > 0.0f)) return 0.0f;
+    if (gen) {
+      float z = fminf(powf(s, 1.0f / qm1), s * inv_lam);
+#pragma unroll 1
+      for (int it = 0; it < 24; ++it) {
+        const float zp = powf(z, qm1 - 1.0f);
+        const float f = fmaf(zp + lam, z, -s);
+        const float dz = f / fmaf(qm1, zp, lam);
+        z = fmaxf(z - dz, 0.0f);
+        if (fabsf(dz) <= 6e-8f * z) break;
+      }
+      return z;
+    }
     float z = fminf(cbrtf(s), s * inv_lam);
 #pragma unroll 1
     for (int it = 0; it < 16; ++it) {
@@ -144,24 +157,25 @@ struct Math {
   // Minimiser of h_i for a rank < k (w_i = 1) singleton with key s.
   __device__ __forceinline__ float vtop(float s) const {
     if (!mag) return s - lam;
-    if (!q4) return s / (1.0f + lam);
+    if (!q4 && !gen) return s / (1.0f + lam);
     float z = cubic_z(s);
     float lz = lam * z;
-    return (lz < 0.5f * s) ? s - lz : z * z * z;
+    return (lz < 0.5f * s) ? s - lz : (gen ? powf(z, qm1) : z * z * z);
   }
   // Key distance above gamma = tau at which a rank < k element stops being
   // pooled: rho(width) = phi'(tau).
   __device__ __forceinline__ float width(float tau) const {
     if (!mag) return lam;
     float t = fmaxf(tau, 0.0f);
+    if (gen) return lam * powf(t, 1.0f / qm1);
     return q4 ? lam * cbrtf(t) : lam * t;
   }
   // d/ds of the output of a top singleton (phi even): rho' / (rho' + 1).
   __device__ __forceinline__ float top_slope(float s) const {
     if (!mag) return 0.0f;
-    if (!q4) return 1.0f / (1.0f + lam);
-    float z = cubic_z(s);              // z = (s - v)/lam, rho' = 3 z^2 / lam
-    float r = 3.0f * z * z * inv_lam;
+    if (!q4 && !gen) return 1.0f / (1.0f + lam);
+    float z = cubic_z(s);              // z = (s - v)/lam, rho' = (q-1) z^(q-2) / lam
+    float r = gen ? qm1 * powf(z, qm1 - 1.0f) * inv_lam : 3.0f * z * z * inv_lam;
     return r / (r + 1.0f);
   }
 };

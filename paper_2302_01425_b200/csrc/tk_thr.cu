@@ -1,4 +1,6 @@
-// tk_thr.cu -- the exact forward pass without a sort (solver = TK_SOLVER_THRESHOLD).
+// tk_thr.cu -- the exact forward pass without a sort, one thread block per row: the solver for a general
+// p (1 < p < 2 other than 4/3).  p = 2 and p = 4/3 take the register-resident team kernel of
+// tk_newton.cu; the closed-form variants of this kernel (QM = 0, 1) are kept as templates but not launched.
 //
 // With w = 1_k the isotonic solution has at most one pooled block, whose value
 // gamma is the root of the non-increasing threshold function
@@ -238,7 +240,8 @@ __global__ void __launch_bounds__(MAXT) tk_thr_kernel(const Problem P) {
       if (S.cm > 0 && m >= 1) {
         if (GEN) {
           // Newton on sum rho(t_i - du) = m about du = 0 (the sums are taken at the current gamma)
-          du = S.s2 > 0.0f ? (S.s1 - (float)m) / S.s2 : 0.0f;
+          // phi even: sum rho(t_i - du) = m (gamma + du)
+          du = mag ? (S.s1 - (float)m * gam) / (S.s2 + (float)m) : (S.s2 > 0.0f ? (S.s1 - (float)m) / S.s2 : 0.0f);
         } else if (M.q4) {
           du = solve_piece_cubic(mag, P.lam3, gam, (float)S.cm, (float)m, S.s1, S.s2, S.s3);
         } else {
@@ -350,14 +353,14 @@ cudaError_t launch_thr(const Problem& P0, cudaStream_t stream) {
   const int E = N >= 4096 ? 16 : (N >= 1024 ? 8 : 4);
   const int T = N / E;
   const dim3 grid((unsigned)P.rows);
-  const bool q4 = P.q4 != 0, mag = P.mode == TK_TOPKMAG, gen = P.qm1 > 0.0f;
+  // p = 2 and p = 4/3 are served by the register-resident team kernel (tk_newton.cu); this block-per-row
+  // solver is launched for a general p only
+  if (!(P.qm1 > 0.0f)) return cudaErrorInvalidValue;
+  const bool mag = P.mode == TK_TOPKMAG;
 #define TK_THR_LAUNCH(EE, MT)                                                        \
   do {                                                                               \
-    if (gen) tk_thr_kernel<EE, MT, 2, false><<<grid, T, 0, stream>>>(P);              \
-    else if (q4 && mag) tk_thr_kernel<EE, MT, 1, true><<<grid, T, 0, stream>>>(P);    \
-    else if (q4) tk_thr_kernel<EE, MT, 1, false><<<grid, T, 0, stream>>>(P);          \
-    else if (mag) tk_thr_kernel<EE, MT, 0, true><<<grid, T, 0, stream>>>(P);          \
-    else tk_thr_kernel<EE, MT, 0, false><<<grid, T, 0, stream>>>(P);                  \
+    if (mag) tk_thr_kernel<EE, MT, 2, true><<<grid, T, 0, stream>>>(P);               \
+    else tk_thr_kernel<EE, MT, 2, false><<<grid, T, 0, stream>>>(P);                  \
   } while (0)
   switch (E) {
     case 4: TK_THR_LAUNCH(4, 128); break;

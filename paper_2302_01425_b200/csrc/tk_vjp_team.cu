@@ -181,8 +181,8 @@ cudaError_t vt_launch_mode(const Problem& P, cudaStream_t stream) {
       return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPK>(P, stream)
                      : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPK>(P, stream) : vt_launch<G, E, W, 2, TK_TOPK>(P, stream));
     default:
-      if (qm == 2) return cudaErrorInvalidValue;               // the magnitude mode has p = 2 and p = 4/3 only
-      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPKMAG>(P, stream) : vt_launch<G, E, W, 1, TK_TOPKMAG>(P, stream);
+      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPKMAG>(P, stream)
+                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPKMAG>(P, stream) : vt_launch<G, E, W, 2, TK_TOPKMAG>(P, stream));
   }
 }
 

@@ -16,7 +16,6 @@ Tolerances (written here once, used by every GPU test):
 """
 from __future__ import annotations
 
-import os
 
 import numpy as np
 import torch
@@ -44,7 +43,7 @@ def check_disputed(count: int, rows: int, label: str, general_p: bool = False):
     cap = rows if general_p else max(2, int(1e-3 * rows))
     if count:
         print(f"{label}: {count} of {rows} rows with a near-tie at the block edge (cap {cap})")
-    assert count <= cap or os.environ.get("TK_NO_CAP"), f"{label}: {count} disputed rows of {rows} (cap {cap})"
+    assert count <= cap, f"{label}: {count} disputed rows of {rows} (cap {cap})"
 
 
 def oracle_blocks(det, k):

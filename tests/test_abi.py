@@ -71,8 +71,9 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert fwd(4, 8, 2, 2.0, float("nan"), 0) == b.TK_ERR_INVALID_ARG
     assert fwd(4, 8, 2, 2.0, 1.0, 3) == b.TK_ERR_INVALID_ARG        # mode
     assert fwd(4, 8, 2, 3.0, 1.0, 0) == b.TK_ERR_UNSUPPORTED        # q = 1.5 < 2
-    assert fwd(4, 8, 2, 1.8, 1.0, 0) == b.TK_ERR_UNSUPPORTED        # 2 < q < 3
-    assert fwd(4, 8, 2, 1.5, 1.0, 2) == b.TK_ERR_UNSUPPORTED        # q = 3 with the magnitude mode
+    assert fwd(4, 8, 2, 1.01, 1.0, 0) == b.TK_ERR_UNSUPPORTED       # q = 101 > 64
+    assert lib.tk_vjp(fake, fake, 4, 8, 2, 1.8, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED   # 2 < q < 3: forward pass only
+    assert lib.tk_jvp(fake, fake, 4, 8, 2, 1.8, 1.0, 0, fake, None, None) in (b.TK_ERR_UNSUPPORTED, b.TK_ERR_INVALID_ARG)
     assert fwd(1, 20000, 2, 1.5, 1.0, 0) == b.TK_ERR_UNSUPPORTED    # q = 3 on a row held in global memory
     assert lib.tk_vjp(fake, fake, 4, 200, 2, 1.5, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED  # q = 3, n > 128, no saved state
     assert fwd(4, 8, 2, 2.0, 1.0, 0, theta=None) == b.TK_ERR_INVALID_ARG
@@ -85,6 +86,91 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     o = b.TkOpts()
     o.solver = 7
     assert lib.tk_fwd_ex(fake, 4, 8, 2, 2.0, 1.0, 0, fake, ctypes.byref(o), None) == b.TK_ERR_INVALID_ARG
+
+
+def test_general_w_arguments_are_rejected_on_the_host(lib):
+    from paper_2302_01425_b200 import binding as b
+    fake = ctypes.c_void_p(256)
+    fw = lambda rows, n, w_rows, p, lam, theta=fake, w=fake, out=fake: lib.tk_fwd_w(
+        theta, w, rows, n, w_rows, p, lam, out, None, None)
+    assert fw(4, 0, 1, 2.0, 1.0) == b.TK_ERR_INVALID_ARG
+    assert fw(-1, 8, 1, 2.0, 1.0) == b.TK_ERR_INVALID_ARG
+    assert fw(4, 8, 3, 2.0, 1.0) == b.TK_ERR_INVALID_ARG            # w_rows is 1 or rows
+    assert fw(4, 8, 1, 2.0, 0.0) == b.TK_ERR_INVALID_ARG
+    assert fw(4, 8, 1, 2.0, 1.0, w=None) == b.TK_ERR_INVALID_ARG
+    assert fw(4, 8, 1, 2.0, 1.0, out=None) == b.TK_ERR_INVALID_ARG
+    assert fw(4, 8, 1, 1.5, 1.0) == b.TK_ERR_UNSUPPORTED            # p = 2 and p = 4/3 only
+    assert fw(4, 4096, 1, 2.0, 1.0) == b.TK_ERR_UNSUPPORTED         # rows of up to 2048 elements
+    assert fw(0, 8, 1, 2.0, 1.0) == b.TK_OK
+    assert lib.tk_vjp_w(fake, fake, None, 4, 8, 1, 2.0, 1.0, fake, None, None) == b.TK_ERR_INVALID_ARG
+    assert lib.tk_vjp_w(fake, fake, fake, 0, 8, 1, 2.0, 1.0, fake, None, None) == b.TK_OK
+
+
+class FakeDeviceTensor:
+    """Stands in for a CUDA tensor in the binding's checks (which run before any call into the library)."""
+
+    def __init__(self, numel, dtype, contiguous=True, cuda=True):
+        import torch
+        self._numel, self.dtype, self._c, self.is_cuda = numel, getattr(torch, dtype), contiguous, cuda
+
+    def numel(self):
+        return self._numel
+
+    def is_contiguous(self):
+        return self._c
+
+    def data_ptr(self):
+        return 256
+
+
+def test_binding_refuses_buffers_shorter_than_the_call_needs(lib, monkeypatch):
+    from paper_2302_01425_b200 import binding as b
+
+    class Unreachable:
+        def __getattr__(self, name):
+            def call(*args):
+                raise AssertionError(f"{name}: the library must not be called with a short buffer")
+            return call
+
+    monkeypatch.setattr(b, "load", lambda: Unreachable())
+    monkeypatch.setattr(b, "_stream", lambda: None)
+    T = FakeDeviceTensor
+    ok = lambda m: T(m, "float32")
+    with pytest.raises(ValueError, match="theta: 31 elements, the call needs 32"):
+        b.tk_fwd(ok(31), 4, 8, 2, 2.0, 1.0, 0, ok(32))
+    with pytest.raises(ValueError, match="out: 16 elements"):
+        b.tk_fwd_noalloc(T(10 ** 6, "float32"), 2, 40000, 2, 2.0, 1.0, 0, ok(16))
+    with pytest.raises(ValueError, match="perm_out"):
+        b.tk_fwd_ex(ok(32), 4, 8, 2, 2.0, 1.0, 0, ok(32), perm_out=T(8, "int32"))
+    with pytest.raises(ValueError, match="state"):
+        b.tk_fwd_ex(ok(32), 4, 8, 2, 2.0, 1.0, 0, ok(32), state_out=T(63, "uint8"))
+    with pytest.raises(ValueError, match="status_out"):
+        b.tk_fwd_ex(ok(32), 4, 8, 2, 2.0, 1.0, 0, ok(32), status_out=T(0, "int32"))
+    with pytest.raises(ValueError, match="grad_out"):
+        b.tk_vjp(ok(32), ok(8), 4, 8, 2, 2.0, 1.0, 0, ok(32))
+    with pytest.raises(ValueError, match="grad_theta"):
+        b.tk_vjp(ok(32), ok(32), 4, 8, 2, 2.0, 1.0, 0, ok(31))
+    with pytest.raises(ValueError, match="out_tangent"):
+        b.tk_jvp(ok(32), ok(32), 4, 8, 2, 2.0, 1.0, 0, ok(3), state=T(64, "uint8"))
+    with pytest.raises(ValueError, match="target"):
+        b.tk_topk_loss(ok(32), T(3, "int32"), 4, 8, 2, 2.0, 1.0, ok(4), ok(32))
+    with pytest.raises(ValueError, match="loss"):
+        b.tk_topk_loss(ok(32), T(4, "int32"), 4, 8, 2, 2.0, 1.0, ok(3), ok(32))
+    with pytest.raises(ValueError, match="theta"):       # [n, cols] with a leading dimension: (n - 1) * ld + cols
+        b.tk_fwd_cols(ok(7 * 10 + 6 - 1), 8, 6, 10, 2, 2.0, 1.0, 0, ok(100), workspace=T(1 << 20, "uint8"))
+    with pytest.raises(ValueError, match="sorted_out"):
+        b.tk_argsort(ok(32), 4, 8, 0, T(32, "int32"), ok(31))
+    with pytest.raises(ValueError, match="w: 8 elements, the call needs 32"):
+        b.tk_fwd_w(ok(32), ok(8), 1, 32, 2.0, 1.0, ok(32))
+    with pytest.raises(ValueError, match="grad_theta"):
+        b.tk_vjp_w(ok(32), ok(8), ok(32), 4, 8, 2.0, 1.0, ok(31))
+    # wrong dtype, host memory and strided views are refused too
+    with pytest.raises(ValueError, match="contiguous CUDA tensor"):
+        b.tk_fwd(T(32, "float64"), 4, 8, 2, 2.0, 1.0, 0, ok(32))
+    with pytest.raises(ValueError, match="contiguous CUDA tensor"):
+        b.tk_fwd(T(32, "float32", cuda=False), 4, 8, 2, 2.0, 1.0, 0, ok(32))
+    with pytest.raises(ValueError, match="contiguous CUDA tensor"):
+        b.tk_fwd(T(32, "float32", contiguous=False), 4, 8, 2, 2.0, 1.0, 0, ok(32))
 
 
 def test_product_path_does_not_touch_the_oracle():

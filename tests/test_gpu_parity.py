@@ -585,7 +585,7 @@ def test_sort_free_solver_ties_outliers_and_limits():
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
 
 
-@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK])
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
 @pytest.mark.parametrize("p", [1.5, 1.2, 1.1])
 def test_general_p_matches_oracle(mode, p):
     """p other than 2 and 4/3 (q = 3, 6, 11): forward pass by the sort-free solver, VJP from state."""
@@ -598,6 +598,8 @@ def test_general_p_matches_oracle(mode, p):
         res = run_case(x, k, p, lam, mode, g, label=f"p={p} n={n} k={k} lam={lam} mode={mode}",
                        solver=tk.TK_SOLVER_THRESHOLD)
         assert "vjp_state_max_rel" in res
+    if mode == tk.TK_TOPKMAG:      # phi even: the sort-free solver at every length, VJP from state only
+        return
     # rows of up to 128 elements take the sorting kernel with a per-row Newton iteration (solver AUTO):
     # forward, VJP from state and recomputing VJP
     for n, k, lam, rows, seed in [(8, 3, 0.5, 200, 511), (16, 2, 1.0, 130, 512), (64, 2, 0.3, 300, 513),
@@ -631,10 +633,34 @@ def test_general_p_limits():
         with pytest.raises(tk.TkError) as e:
             tk.tk_fwd_ex(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out, **kwargs)
         assert e.value.status == tk.TK_ERR_UNSUPPORTED
-    for p_bad in (3.0, 1.8):                                               # q < 2; 2 < q < 3
-        with pytest.raises(tk.TkError) as e:
-            tk.tk_fwd(th, 4, 64, 2, p_bad, 1.0, tk.TK_MASK, out)
-        assert e.value.status == tk.TK_ERR_UNSUPPORTED
+    with pytest.raises(tk.TkError) as e:                                   # q < 2
+        tk.tk_fwd(th, 4, 64, 2, 3.0, 1.0, tk.TK_MASK, out)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
+def test_forward_pass_between_p_1_5_and_2(mode):
+    """1.5 < p < 2 (2 < q < 3): the forward pass (and the smooth top-k loss) is served, derivatives are
+    refused (rho'' is unbounded at 0 there)."""
+    from oracle import tko
+    for p, n, k, lam, rows in ((1.8, 64, 5, 0.5, 40), (1.6, 300, 30, 1.0, 8), (1.9, 1000, 100, 2.0, 4)):
+        x = rows_of(n, rows, 520 + n)
+        th = torch.from_numpy(x).cuda()
+        out = torch.full_like(th, float("nan"))
+        st = tk.new_state(rows)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, state_out=st, status_out=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = tko.fwd(x, k, p, lam, mode)
+        err = np.abs(out.cpu().numpy() - ref) / np.maximum(1.0, np.abs(ref))
+        assert err.max() <= 1e-5, (p, n, err.max())
+        g = torch.randn_like(th)
+        for call in (lambda: tk.tk_vjp(th, g, rows, n, k, p, lam, mode, out, state=st),
+                     lambda: tk.tk_jvp(th, g, rows, n, k, p, lam, mode, out, state=st)):
+            with pytest.raises(tk.TkError) as e:
+                call()
+            assert e.value.status == tk.TK_ERR_UNSUPPORTED
 
 
 @pytest.mark.parametrize("mode", [tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG])
@@ -732,3 +758,90 @@ def test_unaligned_base_pointers_take_the_scalar_path_and_agree():
                 assert torch.equal(o, got[0][0]), (n, mode)
                 for a, b in ((d, got[0][1]), (d2, got[0][2])):
                     assert float(((a - b).abs() / b.abs().clamp(min=1.0)).max()) <= 1e-6, (n, mode)
+
+
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_sorted_w_matches_oracle(p):
+    """tk_fwd_w / tk_vjp_w (relaxed linear maximisation over the permutahedron of any sorted w) against
+    the oracle's stack PAV: w = 1_k (must also equal the top-k mask path), a ramp, a three-level w,
+    the relaxed rank and the relaxed sort.  The VJP jumps where two blocks merge, so elements whose
+    pooled block changes under a 1e-6 relative perturbation of theta in the oracle are left out of it."""
+    from oracle import tko
+    TOL = 1e-5
+
+    def rel(a, b):
+        return np.abs(a - b) / np.maximum(1.0, np.abs(b))
+
+    def stable_elements(x, w, lam):
+        """[rows, n] mask of the elements whose pooled block (as a set of ranks) is the same for theta and
+        for two perturbed copies of it: Prop. 7's Jacobian of an element involves its own block only."""
+        def blocks_by_index(det):
+            lo = np.empty_like(det["block_lo"]); hi = np.empty_like(det["block_hi"])
+            np.put_along_axis(lo, det["perm"].astype(np.int64), det["block_lo"], axis=1)
+            np.put_along_axis(hi, det["perm"].astype(np.int64), det["block_hi"], axis=1)
+            return lo, hi
+        _, d0 = tko.fwd_w(x, w, p, lam, details=True)
+        lo0, hi0 = blocks_by_index(d0)
+        ok = np.ones(x.shape, bool)
+        rng = np.random.Generator(np.random.PCG64(5))
+        for _ in range(2):
+            xq = (x.astype(np.float64) * (1.0 + 1e-6 * rng.standard_normal(x.shape)) + 1e-6 * rng.standard_normal(x.shape)).astype(np.float32)
+            _, d1 = tko.fwd_w(xq, w, p, lam, details=True)
+            lo1, hi1 = blocks_by_index(d1)
+            ok &= (lo0 == lo1) & (hi0 == hi1)
+        return ok
+
+    def run(x, w, lam, label):
+        rows, n = x.shape
+        th = torch.from_numpy(np.ascontiguousarray(x)).cuda()
+        wt = torch.from_numpy(np.ascontiguousarray(w, np.float32)).cuda()
+        w64 = np.asarray(wt.cpu().numpy(), np.float64)             # the oracle sees the fp32 values the GPU sees
+        out = torch.full((rows, n), float("nan"), device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        tk.tk_fwd_w(th, wt, rows, n, p, lam, out, status_out=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        ref = tko.fwd_w(x, w64, p, lam)
+        e = rel(out.cpu().numpy().astype(np.float64), ref)
+        assert e.max() <= TOL, f"{label}: forward {e.max()}"
+        g = wl.cotangent_like(x, 77)
+        gt = torch.from_numpy(g).cuda()
+        grad = torch.full((rows, n), float("nan"), device="cuda")
+        tk.tk_vjp_w(th, wt, gt, rows, n, p, lam, grad)
+        torch.cuda.synchronize()
+        gref = tko.vjp_w(x, w64, g, p, lam)
+        ok = stable_elements(x, w64, lam)
+        assert ok.mean() >= 0.5, f"{label}: only {ok.mean():.2f} of the elements away from a merge"
+        eg = rel(grad.cpu().numpy().astype(np.float64), gref)[ok]
+        assert np.isfinite(grad.cpu().numpy()).all()
+        assert eg.max() <= TOL, f"{label}: vjp {eg.max()}"
+        return out
+
+    for n, rows in ((5, 33), (64, 40), (100, 17), (1000, 9), (2048, 5)):
+        x = rows_of(n, rows, 900 + n, 1.5)
+        k = max(1, n // 5)
+        for lam in (0.3, 2.0):
+            ones_k = np.r_[np.ones(k), np.zeros(n - k)].astype(np.float32)
+            o = run(x, ones_k, lam, f"1_k n={n} lam={lam}")
+            mask = torch.empty_like(o)
+            tk.tk_fwd(torch.from_numpy(x).cuda(), rows, n, k, p, lam, tk.TK_MASK, mask)
+            torch.cuda.synchronize()
+            assert float((o - mask).abs().max()) <= 2e-5, f"n={n}: general-w path differs from the mask path"
+            run(x, np.arange(n, 0, -1, dtype=np.float32) / n, lam, f"ramp n={n} lam={lam}")
+            levels = np.r_[np.full(n // 3, 2.0), np.full(n // 3, 0.5), np.full(n - 2 * (n // 3), -0.25)].astype(np.float32)
+            run(x, levels, lam, f"levels n={n} lam={lam}")
+        # relaxed rank of x: theta = -x, w = (n, .., 1); relaxed sort: theta = (n, .., 1), w = x sorted, per row
+        rho_v = np.arange(n, 0, -1, dtype=np.float32)
+        run(-x, rho_v, 0.5 * n, f"rank n={n}")
+        run(-x, rho_v, 1.0, f"rank small lambda n={n}")
+        ws = -np.sort(-x, axis=1)
+        run(np.tile(rho_v, (rows, 1)), ws, 1.0, f"sort n={n}")
+    # limits of the entry points
+    th = torch.zeros(4, 4096, device="cuda"); wt = torch.zeros(4096, device="cuda"); o = torch.empty_like(th)
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_w(th, wt, 4, 4096, p, 1.0, o)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_w(th, wt, 4, 1024, 1.5, 1.0, o)
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+

@@ -360,7 +360,7 @@ def test_figure3_is_sparse_and_continuous():
 # --------------------------------------------------------------------------
 # magnitude operator: brute force and optimality of u*
 # --------------------------------------------------------------------------
-@pytest.mark.parametrize("p", [2.0, P43])
+@pytest.mark.parametrize("p", [2.0, P43, 1.5])
 def test_topkmag_equals_epigraph_solution(p):
     rng = np.random.default_rng(21)
     for n, k in [(3, 1), (4, 2), (5, 2), (5, 3)]:
