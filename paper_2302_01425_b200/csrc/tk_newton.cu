@@ -33,6 +33,7 @@
 // accesses straight from the registers; with one or two lanes per row through a shared-memory
 // tile instead.
 #include <float.h>
+#include <stdlib.h>
 #include <math.h>
 
 #include "tk_newton_core.cuh"
@@ -141,6 +142,35 @@ struct NtIO {
   }
 };
 
+// One key against the window (t = key - tau): capped (t >= width), inside (0 < t < width) or zero.
+// Counts and the inside keys' sums of t, t^2, t^3.
+template <bool Q4>
+__device__ __forceinline__ void nt_classify(float t, float wid, float& ct, float& cm, float& a, float& b, float& e) {
+  // two compares, then adds under their predicates (written out so that no select is formed)
+  if (!Q4) {
+    asm("{\n\t.reg .pred ptop, pmid;\n\t"
+        "setp.ge.f32 ptop, %3, %4;\n\t"
+        "setp.gt.and.f32 pmid, %3, 0f00000000, !ptop;\n\t"
+        "@ptop add.f32 %0, %0, 0f3F800000;\n\t"
+        "@pmid add.f32 %1, %1, 0f3F800000;\n\t"
+        "@pmid add.f32 %2, %2, %3;\n\t}"
+        : "+f"(ct), "+f"(cm), "+f"(a)
+        : "f"(t), "f"(wid));
+  } else {
+    asm("{\n\t.reg .pred ptop, pmid;\n\t.reg .f32 t2;\n\t"
+        "setp.ge.f32 ptop, %5, %6;\n\t"
+        "setp.gt.and.f32 pmid, %5, 0f00000000, !ptop;\n\t"
+        "mul.f32 t2, %5, %5;\n\t"
+        "@ptop add.f32 %0, %0, 0f3F800000;\n\t"
+        "@pmid add.f32 %1, %1, 0f3F800000;\n\t"
+        "@pmid add.f32 %2, %2, %5;\n\t"
+        "@pmid add.f32 %3, %3, t2;\n\t"
+        "@pmid fma.rn.f32 %4, t2, %5, %4;\n\t}"
+        : "+f"(ct), "+f"(cm), "+f"(a), "+f"(b), "+f"(e)
+        : "f"(t), "f"(wid));
+  }
+}
+
 // Keeps the loads of later chunks behind this point: the second passes over a row (new pivot, top-k
 // values, smallest capped key) run while the row's registers are live, and E more words in flight would spill.
 __device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
@@ -149,7 +179,7 @@ __device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
 // G lanes per row (W == 1) or W warps per row (G == 32), E keys per lane (E / 4 a power of two).
 // KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1, phi = x only).  MAG: phi(x) = x^2/2, keys |theta|.
 template <int G, int E, int W, bool Q4, int KSEL, bool STAGED, bool MAG>
-__global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_kernel(const Problem P, const float zq) {
+__global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_kernel(const Problem P, const float zq, const int pf_rows) {
   extern __shared__ float4 nt_smem4[];
   static_assert(W == 1 || G == 32, "several warps per row: every lane of them belongs to the row");
   static_assert(!STAGED || W == 1, "the staging tile belongs to one warp");
@@ -324,6 +354,21 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
 #pragma unroll
   for (int i = 0; i < E; ++i) d[i] -= S.piv;
 
+  // The rows this SM slot will hold one wave of blocks from now are asked into L2 once this wave's
+  // own keys have arrived: HBM keeps streaming while the warps iterate on their registers.  One 128-byte
+  // line per lane covers the team's E * T keys.
+  if (!STAGED) {
+    const long long prow = row + pf_rows;
+    const int line = (W > 1 ? wit * 32 + lane : lig) * 32;            // first key of this lane's line
+    if (pf_rows > 0 && prow < P.rows && line < n)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(P.theta + prow * (long long)n + line));
+  } else {
+    const long long prow0 = row0 + pf_rows;                            // the warp's rows are contiguous
+    const long long first = prow0 * (long long)n + lane * 32, end = P.rows * (long long)n;
+    if (pf_rows > 0 && first < end && lane * 32 < R * n)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(P.theta + first));
+  }
+
   // ---- the iteration
   int passes = 0;
 #pragma unroll 1
@@ -332,32 +377,20 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     if (MAG) wid = nt_width<Q4, true>(S.piv + S.off, lam);
     // phi even: tau enters the width and the piece's equation itself, so a step is small against tau too
     const float tol = kTolRel * (MAG ? fminf(wid, fmaxf(S.piv + S.off, 0.0f)) : wid);
-    int ct0 = 0, ct1 = 0, cm0 = 0, cm1 = 0;
+    // Counts are kept as floats (exact: a lane holds at most E keys) and every update is an add under a
+    // predicate: two compares per key on the ALU pipe, everything else on the FMA pipe.
+    float ct0 = 0.f, ct1 = 0.f, cm0 = 0.f, cm1 = 0.f;
     float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f, e0 = 0.f, e1 = 0.f;
     const float off = S.off;
 #pragma unroll
     for (int i = 0; i < E; i += 2) {
-      {
-        const float t = d[i] - off;
-        const bool top = t >= wid, mid = t > 0.0f && !top;
-        ct0 += top; cm0 += mid;
-        const float tm = mid ? t : 0.0f;
-        a0 += tm;
-        if (Q4) { const float t2 = tm * tm; b0 += t2; e0 = fmaf(t2, tm, e0); }
-      }
-      {
-        const float t = d[i + 1] - off;
-        const bool top = t >= wid, mid = t > 0.0f && !top;
-        ct1 += top; cm1 += mid;
-        const float tm = mid ? t : 0.0f;
-        a1 += tm;
-        if (Q4) { const float t2 = tm * tm; b1 += t2; e1 = fmaf(t2, tm, e1); }
-      }
+      nt_classify<Q4>(d[i] - off, wid, ct0, cm0, a0, b0, e0);
+      nt_classify<Q4>(d[i + 1] - off, wid, ct1, cm1, a1, b1, e1);
     }
     float v[Q4 ? 3 : 1];
     v[0] = a0 + a1;
     if (Q4) { v[1] = b0 + b1; v[2] = e0 + e1; }
-    uint32_t packed = (uint32_t)(ct0 + ct1) | ((uint32_t)(cm0 + cm1) << 16);
+    uint32_t packed = (uint32_t)(int)(ct0 + ct1) | ((uint32_t)(int)(cm0 + cm1) << 16);
     team_allsum<G, W, Q4 ? 3 : 1>(v, packed, red + (phase & 1) * (W * 4), wit, lane, bar);
     ++phase;
     if (!S.done) {
@@ -502,6 +535,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
 
 template <int G, int E, int W, bool Q4, int KSEL, bool STAGED, bool MAG>
 cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
+  static const bool no_pf = getenv("TK_NT_NOPF") != nullptr;
   constexpr int BW = kNtWarps > W ? kNtWarps : W;
   constexpr int TEAMS = BW / W;
   constexpr int smem = (STAGED ? BW * 32 * E * (int)sizeof(float) : 0) + (W > 1 ? TEAMS * 2 * W * 4 * (int)sizeof(float) : 0);
@@ -519,7 +553,10 @@ cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
   }
   constexpr long long rows_per_block = (long long)TEAMS * (W > 1 ? 1 : 32 / G);
   const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
-  kern<<<blocks, BW * 32, smem, stream>>>(P, zq);
+  // rows in flight on the whole GPU: the distance the prefetch looks ahead
+  const long long wave = (long long)sm_count() * nt_min_blocks(E, W) * rows_per_block;
+  const int pf_rows = no_pf ? 0 : (int)(wave < 0x7fffffff ? wave : 0);
+  kern<<<blocks, BW * 32, smem, stream>>>(P, zq, pf_rows);
   return cudaGetLastError();
 }
 
