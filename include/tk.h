@@ -1,10 +1,17 @@
 /* tk.h -- C ABI of the sm_100a library for p-norm-regularised (smoothed) top-k
  * operators: the batched forward pass and vector-Jacobian product of
  *   topkmask_R, topk_R, topkmag_R   with   R(y) = (lambda/p) * sum_i |y_i|^p,
- * p = 2 or p = 4/3, w = 1_k (k ones followed by zeros).
+ * p = 2 or p = 4/3 (any other 1 < p < 2 with the limits below), w = 1_k (k ones
+ * followed by zeros); tk_fwd_w / tk_vjp_w take any sorted w.
  *
- * Per row the library sorts theta (or |theta|), solves the isotonic problem the
- * operator reduces to, maps the solution back through grad R*, and un-permutes.
+ * With w = 1_k the isotonic problem the operator reduces to (Prop. 5, Prop. 6) has
+ * at most one pooled block, whose value is the root of a non-increasing threshold
+ * function of one variable (the capped-simplex condition sum y = k of Sec. 3).
+ * By default that root is found per row without sorting, by Newton's iteration
+ * on the pieces of the function, and the result is placed by value; when the
+ * permutation is asked for (or tk_opts.solver says so) the row is sorted and
+ * solved by pool-adjacent-violators on the one block, or by the alternating
+ * projections of Algorithm 1.  All three reach the same solution.
  * Paper references are to "Fast, Differentiable and Sparse Top-k: a Convex
  * Analysis Perspective": Sec. 3 = Background, Sec. 4 = Proposed generalized
  * framework, Sec. 5 = Algorithms, App. A = proofs.
@@ -21,15 +28,16 @@
  *    without a launch.
  *  - 1 <= k <= n, lambda > 0, p > 1.  q = p/(p-1) within 1e-6 of 2 or 4 (p = 2,
  *    p = 4/3: closed-form block solves, App. A.6) runs on every path.  Any other
- *    1 < p <= 1.5 (3 <= q <= 64; Sec. 7, "sensitivity to the choice of p") runs
- *    for TK_MASK and TK_TOPK on rows of up to 16384 elements, without a
- *    permutation output: rows of up to 128 elements are sorted and solved by a
- *    Newton iteration per row (forward pass and tk_vjp with or without saved
- *    state); longer rows go through the sort-free solver whatever
- *    tk_opts.solver says, and tk_vjp needs the saved row state.  Everything else:
- *    TK_ERR_UNSUPPORTED (p > 2 makes rho' unbounded at 0; for 1.5 < p < 2 rho''
- *    is, and fp32 keys cannot carry the VJP to 1e-5).  Outputs must not alias
- *    inputs.
+ *    p with 2 < q <= 64 (Sec. 7, "sensitivity to the choice of p") runs in all
+ *    three modes on rows of up to 16384 elements, without a permutation output
+ *    and with TK_SOLVER_AUTO or TK_SOLVER_THRESHOLD only: rows of up to 128
+ *    elements (TK_MASK, TK_TOPK) are sorted and solved by a Newton iteration per
+ *    row (forward pass and tk_vjp with or without saved state); longer rows and
+ *    TK_TOPKMAG go through the block-per-row threshold solver, and tk_vjp needs
+ *    the saved row state there.  For 1.5 < p < 2 (2 < q < 3) only the forward
+ *    pass runs: rho'' is unbounded at 0 and fp32 keys cannot carry the VJP to
+ *    1e-5, so tk_vjp / tk_jvp return TK_ERR_UNSUPPORTED.  p > 2 (rho' unbounded
+ *    at 0) and q > 64: TK_ERR_UNSUPPORTED.  Outputs must not alias inputs.
  *  - Inputs must be finite.  A NaN/Inf sets TK_FLAG_NONFINITE in *status_out
  *    (when given); that row's output is unspecified, the call still completes.
  */
@@ -54,14 +62,18 @@ typedef enum {
 } tk_mode;
 
 typedef enum {
-  TK_SOLVER_AUTO = 0,
-  TK_SOLVER_PAV = 1,      /* exact pooling of adjacent violators (Sec. 5, App. B.2)          */
+  TK_SOLVER_AUTO = 0,     /* the fastest exact path for the request: the threshold form when
+                             only values are asked for (rows of more than 16 elements, up to
+                             32768; longer rows when there are at most 16 of them), else the
+                             sort and TK_SOLVER_PAV                                          */
+  TK_SOLVER_PAV = 1,      /* sort, then exact pooling of adjacent violators (Sec. 5, App. B.2) */
   TK_SOLVER_DYKSTRA = 2,  /* alternating projections on odd/even pairs (Algorithm 1; for
                              p != 2 the dual block coordinate ascent of App. A.8); rows of
                              up to 131072 elements, those above 16384 with a workspace       */
   TK_SOLVER_THRESHOLD = 3 /* the same exact result as TK_SOLVER_PAV without sorting: root of
                              the capped-simplex threshold function (Sec. 3, P(1_k)); rows of
-                             up to 16384 elements; no permutation output                     */
+                             up to 32768 elements (any length when rows <= 16, with a
+                             workspace); no permutation output                               */
 } tk_solver;
 
 typedef enum {
@@ -77,14 +89,19 @@ typedef enum {
  * return it as a status.                                                                       */
 #define TK_FLAG_NONFINITE 1      /* some input was NaN or Inf                                */
 #define TK_FLAG_NOT_CONVERGED 2  /* an iterative solve stopped at its iteration cap          */
+#define TK_FLAG_BOUNDS 4         /* range-checked build of the library only (libtk_bounds.so):
+                                    an index left its array; that access was skipped         */
 
 /* What the forward pass found for one row, enough to run the VJP without
- * sorting again.  With s the keys in descending order, ranks [a, b) form the
+ * solving again.  With s the keys in descending order, ranks [a, b) form the
  * single pooled block of the isotonic solution (w = 1_k admits at most one),
- * whose common value is gamma = pivot + offset; pivot is the k-th largest key
- * (kept apart from offset so that key - gamma can be formed without
- * cancellation).  a == b == k means no pooled block: every rank < k is a top
- * singleton, every other rank a bottom singleton.                              */
+ * whose common value is gamma = pivot + offset.  pivot is a value near gamma
+ * (the k-th largest key on the sorted paths, the last pivot of the iteration on
+ * the threshold path), kept apart from offset so that key - gamma can be formed
+ * as (key - pivot) - offset without cancellation; every consumer classifies a
+ * key by that expression: capped at width or more, pooled above 0, zero else.
+ * a == b == k means no pooled block: every key >= pivot is a top singleton,
+ * every other key a bottom singleton (offset is 0 then).                       */
 typedef struct {
   float pivot;
   float offset;
@@ -93,7 +110,7 @@ typedef struct {
 } tk_rowstate;
 
 typedef struct {
-  int solver;              /* tk_solver; AUTO = PAV                                           */
+  int solver;              /* tk_solver                                                       */
   int sweeps;              /* Dykstra sweeps; <= 0 means 100 (the count used in Sec. 5)       */
   int32_t *perm_out;       /* [rows*n] sorted rank -> original index, or NULL                 */
   tk_rowstate *state_out;  /* tk_fwd_ex: [rows] written.  tk_vjp: [rows] read (saved by a
@@ -118,7 +135,9 @@ typedef struct {
  * of up to 16384 elements.  Rows of 16385..32768 elements need it only when a
  * permutation is returned (perm_out, tk_argsort), tk_vjp has no saved row
  * state, or the solver is TK_SOLVER_DYKSTRA; the plain forward pass and the VJP
- * from state run without.  solver as in tk_opts.                               */
+ * from state run without.  Longer rows always need it (the threshold path for
+ * at most 16 such rows keeps its per-block partial sums there; the sorting
+ * pipeline its buffers).  solver as in tk_opts.                                */
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver);
 
 /* Forward pass (Prop. 2 with Prop. 5 / Prop. 6): out[r, :] = operator(theta[r, :]).

@@ -20,7 +20,7 @@ TK_MASK, TK_TOPK, TK_TOPKMAG = 0, 1, 2
 TK_SOLVER_AUTO, TK_SOLVER_PAV, TK_SOLVER_DYKSTRA, TK_SOLVER_THRESHOLD = 0, 1, 2, 3
 TK_OK = 0
 TK_ERR_INVALID_ARG, TK_ERR_UNSUPPORTED, TK_ERR_WORKSPACE, TK_ERR_CUDA = 1, 2, 3, 4
-TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED = 1, 2
+TK_FLAG_NONFINITE, TK_FLAG_NOT_CONVERGED, TK_FLAG_BOUNDS = 1, 2, 4
 TK_OPT_STRAIGHT_THROUGH = 1
 ROWSTATE_BYTES = 16
 
@@ -50,6 +50,14 @@ class TkError(RuntimeError):
 
 
 _lib: Optional[ctypes.CDLL] = None
+
+
+def use_library(path: str) -> None:
+    """Bind the calls below to another build of the library (the range-checked libtk_bounds.so);
+    takes effect at the next load()."""
+    global _lib, LIB_PATH
+    LIB_PATH = path
+    _lib = None
 
 
 def load() -> ctypes.CDLL:

@@ -1,6 +1,10 @@
 """Builds the CUDA library (libtk.so) in-tree for sm_100a with nvcc.
 
-    python -m paper_2302_01425_b200.build [--force] [--verbose]
+    python -m paper_2302_01425_b200.build [--force] [--verbose] [--bounds]
+
+--bounds builds the second target, libtk_bounds.so: the same sources with -DTK_DEBUG_BOUNDS, in which
+the kernels of the default path range-check every index they form (a violation sets TK_FLAG_BOUNDS in
+the status word and skips the access).  It stands in for a memory checker where none can be run.
 """
 from __future__ import annotations
 
@@ -13,6 +17,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 CSRC = os.path.join(_PKG, "csrc")
 LIB = os.path.join(_PKG, "libtk.so")
+LIB_BOUNDS = os.path.join(_PKG, "libtk_bounds.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -24,28 +29,31 @@ def sources():
     return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
 
 
-def _stale() -> bool:
-    if not os.path.exists(LIB):
+def _stale(lib: str = LIB) -> bool:
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(
         os.path.join(_ROOT, "include", "*.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, bounds: bool = False) -> str:
+    lib = LIB_BOUNDS if bounds else LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "nvcc")
-    tmp = LIB + f".tmp{os.getpid()}"
+    tmp = lib + f".tmp{os.getpid()}"
     cmd = [nvcc] + NVCC_FLAGS
+    if bounds:
+        cmd += ["-DTK_DEBUG_BOUNDS"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += ["-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-o", tmp] + sources()
     subprocess.run(cmd, check=True)
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, bounds="--bounds" in sys.argv))

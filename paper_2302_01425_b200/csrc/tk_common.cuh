@@ -40,6 +40,23 @@ struct Problem {
   int jvp;                  // tk_vjp_state kernels: the tangent goes through J instead of the cotangent through J^T
 };
 
+// ---------------------------------------------------------------- range-checked build
+// With -DTK_DEBUG_BOUNDS (the second library target of build.py) the kernels of the default path test
+// every global and shared index they form against the extent of its array: an index outside sets
+// TK_FLAG_BOUNDS in the status word and the access is skipped -- no trap, the launch completes.  In the
+// regular build the test is the constant true and costs nothing.
+#ifdef TK_DEBUG_BOUNDS
+__device__ __forceinline__ bool tk_bounds_ok(long long first, long long count, long long extent, int32_t* status) {
+  const bool ok = first >= 0 && count >= 0 && first + count <= extent;
+  if (!ok && status) atomicOr(status, TK_FLAG_BOUNDS);
+  return ok;
+}
+#define TK_IN_BOUNDS(first, count, extent, status) \
+  tk::tk_bounds_ok((long long)(first), (long long)(count), (long long)(extent), (status))
+#else
+#define TK_IN_BOUNDS(first, count, extent, status) true
+#endif
+
 // ---------------------------------------------------------------- host helpers
 // Number of SMs of the current device, asked once per device (148, a B200, if the query fails).
 inline int sm_count() {

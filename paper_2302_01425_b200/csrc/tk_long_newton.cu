@@ -94,17 +94,19 @@ __device__ __forceinline__ float ln_grid_min(float a, float* buf, float* sh, cg:
 
 // f(key, index) over this thread's share of the row: float4 chunks, grid-strided
 template <bool MAG, class F>
-__device__ __forceinline__ void ln_for_each(const float* x_row, int n, int vec4, F f) {
+__device__ __forceinline__ void ln_for_each(const float* x_row, int n, int vec4, int32_t* status, F f) {
   const long long stride = (long long)gridDim.x * kLnThreads;
   const long long first = (long long)blockIdx.x * kLnThreads + threadIdx.x;
   if (vec4) {
     const float4* x4 = reinterpret_cast<const float4*>(x_row);
     for (long long v = first; 4 * v < n; v += stride) {
+      if (!TK_IN_BOUNDS(4 * v, 4, n, status)) continue;
       const float4 q = __ldg(x4 + v);
       f(q.x, 4 * v); f(q.y, 4 * v + 1); f(q.z, 4 * v + 2); f(q.w, 4 * v + 3);
     }
   } else {
-    for (long long i = first; i < n; i += stride) f(__ldg(x_row + i), i);
+    for (long long i = first; i < n; i += stride)
+      if (TK_IN_BOUNDS(i, 1, n, status)) f(__ldg(x_row + i), i);
   }
 }
 
@@ -131,7 +133,7 @@ __global__ void __launch_bounds__(kLnThreads) tk_long_newton_kernel(const Proble
     const float x0 = MAG ? 0.0f : __ldg(x_row);
     LnAcc a{0.f, 0.f, 0.f, 0u, 0u};
     bool bad = false;
-    ln_for_each<MAG>(x_row, n, P.vec4, [&](float x, long long) {
+    ln_for_each<MAG>(x_row, n, P.vec4, P.status, [&](float x, long long) {
       const float key = MAG ? fabsf(x) : x;
       const float dd = key - x0;
       a.v0 += dd; a.v1 = fmaf(dd, dd, a.v1);
@@ -173,7 +175,7 @@ __global__ void __launch_bounds__(kLnThreads) tk_long_newton_kernel(const Proble
       const float tol = kTolRel * (MAG ? fminf(wid, fmaxf(S.piv + S.off, 0.0f)) : wid);
       const float piv = S.piv, off = S.off;
       LnAcc c{0.f, 0.f, 0.f, 0u, 0u};
-      ln_for_each<MAG>(x_row, n, P.vec4, [&](float x, long long) {
+      ln_for_each<MAG>(x_row, n, P.vec4, P.status, [&](float x, long long) {
         const float t = ((MAG ? fabsf(x) : x) - piv) - off;
         const bool top = t >= wid, mid = t > 0.0f && !top;
         c.cnt2 += top; c.cnt += mid;
@@ -198,7 +200,7 @@ __global__ void __launch_bounds__(kLnThreads) tk_long_newton_kernel(const Proble
       if (want_p && !safe) {                   // uniform over the grid
         float cmin = INFINITY;
         const float piv = S.piv, off = S.off;
-        ln_for_each<MAG>(x_row, n, P.vec4, [&](float x, long long) {
+        ln_for_each<MAG>(x_row, n, P.vec4, P.status, [&](float x, long long) {
           const float key = MAG ? fabsf(x) : x;
           if ((key - piv) - off >= wid) cmin = fminf(cmin, key);
         });
@@ -236,11 +238,13 @@ __global__ void __launch_bounds__(kLnThreads) tk_long_newton_kernel(const Proble
         const float4* x4 = reinterpret_cast<const float4*>(x_row);
         float4* o4 = reinterpret_cast<float4*>(o_row);
         for (long long v = first; 4 * v < n; v += stride) {
+          if (!TK_IN_BOUNDS(4 * v, 4, n, P.status)) continue;
           const float4 q = __ldg(x4 + v);
           o4[v] = make_float4(y_of(q.x), y_of(q.y), y_of(q.z), y_of(q.w));
         }
       } else {
-        for (long long i = first; i < n; i += stride) o_row[i] = y_of(__ldg(x_row + i));
+        for (long long i = first; i < n; i += stride)
+          if (TK_IN_BOUNDS(i, 1, n, P.status)) o_row[i] = y_of(__ldg(x_row + i));
       }
     }
     if (bad) flags |= TK_FLAG_NONFINITE;

@@ -74,7 +74,11 @@ __device__ __forceinline__ void nt_top3(float x, float& m1, float& m2, float& m3
 // threads per block, and the blocks per SM the register budget is set for: 24 warps of 80 registers with
 // up to 32 keys per lane, 16 warps of 128 registers with 64
 constexpr int nt_threads(int W) { return team_threads(W); }
-constexpr int nt_min_blocks(int E, int W) { return team_min_blocks(E >= 128 ? 8 : (E >= 64 ? 16 : 24), W); }
+// (p = 4/3 with two lanes per row through the staging tile keeps three more sums and the tile's addresses live: 20 warps of 102
+// registers there, or the classification loop spills)
+constexpr int nt_min_blocks(int E, int W, bool Q4 = false, bool STAGED = false, int G = 32) {
+  return team_min_blocks(E >= 128 ? 8 : (E >= 64 ? 16 : ((Q4 && STAGED && E >= 32 && G == 2) ? 20 : 24)), W);
+}
 
 // ---------------------------------------------------------------- row access
 // A row is spread over a team of T = G * W lanes (G lanes of one warp, or W whole warps), E keys per
@@ -91,9 +95,13 @@ struct NtIO {
   const float* src;      // DIRECT: the row in global memory
   float* dst;
   float4* span4;         // STAGED: this lane's span of the tile
-  int n, tl, rot, vec4;
+  int n, tl, rot, vec4, lane_in_warp;
   bool row_ok;
+  long long first, extent;   // range-checked build: index of the row's first element in the tensor, its size
+  int32_t* status;
 
+  // STAGED: first word of this lane's span in the warp's tile
+  __device__ __forceinline__ int tl_span() const { return lane_in_warp * E; }
   // index in the row of the first key of chunk c
   __device__ __forceinline__ int pos(int c) const {
     return STAGED ? tl * E + 4 * ((c + rot) & (CH - 1)) : 4 * (c * T + tl);
@@ -103,14 +111,23 @@ struct NtIO {
   __device__ __forceinline__ void load_raw(int c, float (&x)[4]) const {
     const int p0 = pos(c);
     if (STAGED) {
-      const float4 v = span4[(c + rot) & (CH - 1)];
+      const int slot = (c + rot) & (CH - 1);
+      x[0] = x[1] = x[2] = x[3] = 0.0f;
+      if (!TK_IN_BOUNDS(tl_span() + 4 * slot, 4, 32 * E, status)) return;
+      const float4 v = span4[slot];
       x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
     } else if (vec4) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(src + (p0 < n ? p0 : 0)));
+      const int pc = p0 < n ? p0 : 0;
+      x[0] = x[1] = x[2] = x[3] = 0.0f;
+      if (!TK_IN_BOUNDS(first + pc, 4, extent, status)) return;
+      const float4 v = __ldg(reinterpret_cast<const float4*>(src + pc));
       x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
     } else {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) x[j] = __ldg(src + (p0 + j < n ? p0 + j : 0));
+      for (int j = 0; j < 4; ++j) {
+        const int pc = p0 + j < n ? p0 + j : 0;
+        x[j] = TK_IN_BOUNDS(first + pc, 1, extent, status) ? __ldg(src + pc) : 0.0f;
+      }
     }
   }
   // slots past the end of the row become -infinity, which never takes part.
@@ -131,13 +148,15 @@ struct NtIO {
   __device__ __forceinline__ void store(int c, const float (&y)[4]) const {
     const int p0 = pos(c);
     if (STAGED) {
-      span4[(c + rot) & (CH - 1)] = make_float4(y[0], y[1], y[2], y[3]);
+      const int slot = (c + rot) & (CH - 1);
+      if (TK_IN_BOUNDS(tl_span() + 4 * slot, 4, 32 * E, status)) span4[slot] = make_float4(y[0], y[1], y[2], y[3]);
     } else if (vec4) {
-      if (row_ok && p0 < n) *reinterpret_cast<float4*>(dst + p0) = make_float4(y[0], y[1], y[2], y[3]);
+      if (row_ok && p0 < n && TK_IN_BOUNDS(first + p0, 4, extent, status))
+        *reinterpret_cast<float4*>(dst + p0) = make_float4(y[0], y[1], y[2], y[3]);
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (row_ok && p0 + j < n) dst[p0 + j] = y[j];
+        if (row_ok && p0 + j < n && TK_IN_BOUNDS(first + p0 + j, 1, extent, status)) dst[p0 + j] = y[j];
     }
   }
 };
@@ -179,7 +198,7 @@ __device__ __forceinline__ void nt_fence() { asm volatile("" ::: "memory"); }
 // G lanes per row (W == 1) or W warps per row (G == 32), E keys per lane (E / 4 a power of two).
 // KSEL: 0 = moment start, 1 / 2 = k is 1 / 2 (W == 1, phi = x only).  MAG: phi(x) = x^2/2, keys |theta|.
 template <int G, int E, int W, bool Q4, int KSEL, bool STAGED, bool MAG>
-__global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_kernel(const Problem P, const float zq, const int pf_rows) {
+__global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W, Q4, STAGED, G)) tk_newton_kernel(const Problem P, const float zq, const int pf_rows) {
   extern __shared__ float4 nt_smem4[];
   static_assert(W == 1 || G == 32, "several warps per row: every lane of them belongs to the row");
   static_assert(!STAGED || W == 1, "the staging tile belongs to one warp");
@@ -213,6 +232,8 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
   const long long row_c = row_ok ? row : P.rows - 1;
   io.src = P.theta + row_c * (long long)n;
   io.dst = P.out + row_c * (long long)n;
+  io.first = row_c * (long long)n; io.extent = P.rows * (long long)n; io.status = P.status;
+  io.lane_in_warp = lane;
   io.span4 = nullptr;
   if (STAGED) {
     // ---- stage the warp's rows (contiguous in memory) in its tile, row stride G * E
@@ -226,23 +247,28 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       if (P.vec4) {
         const float4* s4 = reinterpret_cast<const float4*>(src);
         float4* t4 = reinterpret_cast<float4*>(tile);
-        for (int v = lane; 4 * v < total; v += 32) t4[v] = __ldg(s4 + v);
+        for (int v = lane; 4 * v < total; v += 32)
+          if (TK_IN_BOUNDS(row0 * (long long)n + 4 * v, 4, io.extent, P.status) && TK_IN_BOUNDS(4 * v, 4, 32 * E, P.status)) t4[v] = __ldg(s4 + v);
       } else {
-        for (int i = lane; i < total; i += 32) tile[i] = __ldg(src + i);
+        for (int i = lane; i < total; i += 32)
+          if (TK_IN_BOUNDS(row0 * (long long)n + i, 1, io.extent, P.status) && TK_IN_BOUNDS(i, 1, 32 * E, P.status)) tile[i] = __ldg(src + i);
       }
     } else {
       for (int r = 0; r < rows_here; ++r) {
         if (P.vec4) {
           const float4* s4 = reinterpret_cast<const float4*>(src + (long long)r * n);
           float4* t4 = reinterpret_cast<float4*>(tile + r * RS);
-          for (int v = lane; 4 * v < n; v += 32) t4[v] = __ldg(s4 + v);
+          for (int v = lane; 4 * v < n; v += 32)
+            if (TK_IN_BOUNDS((row0 + r) * (long long)n + 4 * v, 4, io.extent, P.status) && TK_IN_BOUNDS(r * RS + 4 * v, 4, 32 * E, P.status)) t4[v] = __ldg(s4 + v);
         } else {
-          for (int i = lane; i < n; i += 32) tile[r * RS + i] = __ldg(src + (long long)r * n + i);
+          for (int i = lane; i < n; i += 32)
+            if (TK_IN_BOUNDS((row0 + r) * (long long)n + i, 1, io.extent, P.status) && TK_IN_BOUNDS(r * RS + i, 1, 32 * E, P.status)) tile[r * RS + i] = __ldg(src + (long long)r * n + i);
         }
       }
     }
     // lanes whose row lies past the last one solve a row of zeros and store nothing
-    for (int i = rows_here * RS + lane; i < R * RS; i += 32) tile[i] = 0.0f;
+    for (int i = rows_here * RS + lane; i < R * RS; i += 32)
+      if (TK_IN_BOUNDS(i, 1, 32 * E, P.status)) tile[i] = 0.0f;
     __syncwarp();
   }
 
@@ -441,7 +467,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       if (W > 1) {
         float* rb = red + (phase & 1) * (W * 4);
         ++phase;
-        if (lane == 0) rb[wit * 4] = cmin;
+        if (lane == 0 && TK_IN_BOUNDS(team * (2 * W * 4) + ((phase - 1) & 1) * (W * 4) + wit * 4, 1, TEAMS * 2 * W * 4, P.status)) rb[wit * 4] = cmin;
         team_barrier(bar, W * 32);
         cmin = rb[0];
 #pragma unroll
@@ -452,7 +478,7 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
     if (want_p && safe) piv_state = (S.piv + S.off) + 0.5f * wid;
     if (!block) off_state = 0.0f;
   }
-  if (P.state_out && row_ok && lig == 0 && wit == 0) {
+  if (P.state_out && row_ok && lig == 0 && wit == 0 && TK_IN_BOUNDS(row, 1, P.rows, P.status)) {
     tk_rowstate st;
     st.pivot = piv_state; st.offset = off_state; st.a = S.a0; st.b = S.b0;
     P.state_out[row] = st;
@@ -511,18 +537,22 @@ __global__ void __launch_bounds__(nt_threads(W), nt_min_blocks(E, W)) tk_newton_
       if (P.vec4) {
         float4* d4 = reinterpret_cast<float4*>(dst);
         const float4* t4 = reinterpret_cast<const float4*>(tile);
-        for (int v = lane; 4 * v < total; v += 32) d4[v] = t4[v];
+        for (int v = lane; 4 * v < total; v += 32)
+          if (TK_IN_BOUNDS(row0 * (long long)n + 4 * v, 4, io.extent, P.status) && TK_IN_BOUNDS(4 * v, 4, 32 * E, P.status)) d4[v] = t4[v];
       } else {
-        for (int i = lane; i < total; i += 32) dst[i] = tile[i];
+        for (int i = lane; i < total; i += 32)
+          if (TK_IN_BOUNDS(row0 * (long long)n + i, 1, io.extent, P.status) && TK_IN_BOUNDS(i, 1, 32 * E, P.status)) dst[i] = tile[i];
       }
     } else {
       for (int r = 0; r < rows_here; ++r) {
         if (P.vec4) {
           float4* d4 = reinterpret_cast<float4*>(dst + (long long)r * n);
           const float4* t4 = reinterpret_cast<const float4*>(tile + r * RS);
-          for (int v = lane; 4 * v < n; v += 32) d4[v] = t4[v];
+          for (int v = lane; 4 * v < n; v += 32)
+            if (TK_IN_BOUNDS((row0 + r) * (long long)n + 4 * v, 4, io.extent, P.status) && TK_IN_BOUNDS(r * RS + 4 * v, 4, 32 * E, P.status)) d4[v] = t4[v];
         } else {
-          for (int i = lane; i < n; i += 32) dst[(long long)r * n + i] = tile[r * RS + i];
+          for (int i = lane; i < n; i += 32)
+            if (TK_IN_BOUNDS((row0 + r) * (long long)n + i, 1, io.extent, P.status) && TK_IN_BOUNDS(r * RS + i, 1, 32 * E, P.status)) dst[(long long)r * n + i] = tile[r * RS + i];
         }
       }
     }
@@ -554,7 +584,7 @@ cudaError_t nt_launch(const Problem& P, float zq, cudaStream_t stream) {
   constexpr long long rows_per_block = (long long)TEAMS * (W > 1 ? 1 : 32 / G);
   const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
   // rows in flight on the whole GPU: the distance the prefetch looks ahead
-  const long long wave = (long long)sm_count() * nt_min_blocks(E, W) * rows_per_block;
+  const long long wave = (long long)sm_count() * nt_min_blocks(E, W, Q4, STAGED, G) * rows_per_block;
   const int pf_rows = no_pf ? 0 : (int)(wave < 0x7fffffff ? wave : 0);
   kern<<<blocks, BW * 32, smem, stream>>>(P, zq, pf_rows);
   return cudaGetLastError();

@@ -71,20 +71,26 @@ __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk
     const int p0 = 4 * (c * T + tl);
     if (P.vec4) {
       const int pc = p0 < n ? p0 : 0;
-      const float4 xv = __ldg(reinterpret_cast<const float4*>(x_row + pc));
-      const float4 gv = __ldg(reinterpret_cast<const float4*>(g_row + pc));
+      float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), gv = xv;
+      if (TK_IN_BOUNDS(row_c * (long long)n + pc, 4, P.rows * (long long)n, P.status)) {
+        xv = __ldg(reinterpret_cast<const float4*>(x_row + pc));
+        gv = __ldg(reinterpret_cast<const float4*>(g_row + pc));
+      }
       x[4 * c] = xv.x; x[4 * c + 1] = xv.y; x[4 * c + 2] = xv.z; x[4 * c + 3] = xv.w;
       g[4 * c] = gv.x; g[4 * c + 1] = gv.y; g[4 * c + 2] = gv.z; g[4 * c + 3] = gv.w;
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int pc = p0 + j < n ? p0 + j : 0;
-        x[4 * c + j] = __ldg(x_row + pc);
-        g[4 * c + j] = __ldg(g_row + pc);
+        const bool okb = TK_IN_BOUNDS(row_c * (long long)n + pc, 1, P.rows * (long long)n, P.status);
+        x[4 * c + j] = okb ? __ldg(x_row + pc) : 0.0f;
+        g[4 * c + j] = okb ? __ldg(g_row + pc) : 0.0f;
       }
     }
   }
-  const tk_rowstate st = P.state_in[row_c];
+  tk_rowstate st;
+  st.pivot = 0.0f; st.offset = 0.0f; st.a = P.k; st.b = P.k;
+  if (TK_IN_BOUNDS(row_c, 1, P.rows, P.status)) st = P.state_in[row_c];
   const bool has_block = st.b > st.a;
   const float piv = st.pivot, off = st.offset;
   const float wid = has_block ? M.width(piv + off) : 0.0f;
@@ -150,11 +156,12 @@ __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk
       o[j] = fmaf(w[i] * (jt ? xv : 1.0f), fmaf(chi, g[i], -ratio) - delta, fixed[i]);
     }
     if (P.vec4) {
-      if (row_ok && p0 < n) *reinterpret_cast<float4*>(o_row + p0) = make_float4(o[0], o[1], o[2], o[3]);
+      if (row_ok && p0 < n && TK_IN_BOUNDS(row_c * (long long)n + p0, 4, P.rows * (long long)n, P.status))
+        *reinterpret_cast<float4*>(o_row + p0) = make_float4(o[0], o[1], o[2], o[3]);
     } else {
 #pragma unroll
       for (int j = 0; j < 4; ++j)
-        if (row_ok && p0 + j < n) o_row[p0 + j] = o[j];
+        if (row_ok && p0 + j < n && TK_IN_BOUNDS(row_c * (long long)n + p0 + j, 1, P.rows * (long long)n, P.status)) o_row[p0 + j] = o[j];
     }
   }
 }

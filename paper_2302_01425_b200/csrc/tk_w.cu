@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
   for (int i = t; i < N; i += kWThreads) {
     unsigned long long e = 0ull;
     if (i < n) {
-      const float x = __ldg(x_row + i);
+      const float x = TK_IN_BOUNDS(row * (long long)n + i, 1, P.rows * (long long)n, P.status) ? __ldg(x_row + i) : 0.0f;
       bad |= !(fabsf(x) < INFINITY);
       e = ((unsigned long long)f2key(sort_key(x, false)) << 32) | (unsigned)(0xFFFF - i);
       e |= 0x10000ull;                       // a real element outranks the padding (0) even at the smallest key
@@ -138,7 +138,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     for (int j = kk >> 1; j > 0; j >>= 1) {
       for (int i = t; i < N; i += kWThreads) {
         const int l = i ^ j;
-        if (l > i) {
+        if (l > i && TK_IN_BOUNDS(l, 1, N, P.status)) {
           const unsigned long long a = A.keys[i], b = A.keys[l];
           const bool desc = (i & kk) == 0;
           if ((a < b) == desc) { A.keys[i] = b; A.keys[l] = a; }
@@ -151,6 +151,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     const unsigned long long e = A.keys[i];
     A.s[i] = key2f((uint32_t)(e >> 32));
     A.idx[i] = (unsigned short)(0xFFFF - (int)(e & 0xFFFFu));
+    if (!TK_IN_BOUNDS(A.idx[i], 1, n, P.status)) A.idx[i] = 0;
   }
   __syncthreads();
   const double pivot = (double)A.s[n / 2];
@@ -200,7 +201,10 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     double tot;
     int base = (int)w_block_exscan((double)kept, sh_warp, &tot);
     for (int j = j_lo; j < j_hi; ++j)
-      if ((j == 0) || !(A.gam[j - 1] < A.gam[j])) nx[base++] = st[j];
+      if ((j == 0) || !(A.gam[j - 1] < A.gam[j])) {
+        if (TK_IN_BOUNDS(base, 1, n + 1, P.status)) nx[base] = st[j];
+        ++base;
+      }
     const int nb2 = (int)tot;
     __syncthreads();
     cur ^= 1;
@@ -213,7 +217,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     const int* st = A.starts[cur];
     for (int j = t; j < nb; j += kWThreads)
       A.gam[j] = w_block_value<Q4>(A, st[j], j + 1 < nb ? st[j + 1] : n, lam, lam3);
-    if (t == 0) A.starts[cur][nb] = n;
+    if (t == 0 && TK_IN_BOUNDS(nb, 1, n + 1, P.status)) A.starts[cur][nb] = n;
   }
   __syncthreads();
   // ---- 4. results, back through the permutation (out_s reuses the sort buffer)
@@ -259,7 +263,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     __syncthreads();
     for (int i = t; i < n; i += kWThreads) {
       const int b = block_of(i);
-      const int lo = st[b], hi = st[b + 1];
+      const int lo = st[b], hi = TK_IN_BOUNDS(b + 1, 1, n + 1, P.status) ? st[b + 1] : n;
       const double D = A.p1[hi] - A.p1[lo], Ab = A.pw[hi] - A.pw[lo];
       const float tt = (float)(((double)A.s[i] - pivot) - A.gam[b]);
       const float a = tt * inv_lam;
@@ -270,7 +274,8 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
   }
   __syncthreads();
   float* o_row = P.out + row * (long long)n;
-  for (int i = t; i < n; i += kWThreads) o_row[i] = out_s[i];
+  for (int i = t; i < n; i += kWThreads)
+    if (TK_IN_BOUNDS(row * (long long)n + i, 1, P.rows * (long long)n, P.status)) o_row[i] = out_s[i];
   if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
 }
 
