@@ -1,5 +1,5 @@
-// tk_vjp_team.cu -- VJP / JVP from the row state saved by the forward pass, rows of up to 16384
-// elements held in registers.
+// tk_vjp_team.cu -- VJP / JVP from the row state saved by the forward pass, rows of up to 32768
+// elements held in registers (above 16384 in the registers of a cluster of four thread blocks).
 //
 // Prop. 7 makes the Jacobian of the isotonic solution block diagonal with one rank-one block per
 // pooled block; with w = 1_k there is at most one pooled block per row, and its members are
@@ -24,7 +24,11 @@
 // diag(rho') - rho' rho'^T / D, and signs enter as S J S), so the same code serves.  For topk,
 // y = theta o mask(theta): the VJP is g o mask + J_mask^T (theta o g), the JVP is v o mask +
 // theta o (J_mask v): the weight theta moves from inside the block mean to outside it.
+#include <cooperative_groups.h>
+
 #include "tk_team.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace tk {
 
@@ -35,27 +39,51 @@ constexpr int vt_min_blocks(int E, int W, int MODE) {
   return team_min_blocks(E >= 32 ? 16 : (MODE == TK_MASK ? 32 : 24), W);
 }
 
-// QM: 0 = q is 2, 1 = q is 4, 2 = any other q (rho' through powf).  MODE: tk_mode.
-template <int G, int E, int W, int QM, int MODE>
+// The sums of a row shared by the CL thread blocks of a cluster: each block leaves its own total in its
+// shared memory, a cluster barrier, then every block adds the CL totals in rank order (same order, same
+// result in every block).
+template <int NV, int CL>
+__device__ __forceinline__ void vt_cluster_sum(float (&v)[NV], float* slot, cg::cluster_group& cluster) {
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int i = 0; i < NV; ++i) slot[i] = v[i];
+  }
+  cluster.sync();
+#pragma unroll
+  for (int i = 0; i < NV; ++i) v[i] = 0.0f;
+#pragma unroll
+  for (int r = 0; r < CL; ++r) {
+    const float* peer = cluster.map_shared_rank(slot, (unsigned)r);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) v[i] += peer[i];
+  }
+}
+
+// QM: 0 = q is 2, 1 = q is 4, 2 = any other q (rho' through powf).  MODE: tk_mode.  CL: thread blocks
+// per row (above 1: a cluster of CL blocks, each with its share of the row in its registers).
+template <int G, int E, int W, int QM, int MODE, int CL>
 __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk_vjp_team_kernel(const Problem P) {
   extern __shared__ float vt_smem[];
   static_assert(W == 1 || G == 32, "several warps per row: every lane of them belongs to the row");
+  static_assert(CL == 1 || W >= kTeamWarps, "a cluster shares one row: one team per block");
   constexpr int BW = kTeamWarps > W ? kTeamWarps : W;
   constexpr int TEAMS = BW / W;
   constexpr int R = W > 1 ? 1 : 32 / G;
-  constexpr int T = G * W;
+  constexpr int T = G * W * CL;
   constexpr int CH = E / 4;
   constexpr bool MAG = MODE == TK_TOPKMAG, TOPK = MODE == TK_TOPK;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int team = warp / W, wit = warp % W;
-  const long long row0 = ((long long)blockIdx.x * TEAMS + team) * R;
-  if (row0 >= P.rows) return;                  // the whole team
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned crank = CL > 1 ? cluster.block_rank() : 0u;
+  const long long row0 = ((long long)(blockIdx.x / CL) * TEAMS + team) * R;
+  if (row0 >= P.rows) return;                  // the whole team (CL > 1: the grid has exactly CL blocks per row)
   const int n = P.n;
   const int rl = lane / G, lig = lane % G;
   const long long row = row0 + rl;
   const bool row_ok = row < P.rows;
   const long long row_c = row_ok ? row : P.rows - 1;    // a group past the last row repeats it, stores nothing
-  const int tl = W > 1 ? wit * 32 + lane : lig;
+  const int tl = (W > 1 ? wit * 32 + lane : lig) + (CL > 1 ? (int)crank * (W * 32) : 0);
   float* red = vt_smem + team * (2 * W * 4);
   const int bar = 1 + team;
   Math M = make_math(P);
@@ -127,6 +155,8 @@ __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk
   if (__any_sync(0xffffffffu, has_block)) {    // the warps of a row agree: same row state
     uint32_t none = 0;
     team_allsum<G, W, 2>(AD, none, red, wit, lane, bar);
+    float* xch = vt_smem + TEAMS * (2 * W * 4);              // CL == 2: two slots of four words
+    if (CL > 1) vt_cluster_sum<2, CL>(AD, xch, cluster);
     float D = AD[1];
     if (MAG) D += fm;
     const bool ok = has_block && D > 0.0f;
@@ -140,6 +170,10 @@ __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk
       A2[0] = fmaf(fabsf(w[i]), fmaf(chi, g[i], -ratio), A2[0]);   // |w| = rho'
     }
     team_allsum<G, W, 1>(A2, none, red + W * 4, wit, lane, bar);
+    if (CL > 1) {
+      vt_cluster_sum<1, CL>(A2, xch + 4, cluster);
+      cluster.sync();                          // no block leaves while the other may still read its slot
+    }
     if (MAG) A2[0] -= fm * ratio;
     delta = ok ? A2[0] / D : 0.0f;
   }
@@ -166,36 +200,53 @@ __global__ void __launch_bounds__(team_threads(W), vt_min_blocks(E, W, MODE)) tk
   }
 }
 
-template <int G, int E, int W, int QM, int MODE>
+template <int G, int E, int W, int QM, int MODE, int CL>
 cudaError_t vt_launch(const Problem& P, cudaStream_t stream) {
   constexpr int BW = kTeamWarps > W ? kTeamWarps : W;
   constexpr int TEAMS = BW / W;
-  constexpr int smem = TEAMS * 2 * W * 4 * (int)sizeof(float);
+  constexpr int smem = (TEAMS * 2 * W * 4 + (CL > 1 ? 8 : 0)) * (int)sizeof(float);
   constexpr long long rows_per_block = (long long)TEAMS * (W > 1 ? 1 : 32 / G);
-  const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
-  tk_vjp_team_kernel<G, E, W, QM, MODE><<<blocks, BW * 32, smem, stream>>>(P);
-  return cudaGetLastError();
+  if (CL == 1) {
+    const unsigned blocks = (unsigned)((P.rows + rows_per_block - 1) / rows_per_block);
+    tk_vjp_team_kernel<G, E, W, QM, MODE, CL><<<blocks, BW * 32, smem, stream>>>(P);
+    return cudaGetLastError();
+  }
+  // CL thread blocks per row, launched as a cluster
+  if (P.rows > 0x3fffffffLL) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)(P.rows * CL));
+  cfg.blockDim = dim3(BW * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = CL;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tk_vjp_team_kernel<G, E, W, QM, MODE, CL>, P);
 }
 
-template <int G, int E, int W>
+template <int G, int E, int W, int CL = 1>
 cudaError_t vt_launch_mode(const Problem& P, cudaStream_t stream) {
   const int qm = P.qm1 > 0.0f ? 2 : (P.q4 ? 1 : 0);
   switch (P.mode) {
     case TK_MASK:
-      return qm == 0 ? vt_launch<G, E, W, 0, TK_MASK>(P, stream)
-                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_MASK>(P, stream) : vt_launch<G, E, W, 2, TK_MASK>(P, stream));
+      return qm == 0 ? vt_launch<G, E, W, 0, TK_MASK, CL>(P, stream)
+                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_MASK, CL>(P, stream) : vt_launch<G, E, W, 2, TK_MASK, CL>(P, stream));
     case TK_TOPK:
-      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPK>(P, stream)
-                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPK>(P, stream) : vt_launch<G, E, W, 2, TK_TOPK>(P, stream));
+      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPK, CL>(P, stream)
+                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPK, CL>(P, stream) : vt_launch<G, E, W, 2, TK_TOPK, CL>(P, stream));
     default:
-      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPKMAG>(P, stream)
-                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPKMAG>(P, stream) : vt_launch<G, E, W, 2, TK_TOPKMAG>(P, stream));
+      return qm == 0 ? vt_launch<G, E, W, 0, TK_TOPKMAG, CL>(P, stream)
+                     : (qm == 1 ? vt_launch<G, E, W, 1, TK_TOPKMAG, CL>(P, stream) : vt_launch<G, E, W, 2, TK_TOPKMAG, CL>(P, stream));
   }
 }
 
 }  // namespace
 
-int vjp_team_max_n() { return 16384; }
+int vjp_team_max_n() { return 32768; }
 
 // VJP (or JVP) from saved row state for rows of up to vjp_team_max_n() elements.
 cudaError_t launch_vjp_team(const Problem& P, cudaStream_t stream) {
@@ -211,7 +262,8 @@ cudaError_t launch_vjp_team(const Problem& P, cudaStream_t stream) {
   if (n <= 2048) return vt_launch_mode<32, 16, 4>(P, stream);
   if (n <= 4096) return vt_launch_mode<32, 16, 8>(P, stream);
   if (n <= 8192) return vt_launch_mode<32, 16, 16>(P, stream);
-  return vt_launch_mode<32, 32, 16>(P, stream);
+  if (n <= 16384) return vt_launch_mode<32, 32, 16>(P, stream);
+  return vt_launch_mode<32, 16, 16, 4>(P, stream);     // a cluster of four thread blocks per row (two were slower: one block per SM; eight too)
 }
 
 }  // namespace tk
