@@ -404,6 +404,40 @@ def solver_paths(name, r, dev, tk, torch, peak):
     if name in ("sweep_n64", "sweep_n4096"):
         # p = 1.5 (q = 3): no closed-form block solve; the library picks the path
         out["general_p_1.5_forward"] = time_solver_forward(name, dev, tk, torch, tk.TK_SOLVER_AUTO, p_override=1.5)
+    if name == "sweep_n512":
+        # any sorted w (relaxed rank / sort, Sec. 3): a ramp w = (n, .., 1)/n, and w = 1_k through the same kernel
+        out["general_w"] = time_general_w(name, dev, tk, torch)
+    return out
+
+
+def time_general_w(workload, dev, tk, torch, launches=3):
+    """tk_fwd_w and tk_vjp_w (parallel pool-adjacent-violators, one thread block per row) on the
+    workload's rows, p = 2 and p = 4/3."""
+    out = []
+    for c in workload_cases(workload):
+        x = c.theta()
+        th = torch.from_numpy(x).to(dev)
+        gt = torch.from_numpy(c.cotangent(x)).to(dev)
+        y, grad = torch.empty_like(th), torch.empty_like(th)
+        ramp = np.arange(c.n, 0, -1, dtype=np.float32) / c.n
+        ones_k = np.r_[np.ones(c.k), np.zeros(c.n - c.k)].astype(np.float32)
+        for label, w in (("ramp", ramp), ("1_k", ones_k)):
+            wt = torch.from_numpy(w).to(dev)
+            rec = {"p": round(c.p, 6), "w": label}
+            for key, run in (("fwd_us", lambda: tk.tk_fwd_w(th, wt, c.rows, c.n, c.p, c.lam, y)),
+                             ("vjp_us", lambda: tk.tk_vjp_w(th, wt, gt, c.rows, c.n, c.p, c.lam, grad))):
+                run()
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(launches):
+                    run()
+                e1.record()
+                torch.cuda.synchronize()
+                rec[key] = e0.elapsed_time(e1) * 1e3 / launches
+            rec["elements_per_s"] = c.elements / ((rec["fwd_us"] + rec["vjp_us"]) * 1e-6)
+            out.append(rec)
+        del th, gt, y, grad
     return out
 
 

@@ -119,6 +119,13 @@ typedef struct {
   size_t workspace_bytes;
   int32_t *status_out;     /* one device word, OR of TK_FLAG_*; the caller zeroes it          */
   int flags;               /* OR of TK_OPT_*                                                  */
+  float tol;               /* TK_SOLVER_DYKSTRA only.  0: exactly `sweeps` sweeps (Sec. 5 uses fixed
+                              counts).  > 0: the sweeps of a row end as soon as no entry of its
+                              iterate (p = 2) / none of its duals (p = 4/3) moved by more than tol
+                              in any projection of a sweep; `sweeps` is then the cap, and a row that
+                              reaches it sets TK_FLAG_NOT_CONVERGED (a tol below the fp32 spacing of the keys
+                              is never met).  Rows of up to 16384 elements
+                              (longer: TK_ERR_UNSUPPORTED); negative or non-finite: invalid       */
 } tk_opts;
 
 /* tk_fwd_ex only: the "straight-through" use of Sec. 6 (experiments, weight pruning).  out

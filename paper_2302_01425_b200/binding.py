@@ -40,6 +40,7 @@ class TkOpts(ctypes.Structure):
         ("workspace_bytes", ctypes.c_size_t),
         ("status_out", ctypes.c_void_p),
         ("flags", ctypes.c_int),
+        ("tol", ctypes.c_float),
     ]
 
 
@@ -128,9 +129,10 @@ def _stream() -> int:
 
 
 def _opts(solver=TK_SOLVER_AUTO, sweeps=0, perm_out=None, state=None, workspace=None,
-          status_out=None, flags=0, rows=0, n=0) -> TkOpts:
+          status_out=None, flags=0, rows=0, n=0, tol=0.0) -> TkOpts:
     o = TkOpts()
     o.flags = int(flags)
+    o.tol = float(tol)
     o.solver, o.sweeps = int(solver), int(sweeps)
     o.perm_out = _dev(perm_out, torch.int32, "perm_out", rows * n)
     o.state_out = None if state is None else _dev(state, torch.uint8, "state", rows * ROWSTATE_BYTES)
@@ -168,8 +170,8 @@ def tk_fwd_noalloc(theta: torch.Tensor, rows: int, n: int, k: int, p: float, lam
 
 
 def tk_fwd_ex(theta, rows, n, k, p, lam, mode, out, *, solver=TK_SOLVER_AUTO, sweeps=0,
-              perm_out=None, state_out=None, workspace=None, status_out=None, flags=0) -> None:
-    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out, flags, rows=rows, n=n)
+              perm_out=None, state_out=None, workspace=None, status_out=None, flags=0, tol=0.0) -> None:
+    o = _opts(solver, sweeps, perm_out, state_out, workspace, status_out, flags, rows=rows, n=n, tol=tol)
     rc = load().tk_fwd_ex(_dev(theta, torch.float32, "theta", rows * n), rows, n, k, p, lam, mode,
                           _dev(out, torch.float32, "out", rows * n), ctypes.byref(o), _stream())
     if rc != TK_OK:

@@ -204,6 +204,9 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
     if (n > tk::dykstra_cluster_max_n() || (opts && opts->state_out)) return TK_ERR_UNSUPPORTED;
     if (mode == TK_TOPKMAG && q4) return TK_ERR_UNSUPPORTED;
     P.sweeps = opts ? opts->sweeps : 0;
+    P.tol = opts ? opts->tol : 0.0f;
+    if (!(P.tol >= 0.0f) || !isfinite(P.tol)) return TK_ERR_INVALID_ARG;
+    if (P.tol > 0.0f && n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;   // rows of one thread block only
     if (n > tk::kMaxOnChipN) {
       // rows shared by a thread-block cluster: sorted in global memory first (needs the workspace)
       s = check_workspace(opts, rows, n);

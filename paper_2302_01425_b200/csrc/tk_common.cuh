@@ -36,7 +36,8 @@ struct Problem {
   int what;                 // What
   int vec4;                 // rows may be accessed as float4
   float lam, inv_lam, lam3; // lambda, 1/lambda, lambda^3
-  int sweeps;               // Dykstra path
+  int sweeps;               // Dykstra path: number of sweeps, or their cap when tol > 0
+  float tol;                // Dykstra path: > 0 = stop once no entry moved by more than this in a sweep
   int jvp;                  // tk_vjp_state kernels: the tangent goes through J instead of the cotangent through J^T
 };
 

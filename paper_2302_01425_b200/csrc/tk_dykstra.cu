@@ -75,12 +75,17 @@ __device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w
 // projection loses its division and the weights their registers.
 // key_again(i): the key s[i] once more, for the output map of the p = 2 iteration, which does not
 // touch s between its first line and its last: a kernel short of registers reads it from memory there.
-template <int E, bool MAG, typename NextF, typename PrevF, typename SyncF, typename KeyF>
-__device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, const float (&s)[E], int rank0,
+// TOL (run to a tolerance, tk_opts.tol > 0): the largest move of an entry of the iterate (p = 2) or of a
+// dual (p = 4/3) in any projection of a sweep is taken over the row by row_max(x), which returns the same
+// value to every thread of the row; the sweeps end when it is at most P.tol, or at the cap `sweeps`
+// (returns false then: not converged).
+template <int E, bool MAG, bool TOL, typename NextF, typename PrevF, typename SyncF, typename KeyF, typename MaxF>
+__device__ __forceinline__ bool solve_pairs_m(const Problem& P, const Math& M, const float (&s)[E], int rank0,
                                             bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
-                                            SyncF sync, KeyF key_again, float (&y)[E]) {
+                                            SyncF sync, KeyF key_again, MaxF row_max, float (&y)[E]) {
   const int n = P.n, k = P.k;
   const int sweeps = P.sweeps > 0 ? P.sweeps : 100;
+  bool met = !TOL;
   const float s_next = next_of(s[0]);                      // key of the next thread's first rank
   sync();
   const bool cross = has_next && (rank0 + E) < n;          // pair (rank0 + E - 1, rank0 + E) exists
@@ -98,21 +103,35 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
     const float c_next = MAG ? 1.0f + M.lam * wgt(rank0 + E) : 1.0f;
 #pragma unroll 1
     for (int it = 0; it < sweeps; ++it) {
+      float chg = 0.0f;                                    // TOL: largest move of one of this thread's entries
 #pragma unroll
       for (int j = 0; j < E / 2; ++j)
-        if (rank0 + 2 * j + 1 < n) dyk_pair(v[2 * j], v[2 * j + 1], pd[j], c[2 * j], c[2 * j + 1]);
+        if (rank0 + 2 * j + 1 < n) {
+          const float o0 = v[2 * j], o1 = v[2 * j + 1];
+          dyk_pair(v[2 * j], v[2 * j + 1], pd[j], c[2 * j], c[2 * j + 1]);
+          if (TOL) chg = fmaxf(chg, fmaxf(fabsf(v[2 * j] - o0), fabsf(v[2 * j + 1] - o1)));
+        }
       // C2: the pair that crosses to the next thread, then the thread-local ones
       float nb = next_of(v[0]);
       float mine = v[E - 1];
-      if (cross) dyk_pair(mine, nb, qd[E / 2 - 1], c[E - 1], c_next);
+      if (cross) {
+        const float o0 = mine, o1 = nb;
+        dyk_pair(mine, nb, qd[E / 2 - 1], c[E - 1], c_next);
+        if (TOL) chg = fmaxf(chg, fmaxf(fabsf(mine - o0), fabsf(nb - o1)));
+      }
       v[E - 1] = mine;
 #pragma unroll
       for (int j = 0; j < E / 2 - 1; ++j)
-        if (rank0 + 2 * j + 2 < n) dyk_pair(v[2 * j + 1], v[2 * j + 2], qd[j], c[2 * j + 1], c[2 * j + 2]);
+        if (rank0 + 2 * j + 2 < n) {
+          const float o0 = v[2 * j + 1], o1 = v[2 * j + 2];
+          dyk_pair(v[2 * j + 1], v[2 * j + 2], qd[j], c[2 * j + 1], c[2 * j + 2]);
+          if (TOL) chg = fmaxf(chg, fmaxf(fabsf(v[2 * j + 1] - o0), fabsf(v[2 * j + 2] - o1)));
+        }
       sync();
       const float back = prev_of(nb);                      // what the previous thread made of my first rank
       if (has_prev && rank0 < n) v[0] = back;
       sync();
+      if (TOL && row_max(chg) <= P.tol) { met = true; break; }
     }
 #pragma unroll
     for (int i = 0; i < E; ++i) {
@@ -127,12 +146,15 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
     float prev_e = 0.0f;                                   // previous thread's last even-family dual
 #pragma unroll 1
     for (int it = 0; it < sweeps; ++it) {
+      float chg = 0.0f;                                    // TOL: largest move of one of this thread's duals
 #pragma unroll
       for (int j = 0; j < E / 2; ++j) {
         const int rk = rank0 + 2 * j;
         if (rk + 1 < n) {
           const float a_prev = (j == 0) ? prev_e : ae[j - 1];
+          const float old = ao[j];
           ao[j] = bca_alpha(s[2 * j], s[2 * j + 1], wgt(rk), wgt(rk + 1), a_prev, ae[j], M);
+          if (TOL) chg = fmaxf(chg, fabsf(ao[j] - old));
         }
       }
       const float next_o = next_of(ao[0]);
@@ -140,16 +162,19 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
 #pragma unroll
       for (int j = 0; j < E / 2; ++j) {
         const int rk = rank0 + 2 * j + 1;
+        const float old = ae[j];
         if (j < E / 2 - 1) {
           if (rk + 1 < n) ae[j] = bca_alpha(s[2 * j + 1], s[2 * j + 2], wgt(rk), wgt(rk + 1), ao[j], ao[j + 1], M);
         } else if (cross) {
           const float a_next = (rk + 2 < n) ? next_o : 0.0f;
           ae[j] = bca_alpha(s[E - 1], s_next, wgt(rk), wgt(rk + 1), ao[j], a_next, M);
         }
+        if (TOL) chg = fmaxf(chg, fabsf(ae[j] - old));
       }
       const float pe = prev_of(ae[E / 2 - 1]);
       prev_e = has_prev ? pe : 0.0f;
       sync();
+      if (TOL && row_max(chg) <= P.tol) { met = true; break; }
     }
 #pragma unroll
     for (int i = 0; i < E; ++i) {
@@ -158,14 +183,16 @@ __device__ __forceinline__ void solve_pairs_m(const Problem& P, const Math& M, c
       y[i] = wgt(rank0 + i) - a_i + a_im1;
     }
   }
+  return met;
 }
 
-template <int E, typename NextF, typename PrevF, typename SyncF, typename KeyF>
-__device__ __forceinline__ void solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
+// returns false when a run to tolerance (TOL) stopped at the cap
+template <int E, bool TOL, typename NextF, typename PrevF, typename SyncF, typename KeyF, typename MaxF>
+__device__ __forceinline__ bool solve_pairs(const Problem& P, const Math& M, const float (&s)[E], int rank0,
                                             bool has_next, bool has_prev, NextF next_of, PrevF prev_of,
-                                            SyncF sync, KeyF key_again, float (&y)[E]) {
-  if (M.mag) solve_pairs_m<E, true>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
-  else solve_pairs_m<E, false>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
+                                            SyncF sync, KeyF key_again, MaxF row_max, float (&y)[E]) {
+  if (M.mag) return solve_pairs_m<E, true, TOL>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, row_max, y);
+  return solve_pairs_m<E, false, TOL>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, row_max, y);
 }
 
 // ------------------------------------------------------------------ rows of up to 256 elements
@@ -199,8 +226,16 @@ __global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) 
   auto next_of = [&](float x) -> float { return __shfl_down_sync(mask, x, 1, G); };
   auto prev_of = [&](float x) -> float { return __shfl_up_sync(mask, x, 1, G); };
   auto sync = [&]() {};
-  solve_pairs<EPL>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync,
-                   [&](int i) -> float { return s[i]; }, y);
+  auto row_max = [&](float x) -> float {
+#pragma unroll
+    for (int o = G >> 1; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(mask, x, o, G));
+    return x;
+  };
+  auto key_of = [&](int i) -> float { return s[i]; };
+  const bool met = P.tol > 0.0f
+      ? solve_pairs<EPL, true>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync, key_of, row_max, y)
+      : solve_pairs<EPL, false>(P, M, s, EPL * lig, lig < G - 1, lig > 0, next_of, prev_of, sync, key_of, row_max, y);
+  if (!met && lig == 0 && P.status) atomicOr(P.status, TK_FLAG_NOT_CONVERGED);
 
   float* stage = stage_all[grp];
 #pragma unroll
@@ -249,7 +284,24 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   auto prev_of = [&](float x) -> float { xch_b[t] = x; __syncthreads(); return (t > 0) ? xch_b[t - 1] : 0.0f; };
   bool before_sweeps = true;
   auto sync = [&]() { if (before_sweeps) { __syncthreads(); before_sweeps = false; } };
-  solve_pairs<E>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, [&](int i) -> float { return s[i]; }, y);
+  // largest value over the block: warp maxima through a third array (its two barriers also fence the
+  // exchanges of the sweep that follows against this one's)
+  __shared__ float red_max[32];
+  auto row_max = [&](float x) -> float {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    __syncthreads();
+    if ((t & 31) == 0) red_max[t >> 5] = x;
+    __syncthreads();
+    float r = red_max[0];
+    for (int w = 1; w < (T >> 5); ++w) r = fmaxf(r, red_max[w]);
+    return r;
+  };
+  auto key_of = [&](int i) -> float { return s[i]; };
+  const bool met = P.tol > 0.0f
+      ? solve_pairs<E, true>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, key_of, row_max, y)
+      : solve_pairs<E, false>(P, M, s, E * t, t + 1 < T, t > 0, next_of, prev_of, sync, key_of, row_max, y);
+  if (!met && t == 0 && P.status) atomicOr(P.status, TK_FLAG_NOT_CONVERGED);
 
   __syncthreads();
 #pragma unroll
@@ -311,7 +363,9 @@ __global__ void __launch_bounds__(kClusterT, 1) tk_cluster_dykstra_kernel(const 
   // of living through the sweeps, which keeps the iterate and its corrections out of local memory
   // (spill traffic was also what every cluster barrier's fence waited for)
   auto key_again = [&](int i) -> float { return (rank0 + i < n) ? key2f(~__ldg(k_row + rank0 + i)) : 0.0f; };
-  solve_pairs<E>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again, y);
+  // (a fixed number of sweeps only: the tolerance mode is served for rows of one thread block)
+  solve_pairs<E, false>(P, M, s, rank0, has_next, has_prev, next_of, prev_of, sync, key_again,
+                        [](float x) -> float { return x; }, y);
   cluster.sync();
 
   // un-permute: out[sigma_i] = y_i (times the sign of theta for the magnitude mode, times theta for

@@ -86,6 +86,22 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     o = b.TkOpts()
     o.solver = 7
     assert lib.tk_fwd_ex(fake, 4, 8, 2, 2.0, 1.0, 0, fake, ctypes.byref(o), None) == b.TK_ERR_INVALID_ARG
+    o = b.TkOpts()
+    o.solver, o.tol = b.TK_SOLVER_DYKSTRA, -1.0
+    assert lib.tk_fwd_ex(fake, 4, 8, 2, 2.0, 1.0, 0, fake, ctypes.byref(o), None) == b.TK_ERR_INVALID_ARG
+    o.tol = float("nan")
+    assert lib.tk_fwd_ex(fake, 4, 8, 2, 2.0, 1.0, 0, fake, ctypes.byref(o), None) == b.TK_ERR_INVALID_ARG
+    o.tol = 1e-6                                                     # run to tolerance: rows of one thread block only
+    assert lib.tk_fwd_ex(fake, 4, 20000, 2, 2.0, 1.0, 0, fake, ctypes.byref(o), None) == b.TK_ERR_UNSUPPORTED
+
+
+def test_opts_layout_matches_header():
+    from paper_2302_01425_b200 import binding as b
+    text = open(os.path.join(ROOT, "include", "tk.h")).read()
+    body = re.search(r"typedef struct \{([^}]*)\} tk_opts;", text).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    names = [f.strip().split()[-1].lstrip("*") for f in body.split(";") if f.strip()]
+    assert names == [f[0] for f in b.TkOpts._fields_]
 
 
 def test_general_w_arguments_are_rejected_on_the_host(lib):

@@ -515,6 +515,46 @@ def test_operator_along_the_slow_axis(mode):
     assert e.value.status == tk.TK_ERR_INVALID_ARG
 
 
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_dykstra_run_to_tolerance_reaches_the_exact_solution(p):
+    """tk_opts.tol > 0: the sweeps of a row end once no projection of a sweep moves an entry (p = 2) or a
+    dual (p = 4/3) by more than tol; `sweeps` is the cap.  Gated against the exact (pool-adjacent-violators)
+    result of the oracle on short rows, where the alternating projections converge quickly; a cap that is
+    too small must be reported in the status word, a generous one must not."""
+    from oracle import tko
+    modes = (tk.TK_MASK, tk.TK_TOPK, tk.TK_TOPKMAG) if p == 2.0 else (tk.TK_MASK, tk.TK_TOPK)
+    for n, k, lam, rows in ((8, 3, 0.5, 64), (33, 4, 0.3, 40), (64, 8, 0.5, 130), (300, 6, 0.2, 9), (1000, 5, 0.1, 5)):
+        x = rows_of(n, rows, 7100 + n, 1.0)
+        th = torch.from_numpy(x).cuda()
+        for mode in modes:
+            ref = tko.fwd(x, k, p, lam, mode)
+            out = torch.full_like(th, float("nan"))
+            status = torch.zeros(1, dtype=torch.int32, device="cuda")
+            tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=50000, tol=2e-6,
+                         status_out=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0, (n, mode)
+            err = np.abs(out.cpu().numpy().astype(np.float64) - ref) / np.maximum(1.0, np.abs(ref))
+            assert err.max() <= 1e-3, f"n={n} mode={mode} p={p}: {err.max()}"
+            # the same rows with a cap of two sweeps: rows that pool more than a pair cannot have settled
+            status.zero_()
+            tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=2, tol=2e-6,
+                         status_out=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) & tk.TK_FLAG_NOT_CONVERGED, (n, mode)
+            # tol = 0 keeps the fixed count, whatever happens in the sweeps: no flag
+            status.zero_()
+            tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=2, status_out=status)
+            torch.cuda.synchronize()
+            assert int(status.item()) == 0
+    big = torch.zeros(2, 20000, device="cuda")
+    with pytest.raises(tk.TkError) as e:
+        tk.tk_fwd_ex(big, 2, 20000, 5, 2.0, 1.0, tk.TK_MASK, torch.empty_like(big), solver=tk.TK_SOLVER_DYKSTRA,
+                     tol=1e-6, workspace=torch.empty(tk.tk_workspace_bytes(2, 20000, 5, 2.0, 0, tk.TK_SOLVER_DYKSTRA),
+                                                     dtype=torch.uint8, device="cuda"))
+    assert e.value.status == tk.TK_ERR_UNSUPPORTED
+
+
 def test_dykstra_default_sweeps_and_limits():
     from oracle import tko
     x = rows_of(64, 16, 77)
