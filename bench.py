@@ -42,6 +42,7 @@ UNIT = "elements/s"
 BYTES_FWD, BYTES_VJP = 8, 12          # algorithmic bytes per element: theta in + out; theta, g in + grad out
 L2_BYTES = 126e6
 FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0         # the 8 TB/s nameplate figure, reported beside the measured copy bandwidth
 
 
 ROWS_LIMIT = 0
@@ -323,8 +324,10 @@ def main():
             "config": dict(res["config"], parallelism=f"rows sharded x{world}, no collective"),
             "rows_per_s": world * res["rows_per_step"] * steps / (ms_total * 1e-3),
             "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * value / world / 1e9 / peak,
+            "path_frac_of_nominal_8TBps": (BYTES_FWD + BYTES_VJP) * value / world / 1e9 / NOMINAL_HBM_GBS,
             "roofline": {"bound": "hbm", "kernel": dom["name"], "achieved": achieved, "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": achieved / peak,
+                         "frac_of_nominal_8TBps": achieved / NOMINAL_HBM_GBS,
                          "avg_launch_us": dom["avg_us"],
                          "alg_bytes_per_launch": dom["alg_bytes_per_launch"],
                          "traffic": recorded_traffic(args.workload, dom["name"])},
@@ -359,6 +362,7 @@ def main():
                                  "path_frac_of_hbm_peak": (BYTES_FWD + BYTES_VJP) * v2 / 1e9 / peak,
                                  "roofline": {"bound": "hbm", "kernel": d2["name"], "achieved": a2, "peak": peak,
                                               "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": a2 / peak,
+                                              "frac_of_nominal_8TBps": a2 / NOMINAL_HBM_GBS,
                                               "avg_launch_us": d2["avg_us"],
                                               "alg_bytes_per_launch": d2["alg_bytes_per_launch"]},
                                  "kernels": r["kernels"], "config": r["config"]}
