@@ -315,6 +315,115 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
   if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
 }
 
+// ------------------------------------------------------------------ p = 4/3, rows of 257..16384 elements
+// The dual block coordinate ascent of App. A.8 with the pairs dealt to the threads round-robin: thread t
+// owns pairs t, t + T, t + 2T, ... (pair q = ranks 2q, 2q + 1).  The pooled block is a run of consecutive
+// ranks and only its pairs pay the cube roots and the Cardano step; with consecutive ranks per thread it
+// sits in a few warps that set the pace while the rest of the block waits at the sweep's barriers, dealt
+// round-robin every warp holds its share.  The price: every pair's neighbour dual crosses threads, so each
+// half-sweep publishes its family's duals in shared memory (one array per family, a barrier after each
+// write: two barriers per sweep as before).  Pairs of one family do not touch each other, so the iterates
+// are those of the kernel above and of the oracle, sweep by sweep.
+template <int E, int MAXT, int MINB>
+__global__ void __launch_bounds__(MAXT, MINB) tk_cta_bca_kernel(const Problem P) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  constexpr int H = E / 2;                                  // pairs per thread
+  const int T = blockDim.x, t = threadIdx.x, n = P.n, N = P.N, k = P.k;
+  const long long row = blockIdx.x;
+  const Math M = make_math_q24(P);
+  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
+  float* xo = reinterpret_cast<float*>(keys + pad(N) + 1);  // odd-family duals, one per pair: N / 2 floats
+  float* xe = xo + N / 2;                                   // even-family duals
+  float* stage = xo;                                        // the output, by original index (N floats: both arrays)
+  const float* x_row = P.theta + row * (long long)n;
+  unsigned long long r[E];
+  bool bad = false;
+  cta_load_sort<E>(P, x_row, keys, r, bad);
+  if (P.perm_out) {
+    int32_t* pr = P.perm_out + row * (long long)n;
+    for (int i = t; i < n; i += T) pr[i] = un_idx(keys[pad(i)]);
+  }
+  auto wgt = [&](int rk) -> float { return rk < k ? 1.0f : 0.0f; };
+  // this thread's pairs: keys of ranks 2q, 2q + 1 and 2q + 2 (sorted order is in shared memory)
+  float s_lo[H], s_hi[H], s_nx[H], ao[H], ae[H];
+#pragma unroll
+  for (int j = 0; j < H; ++j) {
+    const int q = t + j * T;
+    s_lo[j] = un_key(keys[pad(2 * q)]);
+    s_hi[j] = un_key(keys[pad(2 * q + 1)]);
+    s_nx[j] = (2 * q + 2 < N) ? un_key(keys[pad(2 * q + 2)]) : 0.0f;
+    ao[j] = 0.0f; ae[j] = 0.0f;
+    xe[q] = 0.0f;
+  }
+  __shared__ float red_max[32];
+  auto row_max = [&](float x) -> float {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    __syncthreads();
+    if ((t & 31) == 0) red_max[t >> 5] = x;
+    __syncthreads();
+    float m = red_max[0];
+    for (int w = 1; w < (T >> 5); ++w) m = fmaxf(m, red_max[w]);
+    return m;
+  };
+  const int sweeps = P.sweeps > 0 ? P.sweeps : 100;
+  const bool tol_mode = P.tol > 0.0f;
+  bool met = !tol_mode;
+  __syncthreads();
+#pragma unroll 1
+  for (int it = 0; it < sweeps; ++it) {
+    float chg = 0.0f;
+    // odd family: constraint (2q, 2q + 1); neighbours: the even duals of pairs q - 1 and q
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+      const int q = t + j * T;
+      if (2 * q + 1 < n) {
+        const float a_prev = q > 0 ? xe[q - 1] : 0.0f;
+        const float old = ao[j];
+        ao[j] = bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
+        chg = fmaxf(chg, fabsf(ao[j] - old));
+      }
+      xo[q] = ao[j];
+    }
+    __syncthreads();
+    // even family: constraint (2q + 1, 2q + 2); neighbours: the odd duals of pairs q and q + 1
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+      const int q = t + j * T;
+      if (2 * q + 2 < n) {
+        const float a_next = (2 * q + 3 < n) ? xo[q + 1] : 0.0f;
+        const float old = ae[j];
+        ae[j] = bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
+        chg = fmaxf(chg, fabsf(ae[j] - old));
+      }
+      xe[q] = ae[j];
+    }
+    __syncthreads();
+    if (tol_mode && row_max(chg) <= P.tol) { met = true; break; }
+  }
+  if (!met && t == 0 && P.status) atomicOr(P.status, TK_FLAG_NOT_CONVERGED);
+  // y_i = w_i - alpha_i + alpha_{i-1}; the even dual of pair q - 1 is read before the arrays become the stage
+  float y_lo[H], y_hi[H];
+#pragma unroll
+  for (int j = 0; j < H; ++j) {
+    const int q = t + j * T;
+    const float a_im1 = q > 0 ? xe[q - 1] : 0.0f;
+    y_lo[j] = wgt(2 * q) - ao[j] + a_im1;
+    y_hi[j] = wgt(2 * q + 1) - ae[j] + ao[j];
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < H; ++j) {
+    const int q = t + j * T;
+    if (2 * q < n) { const int idx = un_idx(keys[pad(2 * q)]); if (idx < n) stage[idx] = y_lo[j]; }
+    if (2 * q + 1 < n) { const int idx = un_idx(keys[pad(2 * q + 1)]); if (idx < n) stage[idx] = y_hi[j]; }
+  }
+  __syncthreads();
+  float* o_row = P.out + row * (long long)n;
+  for (int i = t; i < n; i += T) { float q = stage[i]; if (P.mode == TK_TOPK) q *= __ldg(x_row + i); o_row[i] = q; }
+  if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
+}
+
 // ------------------------------------------------------------------ rows of 16385..131072 elements
 // keys, idx: the row-major result of the global-memory radix sort (keys as the complemented
 // order-preserving words it sorts ascending, idx = original index of each rank).  Block c of a
@@ -444,17 +553,33 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
       else { kern = tk_cta_dykstra_kernel<16, 512>; slot = 2; }
       break;
   }
-  static bool configured[4][64] = {};
+  size_t smem_used = smem;
+  if (P.q4 && P.mode != TK_TOPKMAG) {
+    // p = 4/3: the pairs dealt round-robin (one dual per pair and family in shared memory)
+    smem_used = (size_t)(P.N + (P.N >> PAD_SHIFT) + 1) * 8 + (size_t)P.N * 4 + 16;
+    switch (E) {
+      case 4: kern = tk_cta_bca_kernel<4, 128, 6>; slot = 4; break;
+      case 8: kern = tk_cta_bca_kernel<8, 256, 3>; slot = 5; break;
+      default:
+        if (T > 512) { kern = tk_cta_bca_kernel<16, 1024, 1>; slot = 7; }
+        else if (T > 256) { kern = tk_cta_bca_kernel<16, 512, 1>; slot = 6; }
+        else { kern = tk_cta_bca_kernel<16, 256, 3>; slot = 8; }     // three rows per SM: 85 registers
+        break;
+    }
+  }
+  static bool configured[9][64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;
   if (dev < 0 || dev >= 64 || !configured[slot][dev]) {
-    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 1) * 8 + (1024 + 2) * 8 + 16;
+    const int max_smem = (16384 + (16384 >> PAD_SHIFT) + 1) * 8 + 16384 * 4 + 16;
     err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
     if (err != cudaSuccess) return err;
+    // several rows per SM need their shared memory at the same time
+    cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (dev >= 0 && dev < 64) configured[slot][dev] = true;
   }
-  kern<<<(unsigned)P.rows, (unsigned)T, smem, stream>>>(P);
+  kern<<<(unsigned)P.rows, (unsigned)T, smem_used, stream>>>(P);
   return cudaGetLastError();
 }
 
