@@ -253,6 +253,124 @@ __global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) 
   if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
 }
 
+// ------------------------------------------------------------------ p = 4/3, rows of up to 256 elements
+// The sub-warp layout of the kernel above with the pairs dealt to the row's G lanes round-robin (lane l owns
+// pairs l, l + G, ...): the pooled block is a run of consecutive ranks, so at every step of a half-sweep the
+// lanes of a row are either all on heavy pairs (cube roots, Cardano) or all on light ones, where with
+// consecutive ranks per lane one or two lanes of a row did all the heavy work and the warp waited for them.
+// The neighbour duals cross lanes by shuffles: pair q - 1 is the lane below at the same step, or the row's
+// last lane at the step before; pair q + 1 the lane above, or the row's first lane at the next step.
+template <int G>
+__global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
+  constexpr int N = G * EPL;
+  constexpr int GROUPS = 128 / G;
+  constexpr int STRIDE = N + (N >> 3) + 1;
+  constexpr int H = EPL / 2;                                // pairs per lane
+  __shared__ float stage_all[GROUPS][STRIDE];
+  const int tid = threadIdx.x;
+  const int grp = tid / G, lig = tid % G;
+  const long long row = (long long)blockIdx.x * GROUPS + grp;
+  if (row >= P.rows) return;
+  constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
+  const unsigned mask = kGroupBits << ((tid & 31) / G * G);
+  const int n = P.n, k = P.k;
+  const Math M = make_math_q24(P);
+  const float* x_row = P.theta + row * (long long)n;
+  unsigned long long r[EPL];
+  bool bad = false;
+  group_load_pack(P, x_row, lig, M.mag, r, bad);
+  group_sort<G>(r, lig, mask);
+  if (P.perm_out) {
+    int32_t* pr = P.perm_out + row * (long long)n;
+#pragma unroll
+    for (int i = 0; i < EPL; ++i) if (EPL * lig + i < n) pr[EPL * lig + i] = un_idx(r[i]);
+  }
+  float* stage = stage_all[grp];
+  // the sorted keys by rank, then this lane's pairs
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) stage[pad8(EPL * lig + i)] = un_key(r[i]);
+  __syncwarp(mask);
+  auto wgt = [&](int rk) -> float { return rk < k ? 1.0f : 0.0f; };
+  float s_lo[H], s_hi[H], s_nx[H], ao[H], ae[H];
+#pragma unroll
+  for (int j = 0; j < H; ++j) {
+    const int q = lig + j * G;
+    s_lo[j] = stage[pad8(2 * q)];
+    s_hi[j] = stage[pad8(2 * q + 1)];
+    s_nx[j] = (2 * q + 2 < N) ? stage[pad8(2 * q + 2)] : 0.0f;
+    ao[j] = 0.0f; ae[j] = 0.0f;
+  }
+  __syncwarp(mask);
+  const int sweeps = P.sweeps > 0 ? P.sweeps : 100;
+  const bool tol_mode = P.tol > 0.0f;
+  bool met = !tol_mode;
+#pragma unroll 1
+  for (int it = 0; it < sweeps; ++it) {
+    float chg = 0.0f;
+    // odd family: constraint (2q, 2q + 1); neighbours: the even duals of pairs q - 1 and q
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+      const int q = lig + j * G;
+      const float below = __shfl_up_sync(mask, ae[j], 1, G);
+      const float wrap = j > 0 ? __shfl_sync(mask, ae[j > 0 ? j - 1 : 0], G - 1, G) : 0.0f;
+      const float a_prev = lig > 0 ? below : wrap;
+      if (2 * q + 1 < n) {
+        const float old = ao[j];
+        ao[j] = bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
+        chg = fmaxf(chg, fabsf(ao[j] - old));
+      }
+    }
+    // even family: constraint (2q + 1, 2q + 2); neighbours: the odd duals of pairs q and q + 1
+#pragma unroll
+    for (int j = 0; j < H; ++j) {
+      const int q = lig + j * G;
+      const float above = __shfl_down_sync(mask, ao[j], 1, G);
+      const float wrap = j < H - 1 ? __shfl_sync(mask, ao[j < H - 1 ? j + 1 : j], 0, G) : 0.0f;
+      const float a_up = lig < G - 1 ? above : wrap;
+      if (2 * q + 2 < n) {
+        const float a_next = (2 * q + 3 < n) ? a_up : 0.0f;
+        const float old = ae[j];
+        ae[j] = bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
+        chg = fmaxf(chg, fabsf(ae[j] - old));
+      }
+    }
+    if (tol_mode) {
+#pragma unroll
+      for (int o = G >> 1; o > 0; o >>= 1) chg = fmaxf(chg, __shfl_xor_sync(mask, chg, o, G));
+      if (chg <= P.tol) { met = true; break; }
+    }
+  }
+  if (!met && lig == 0 && P.status) atomicOr(P.status, TK_FLAG_NOT_CONVERGED);
+  // y_i = w_i - alpha_i + alpha_{i-1}, by rank into the stage, then back to the sorted registers' layout
+#pragma unroll
+  for (int j = 0; j < H; ++j) {
+    const int q = lig + j * G;
+    const float below = __shfl_up_sync(mask, ae[j], 1, G);
+    const float wrap = j > 0 ? __shfl_sync(mask, ae[j > 0 ? j - 1 : 0], G - 1, G) : 0.0f;
+    const float a_im1 = lig > 0 ? below : wrap;
+    stage[pad8(2 * q)] = wgt(2 * q) - ao[j] + a_im1;
+    stage[pad8(2 * q + 1)] = wgt(2 * q + 1) - ae[j] + ao[j];
+  }
+  __syncwarp(mask);
+  float y[EPL];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) y[i] = stage[pad8(EPL * lig + i)];
+  __syncwarp(mask);
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int idx = un_idx(r[i]);
+    if (EPL * lig + i < n && idx < n) stage[pad8(idx)] = y[i];
+  }
+  __syncwarp(mask);
+  float* o_row = P.out + row * (long long)n;
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    const int idx = EPL * lig + i;
+    if (idx < n) { float q = stage[pad8(idx)]; if (P.mode == TK_TOPK) q *= __ldg(x_row + idx); o_row[idx] = q; }
+  }
+  if (bad && P.status) atomicOr(P.status, TK_FLAG_NONFINITE);
+}
+
 // ------------------------------------------------------------------ rows of up to 16384 elements
 template <int E, int MAXT>
 __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P) {
@@ -529,6 +647,17 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
     P.N = G * EPL;
     const long long groups = 128 / G;
     const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
+    if (P.q4 && P.mode != TK_TOPKMAG) {        // p = 4/3: pairs dealt round-robin to the row's lanes
+      switch (G) {
+        case 1: tk_group_bca_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
+        case 2: tk_group_bca_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
+        case 4: tk_group_bca_kernel<4><<<blocks, 128, 0, stream>>>(P); break;
+        case 8: tk_group_bca_kernel<8><<<blocks, 128, 0, stream>>>(P); break;
+        case 16: tk_group_bca_kernel<16><<<blocks, 128, 0, stream>>>(P); break;
+        default: tk_group_bca_kernel<32><<<blocks, 128, 0, stream>>>(P); break;
+      }
+      return cudaGetLastError();
+    }
     switch (G) {
       case 1: tk_group_dykstra_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
       case 2: tk_group_dykstra_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
