@@ -81,6 +81,7 @@ struct WArrays {
   double* pw;                 // [n + 1] prefix of w
   int* starts[2];             // block starts, ping-pong
   double* gam;                // [n] value per block (relative to the pivot)
+  double* gam2;               // [n] the values carried to the next round's list (NaN: to be computed)
 };
 
 template <bool Q4>
@@ -88,6 +89,7 @@ __device__ __forceinline__ double w_block_value(const WArrays& A, int lo, int hi
   const double N = (double)(hi - lo);
   const double S1 = A.p1[hi] - A.p1[lo], W = A.pw[hi] - A.pw[lo];
   if (!Q4) return (S1 - lam * W) / N;
+  if (hi - lo == 1) return S1 - lam * cbrt(W);             // (g - d)^3 + lam^3 w = 0
   const double S2 = A.p2[hi] - A.p2[lo], S3 = A.p3[hi] - A.p3[lo];
   const double mu = S1 / N;
   const double M2 = fmax(S2 - S1 * mu, 0.0);
@@ -114,6 +116,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
   A.p2 = reinterpret_cast<double*>(ptr); if (Q4) ptr += (size_t)(n + 1) * 8;
   A.p3 = reinterpret_cast<double*>(ptr); if (Q4) ptr += (size_t)(n + 1) * 8;
   A.gam = reinterpret_cast<double*>(ptr); ptr += (size_t)n * 8;
+  A.gam2 = reinterpret_cast<double*>(ptr); ptr += (size_t)n * 8;
   A.s = reinterpret_cast<float*>(ptr); ptr += (size_t)n * 4;
   A.starts[0] = reinterpret_cast<int*>(ptr); ptr += (size_t)(n + 1) * 4;
   A.starts[1] = reinterpret_cast<int*>(ptr); ptr += (size_t)(n + 1) * 4;
@@ -184,39 +187,46 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     for (int i = t; i <= n; i += kWThreads) A.starts[0][i] = i;
   }
   __syncthreads();
-  // ---- 3. rounds of merging
+  // ---- 3. rounds of merging.  A block's value is computed when the block is formed and carried from
+  // round to round until a merge changes the block (NaN marks a value still to be computed).
   int nb = n, cur = 0;
+  double* gam = A.gam;
+  double* gnx = A.gam2;
+  for (int j = t; j < n; j += kWThreads) gam[j] = nan("");
+  __syncthreads();
 #pragma unroll 1
   for (int round = 0; round < n; ++round) {
     const int* st = A.starts[cur];
     int* nx = A.starts[cur ^ 1];
     for (int j = t; j < nb; j += kWThreads)
-      A.gam[j] = w_block_value<Q4>(A, st[j], j + 1 < nb ? st[j + 1] : n, lam, lam3);
+      if (gam[j] != gam[j]) gam[j] = w_block_value<Q4>(A, st[j], j + 1 < nb ? st[j + 1] : n, lam, lam3);
     __syncthreads();
     // keep the start of block j unless block j - 1 violates against it
     const int bchunk = (nb + kWThreads - 1) / kWThreads;
     const int j_lo = min(t * bchunk, nb), j_hi = min(j_lo + bchunk, nb);
     int kept = 0;
-    for (int j = j_lo; j < j_hi; ++j) kept += (j == 0) || !(A.gam[j - 1] < A.gam[j]);
+    for (int j = j_lo; j < j_hi; ++j) kept += (j == 0) || !(gam[j - 1] < gam[j]);
     double tot;
     int base = (int)w_block_exscan((double)kept, sh_warp, &tot);
     for (int j = j_lo; j < j_hi; ++j)
-      if ((j == 0) || !(A.gam[j - 1] < A.gam[j])) {
-        if (TK_IN_BOUNDS(base, 1, n + 1, P.status)) nx[base] = st[j];
+      if ((j == 0) || !(gam[j - 1] < gam[j])) {
+        // block j keeps its value unless it absorbs block j + 1
+        const bool grows = j + 1 < nb && gam[j] < gam[j + 1];
+        if (TK_IN_BOUNDS(base, 1, n + 1, P.status)) { nx[base] = st[j]; gnx[base] = grows ? nan("") : gam[j]; }
         ++base;
       }
     const int nb2 = (int)tot;
     __syncthreads();
     cur ^= 1;
+    { double* tmp = gam; gam = gnx; gnx = tmp; }
     if (nb2 == nb) break;
     nb = nb2;
   }
-  // values of the final blocks (the last round computed them for this very list when it did not merge;
-  // after a merging last round -- only when the cap is hit -- they are recomputed)
+  // values of the final blocks (all known unless the round cap was hit)
   {
     const int* st = A.starts[cur];
     for (int j = t; j < nb; j += kWThreads)
-      A.gam[j] = w_block_value<Q4>(A, st[j], j + 1 < nb ? st[j + 1] : n, lam, lam3);
+      if (gam[j] != gam[j]) gam[j] = w_block_value<Q4>(A, st[j], j + 1 < nb ? st[j + 1] : n, lam, lam3);
     if (t == 0 && TK_IN_BOUNDS(nb, 1, n + 1, P.status)) A.starts[cur][nb] = n;
   }
   __syncthreads();
@@ -232,7 +242,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
   if (P.what == W_FWD) {
     for (int i = t; i < n; i += kWThreads) {
       const int b = block_of(i);
-      const float tt = (float)(((double)A.s[i] - pivot) - A.gam[b]);
+      const float tt = (float)(((double)A.s[i] - pivot) - gam[b]);
       const float a = tt * inv_lam;
       out_s[A.idx[i]] = Q4 ? a * a * a : a;
     }
@@ -242,7 +252,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     double a1 = 0.0, a2 = 0.0;
     for (int i = c_lo; i < c_hi; ++i) {
       const int b = block_of(i);
-      const float tt = (float)(((double)A.s[i] - pivot) - A.gam[b]);
+      const float tt = (float)(((double)A.s[i] - pivot) - gam[b]);
       const float a = tt * inv_lam;
       const double dr = Q4 ? 3.0 * (double)a * (double)a * (double)inv_lam : (double)inv_lam;
       a1 += dr; a2 += dr * (double)__ldg(g_row + A.idx[i]);
@@ -254,7 +264,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
     for (int i = c_lo; i < c_hi; ++i) {
       A.p1[i] = b1; A.pw[i] = b2;
       const int b = block_of(i);
-      const float tt = (float)(((double)A.s[i] - pivot) - A.gam[b]);
+      const float tt = (float)(((double)A.s[i] - pivot) - gam[b]);
       const float a = tt * inv_lam;
       const double dr = Q4 ? 3.0 * (double)a * (double)a * (double)inv_lam : (double)inv_lam;
       b1 += dr; b2 += dr * (double)__ldg(g_row + A.idx[i]);
@@ -265,7 +275,7 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
       const int b = block_of(i);
       const int lo = st[b], hi = TK_IN_BOUNDS(b + 1, 1, n + 1, P.status) ? st[b + 1] : n;
       const double D = A.p1[hi] - A.p1[lo], Ab = A.pw[hi] - A.pw[lo];
-      const float tt = (float)(((double)A.s[i] - pivot) - A.gam[b]);
+      const float tt = (float)(((double)A.s[i] - pivot) - gam[b]);
       const float a = tt * inv_lam;
       const double dr = Q4 ? 3.0 * (double)a * (double)a * (double)inv_lam : (double)inv_lam;
       const double gs = (double)__ldg(g_row + A.idx[i]);
@@ -289,7 +299,7 @@ cudaError_t launch_w(const Problem& P, const float* w, long long w_rows, cudaStr
   int N = 32;
   while (N < P.n) N <<= 1;
   const bool q4 = P.q4 != 0;
-  const size_t smem = (size_t)N * 8 + (size_t)(P.n + 1) * 8 * (q4 ? 4 : 2) + (size_t)P.n * 12 + (size_t)(P.n + 1) * 8 +
+  const size_t smem = (size_t)N * 8 + (size_t)(P.n + 1) * 8 * (q4 ? 4 : 2) + (size_t)P.n * 20 + (size_t)(P.n + 1) * 8 +
                       (size_t)P.n * 2 + 64;
   auto kern = q4 ? tk_w_kernel<true> : tk_w_kernel<false>;
   static bool configured[64][2];
