@@ -33,8 +33,9 @@
  *    and with TK_SOLVER_AUTO or TK_SOLVER_THRESHOLD only: rows of up to 128
  *    elements (TK_MASK, TK_TOPK) are sorted and solved by a Newton iteration per
  *    row (forward pass and tk_vjp with or without saved state); longer rows and
- *    TK_TOPKMAG go through the block-per-row threshold solver, and tk_vjp needs
- *    the saved row state there.  For 1.5 < p < 2 (2 < q < 3) only the forward
+ *    TK_TOPKMAG go through the block-per-row threshold solver, and tk_vjp without
+ *    saved row state runs that forward pass again, keeping its row state in the
+ *    workspace (tk_workspace_bytes; TK_ERR_WORKSPACE without one).  For 1.5 < p < 2 (2 < q < 3) only the forward
  *    pass runs: rho'' is unbounded at 0 and fp32 keys cannot carry the VJP to
  *    1e-5, so tk_vjp / tk_jvp return TK_ERR_UNSUPPORTED.  p > 2 (rho' unbounded
  *    at 0) and q > 64: TK_ERR_UNSUPPORTED.  Outputs must not alias inputs.
@@ -142,7 +143,8 @@ typedef struct {
  * of up to 16384 elements.  Rows of 16385..32768 elements need it only when a
  * permutation is returned (perm_out, tk_argsort), tk_vjp has no saved row
  * state, or the solver is TK_SOLVER_DYKSTRA; the plain forward pass and the VJP
- * from state run without.  Longer rows always need it (the threshold path for
+ * from state run without.  A general p needs rows * sizeof(tk_rowstate) bytes for
+ * tk_vjp without saved state (rows above 128 elements, or TK_TOPKMAG).  Longer rows always need it (the threshold path for
  * at most 16 such rows keeps its per-block partial sums there; the sorting
  * pipeline its buffers).  solver as in tk_opts.                                */
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver);

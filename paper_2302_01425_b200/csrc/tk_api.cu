@@ -144,8 +144,16 @@ const char* tk_status_string(int status) {
 }
 
 size_t tk_workspace_bytes(int64_t rows, int64_t n, int64_t k, double p, int mode, int solver) {
-  (void)k; (void)p; (void)mode; (void)solver;
-  if (rows <= 0 || n <= tk::kMaxOnChipN || n > 0x7fffffff) return 0;
+  (void)k; (void)solver;
+  if (rows <= 0 || n > 0x7fffffff) return 0;
+  if (n <= tk::kMaxOnChipN) {
+    // a general p: tk_vjp without saved state runs the forward pass again and keeps its row state here
+    int q4 = 0;
+    double qm1 = 0.0;
+    if (tk::classify_p(p, &q4, &qm1) == TK_OK && qm1 > 0.0 && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG))
+      return (((size_t)rows * sizeof(tk_rowstate)) + 255u) & ~(size_t)255u;
+    return 0;
+  }
   return tk::long_workspace_bytes(rows, (int)n);
 }
 
@@ -264,9 +272,22 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (rows == 0) return TK_OK;
   if (grad_out == nullptr || grad_theta == nullptr) return TK_ERR_INVALID_ARG;
   if (!vjp_supported(qm1)) return TK_ERR_UNSUPPORTED;
-  // general p: from saved state, or recomputed by the sorting kernel for rows of up to 128 elements (phi = x)
-  if (qm1 > 0.0 && !(opts && opts->state_out) && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG))
-    return TK_ERR_UNSUPPORTED;
+  // general p: from saved state, or recomputed by the sorting kernel for rows of up to 128 elements (phi = x);
+  // otherwise the forward pass runs again here -- its output goes to grad_theta, which the VJP overwrites
+  // afterwards, its row state to the caller's workspace
+  const tk_rowstate* recomputed = nullptr;
+  if (qm1 > 0.0 && !(opts && opts->state_out) && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG)) {
+    if (!opts || !opts->workspace || (reinterpret_cast<uintptr_t>(opts->workspace) & 255u) ||
+        opts->workspace_bytes < (size_t)rows * sizeof(tk_rowstate))
+      return TK_ERR_WORKSPACE;
+    tk_opts f = {};
+    f.solver = TK_SOLVER_AUTO;
+    f.state_out = static_cast<tk_rowstate*>(opts->workspace);
+    f.status_out = opts->status_out;
+    s = tk_fwd_ex(theta, rows, n, k, p, lambda, mode, grad_theta, &f, stream);
+    if (s != TK_OK) return s;
+    recomputed = f.state_out;
+  }
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
   P.gout = grad_out;
@@ -292,8 +313,8 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
     }
     e = tk::launch_vjp_state_long(P, tk::long_workspace_partials(opts->workspace, rows, (int)n),
                                   (cudaStream_t)stream);
-  } else if (opts && opts->state_out) {
-    P.state_in = opts->state_out;
+  } else if (recomputed || (opts && opts->state_out)) {
+    P.state_in = recomputed ? recomputed : opts->state_out;
     e = tk::launch_vjp_state(P, (cudaStream_t)stream);
   } else {
     e = tk::launch_on_chip(P, (cudaStream_t)stream);

@@ -75,7 +75,9 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     assert lib.tk_vjp(fake, fake, 4, 8, 2, 1.8, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED   # 2 < q < 3: forward pass only
     assert lib.tk_jvp(fake, fake, 4, 8, 2, 1.8, 1.0, 0, fake, None, None) in (b.TK_ERR_UNSUPPORTED, b.TK_ERR_INVALID_ARG)
     assert fwd(1, 20000, 2, 1.5, 1.0, 0) == b.TK_ERR_UNSUPPORTED    # q = 3 on a row held in global memory
-    assert lib.tk_vjp(fake, fake, 4, 200, 2, 1.5, 1.0, 0, fake, None, None) == b.TK_ERR_UNSUPPORTED  # q = 3, n > 128, no saved state
+    assert lib.tk_vjp(fake, fake, 4, 200, 2, 1.5, 1.0, 0, fake, None, None) == b.TK_ERR_WORKSPACE  # q = 3, n > 128, no saved state: the forward pass is run again and needs room for its row state
+    assert lib.tk_workspace_bytes(4, 200, 2, 1.5, 0, 0) == 256 and lib.tk_workspace_bytes(4, 200, 2, 2.0, 0, 0) == 0
+    assert lib.tk_workspace_bytes(40, 100, 2, 1.5, 2, 0) == 768 and lib.tk_workspace_bytes(40, 100, 2, 1.5, 0, 0) == 0
     assert fwd(4, 8, 2, 2.0, 1.0, 0, theta=None) == b.TK_ERR_INVALID_ARG
     assert fwd(4, 8, 2, P43, 1.0, 0, out=None) == b.TK_ERR_INVALID_ARG
     assert fwd(0, 8, 2, 2.0, 1.0, 0) == b.TK_OK                     # rows = 0: nothing to do
