@@ -29,8 +29,10 @@
  *  - 1 <= k <= n, lambda > 0, p > 1.  q = p/(p-1) within 1e-6 of 2 or 4 (p = 2,
  *    p = 4/3: closed-form block solves, App. A.6) runs on every path.  Any other
  *    p with 2 < q <= 64 (Sec. 7, "sensitivity to the choice of p") runs in all
- *    three modes on rows of up to 16384 elements, without a permutation output
- *    and with TK_SOLVER_AUTO or TK_SOLVER_THRESHOLD only: rows of up to 128
+ *    three modes on rows of up to 16384 elements, with TK_SOLVER_AUTO or
+ *    TK_SOLVER_THRESHOLD (no permutation output) or TK_SOLVER_DYKSTRA (the dual
+ *    coordinate ascent of App. A.8, every pair solved by a bracketed Newton
+ *    iteration; forward pass only).  With the first two solvers rows of up to 128
  *    elements (TK_MASK, TK_TOPK) are sorted and solved by a Newton iteration per
  *    row (forward pass and tk_vjp with or without saved state); longer rows and
  *    TK_TOPKMAG go through the block-per-row threshold solver, and tk_vjp without
@@ -69,8 +71,10 @@ typedef enum {
                              sort and TK_SOLVER_PAV                                          */
   TK_SOLVER_PAV = 1,      /* sort, then exact pooling of adjacent violators (Sec. 5, App. B.2) */
   TK_SOLVER_DYKSTRA = 2,  /* alternating projections on odd/even pairs (Algorithm 1; for
-                             p != 2 the dual block coordinate ascent of App. A.8); rows of
-                             up to 131072 elements, those above 16384 with a workspace       */
+                             p != 2 the dual block coordinate ascent of App. A.8: closed-form
+                             pair step for p = 4/3 with phi(x) = x, a root solve per pair
+                             otherwise); rows of up to 131072 elements, those above 16384 with
+                             a workspace and p = 2, or p = 4/3 without TK_TOPKMAG, only       */
   TK_SOLVER_THRESHOLD = 3 /* the same exact result as TK_SOLVER_PAV without sorting: root of
                              the capped-simplex threshold function (Sec. 3, P(1_k)); rows of
                              up to 32768 elements (any length when rows <= 16, with a

@@ -171,9 +171,10 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
     // general p: no closed-form block solve.  Rows of up to 128 elements: the sorting kernel with a
     // per-row Newton iteration on the threshold function; longer rows (and every explicit request
     // for it): the sort-free solver.  No permutation output either way.
-    if (solver == TK_SOLVER_PAV || solver == TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
-    if (opts && opts->perm_out) return TK_ERR_UNSUPPORTED;
-    if (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG) solver = TK_SOLVER_THRESHOLD;
+    // (TK_SOLVER_DYKSTRA: the dual coordinate ascent of App. A.8 with a root-solving pair step)
+    if (solver == TK_SOLVER_PAV) return TK_ERR_UNSUPPORTED;
+    if (opts && opts->perm_out && solver != TK_SOLVER_DYKSTRA) return TK_ERR_UNSUPPORTED;
+    if (solver != TK_SOLVER_DYKSTRA && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG)) solver = TK_SOLVER_THRESHOLD;
   }
   tk::Problem P;
   fill(P, theta, rows, n, k, q4, qm1, lambda, mode);
@@ -210,7 +211,8 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
     // Forward pass only: the iterate stays on chip; no row state (the iterate of a fixed number of
     // sweeps has no exact block structure to save); phi even with p = 4/3 has no closed-form pair step.
     if (n > tk::dykstra_cluster_max_n() || (opts && opts->state_out)) return TK_ERR_UNSUPPORTED;
-    if (mode == TK_TOPKMAG && q4) return TK_ERR_UNSUPPORTED;
+    // phi even with p = 4/3 (no closed-form pair step: the root-solving one) on rows of one thread block only
+    if (mode == TK_TOPKMAG && q4 && n > tk::kMaxOnChipN) return TK_ERR_UNSUPPORTED;
     P.sweeps = opts ? opts->sweeps : 0;
     P.tol = opts ? opts->tol : 0.0f;
     if (!(P.tol >= 0.0f) || !isfinite(P.tol)) return TK_ERR_INVALID_ARG;

@@ -68,6 +68,67 @@ __device__ __forceinline__ float bca_alpha(float s1, float s2, float w1, float w
   return fmaxf(0.0f, c1 - z * z * z);
 }
 
+// ---- the same coordinate step for any q and for phi even (App. A.8 leaves the two-variable problem to a
+// root solver; the closed form above is the special case q = 4, phi = x).  rho is odd: sign(t) |t/lambda|^(q-1).
+__device__ __forceinline__ float bca_rho(const Math& M, float t) {
+  const float a = fabsf(t) * M.inv_lam;
+  return copysignf(M.gen ? powf(a, M.qm1) : (M.q4 ? a * a * a : a), t);
+}
+__device__ __forceinline__ float bca_drho(const Math& M, float t) {
+  const float a = fabsf(t) * M.inv_lam;
+  return (M.gen ? M.qm1 * powf(a, M.qm1 - 1.0f) : (M.q4 ? 3.0f * a * a : 1.0f)) * M.inv_lam;
+}
+__device__ __forceinline__ float bca_rho_inv(const Math& M, float z) {
+  const float a = fabsf(z);
+  return copysignf(M.lam * (M.gen ? powf(a, 1.0f / M.qm1) : (M.q4 ? cbrtf(a) : a)), z);
+}
+// Root of an increasing function inside [lo, hi] (f(lo) <= 0 <= f(hi)): Newton, bisection when a step
+// leaves the bracket.  fd(x, f, df) evaluates the function and its derivative.
+template <class FD>
+__device__ __forceinline__ float bca_root(float lo, float hi, float x, FD fd) {
+#pragma unroll 1
+  for (int it = 0; it < 60; ++it) {
+    float f, df;
+    fd(x, f, df);
+    if (f > 0.0f) hi = x; else lo = x;
+    float nx = df > 0.0f ? x - f / df : 0.5f * (lo + hi);
+    if (!(nx > lo && nx < hi)) nx = 0.5f * (lo + hi);
+    if (fabsf(nx - x) <= 1e-7f * fabsf(nx) + 1e-30f || !(hi > lo)) { x = nx; break; }
+    x = nx;
+  }
+  return x;
+}
+// argmin_v r*(s - v) + w phi(v) + c v: -rho(s - v) + w phi'(v) + c = 0
+__device__ __forceinline__ float bca_shifted(const Math& M, float s, float w, float c) {
+  if (!M.mag || w == 0.0f) return s - bca_rho_inv(M, (M.mag ? 0.0f : w) + c);
+  // phi even, w = 1: with t = s - v, rho(t) + t = s + c, t between 0 and s + c
+  const float R = s + c;
+  if (R == 0.0f) return s;
+  const float lo = fminf(0.0f, R), hi = fmaxf(0.0f, R);
+  const float t = bca_root(lo, hi, 0.5f * R, [&](float x, float& f, float& df) {
+    f = bca_rho(M, x) + x - R; df = bca_drho(M, x) + 1.0f; });
+  return s - t;
+}
+// the dual of the constraint between keys s1 >= s2, neighbours' duals fixed
+__device__ __forceinline__ float bca_alpha_any(float s1, float s2, float w1, float w2, float a_prev, float a_next,
+                                              const Math& M) {
+  const float c1 = a_prev, c2 = -a_next;
+  if (!M.mag && w1 + c1 <= w2 + c2) return 0.0f;           // separate minimisers in order (rho_inv is increasing)
+  const float v1 = bca_shifted(M, s1, w1, c1), v2 = bca_shifted(M, s2, w2, c2);
+  if (v1 >= v2) return 0.0f;
+  const float ws = w1 + w2, cs = c1 + c2;
+  const float g = bca_root(v1, v2, 0.5f * (v1 + v2), [&](float x, float& f, float& df) {
+    f = -bca_rho(M, s1 - x) - bca_rho(M, s2 - x) + (M.mag ? ws * x : ws) + cs;
+    df = bca_drho(M, s1 - x) + bca_drho(M, s2 - x) + (M.mag ? ws : 0.0f); });
+  return fmaxf(0.0f, -bca_rho(M, s1 - g) + (M.mag ? w1 * g : w1) + a_prev);
+}
+// y_i = rho(s_i - v_i) at the primal iterate v_i = argmin h_i(v) + (alpha_{i-1} - alpha_i) v
+__device__ __forceinline__ float bca_output(const Math& M, float s, float w, float a_im1, float a_i) {
+  if (!M.mag) return w + a_im1 - a_i;
+  const float v = fmaxf(bca_shifted(M, s, w, a_im1 - a_i), 0.0f);
+  return bca_rho(M, s - v);
+}
+
 // The solver on E consecutive ranks per thread.  Exchange with the neighbouring threads goes
 // through the two callables: next0(x) returns the NEXT thread's x, prev_last(x) the PREVIOUS thread's.
 // On return y[i] = rho(s_i - v_i).
@@ -260,8 +321,8 @@ __global__ void __launch_bounds__(128) tk_group_dykstra_kernel(const Problem P) 
 // consecutive ranks per lane one or two lanes of a row did all the heavy work and the warp waited for them.
 // The neighbour duals cross lanes by shuffles: pair q - 1 is the lane below at the same step, or the row's
 // last lane at the step before; pair q + 1 the lane above, or the row's first lane at the next step.
-template <int G>
-__global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
+template <int G, bool ANY>
+__global__ void __launch_bounds__(128, ANY ? 4 : 6) tk_group_bca_kernel(const Problem P) {
   constexpr int N = G * EPL;
   constexpr int GROUPS = 128 / G;
   constexpr int STRIDE = N + (N >> 3) + 1;
@@ -274,11 +335,12 @@ __global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
   constexpr unsigned kGroupBits = (G == 32) ? 0xffffffffu : ((1u << (G & 31)) - 1u);
   const unsigned mask = kGroupBits << ((tid & 31) / G * G);
   const int n = P.n, k = P.k;
-  const Math M = make_math_q24(P);
+  Math M = make_math(P);
+  if (!ANY) { M.gen = false; M.mag = false; }
   const float* x_row = P.theta + row * (long long)n;
   unsigned long long r[EPL];
   bool bad = false;
-  group_load_pack(P, x_row, lig, M.mag, r, bad);
+  group_load_pack(P, x_row, lig, P.mode == TK_TOPKMAG, r, bad);
   group_sort<G>(r, lig, mask);
   if (P.perm_out) {
     int32_t* pr = P.perm_out + row * (long long)n;
@@ -316,7 +378,8 @@ __global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
       const float a_prev = lig > 0 ? below : wrap;
       if (2 * q + 1 < n) {
         const float old = ao[j];
-        ao[j] = bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
+        ao[j] = ANY ? bca_alpha_any(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M)
+                    : bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
         chg = fmaxf(chg, fabsf(ao[j] - old));
       }
     }
@@ -330,7 +393,8 @@ __global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
       if (2 * q + 2 < n) {
         const float a_next = (2 * q + 3 < n) ? a_up : 0.0f;
         const float old = ae[j];
-        ae[j] = bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
+        ae[j] = ANY ? bca_alpha_any(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M)
+                    : bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
         chg = fmaxf(chg, fabsf(ae[j] - old));
       }
     }
@@ -348,8 +412,8 @@ __global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
     const float below = __shfl_up_sync(mask, ae[j], 1, G);
     const float wrap = j > 0 ? __shfl_sync(mask, ae[j > 0 ? j - 1 : 0], G - 1, G) : 0.0f;
     const float a_im1 = lig > 0 ? below : wrap;
-    stage[pad8(2 * q)] = wgt(2 * q) - ao[j] + a_im1;
-    stage[pad8(2 * q + 1)] = wgt(2 * q + 1) - ae[j] + ao[j];
+    stage[pad8(2 * q)] = ANY ? bca_output(M, s_lo[j], wgt(2 * q), a_im1, ao[j]) : wgt(2 * q) - ao[j] + a_im1;
+    stage[pad8(2 * q + 1)] = ANY ? bca_output(M, s_hi[j], wgt(2 * q + 1), ao[j], ae[j]) : wgt(2 * q + 1) - ae[j] + ao[j];
   }
   __syncwarp(mask);
   float y[EPL];
@@ -359,7 +423,7 @@ __global__ void __launch_bounds__(128, 6) tk_group_bca_kernel(const Problem P) {
 #pragma unroll
   for (int i = 0; i < EPL; ++i) {
     const int idx = un_idx(r[i]);
-    if (EPL * lig + i < n && idx < n) stage[pad8(idx)] = y[i];
+    if (EPL * lig + i < n && idx < n) stage[pad8(idx)] = (ANY && M.mag && un_neg(r[i])) ? -y[i] : y[i];
   }
   __syncwarp(mask);
   float* o_row = P.out + row * (long long)n;
@@ -442,13 +506,16 @@ __global__ void __launch_bounds__(MAXT, 1) tk_cta_dykstra_kernel(const Problem P
 // half-sweep publishes its family's duals in shared memory (one array per family, a barrier after each
 // write: two barriers per sweep as before).  Pairs of one family do not touch each other, so the iterates
 // are those of the kernel above and of the oracle, sweep by sweep.
-template <int E, int MAXT, int MINB>
+// ANY: any q and phi even through the root-solving pair step (one Newton iteration inside another: slow,
+// but the same sweeps); otherwise q = 4, phi = x with the closed form.
+template <int E, int MAXT, int MINB, bool ANY>
 __global__ void __launch_bounds__(MAXT, MINB) tk_cta_bca_kernel(const Problem P) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   constexpr int H = E / 2;                                  // pairs per thread
   const int T = blockDim.x, t = threadIdx.x, n = P.n, N = P.N, k = P.k;
   const long long row = blockIdx.x;
-  const Math M = make_math_q24(P);
+  Math M = make_math(P);
+  if (!ANY) { M.gen = false; M.mag = false; }
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
   float* xo = reinterpret_cast<float*>(keys + pad(N) + 1);  // odd-family duals, one per pair: N / 2 floats
   float* xe = xo + N / 2;                                   // even-family duals
@@ -498,7 +565,8 @@ __global__ void __launch_bounds__(MAXT, MINB) tk_cta_bca_kernel(const Problem P)
       if (2 * q + 1 < n) {
         const float a_prev = q > 0 ? xe[q - 1] : 0.0f;
         const float old = ao[j];
-        ao[j] = bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
+        ao[j] = ANY ? bca_alpha_any(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M)
+                    : bca_alpha(s_lo[j], s_hi[j], wgt(2 * q), wgt(2 * q + 1), a_prev, ae[j], M);
         chg = fmaxf(chg, fabsf(ao[j] - old));
       }
       xo[q] = ao[j];
@@ -511,7 +579,8 @@ __global__ void __launch_bounds__(MAXT, MINB) tk_cta_bca_kernel(const Problem P)
       if (2 * q + 2 < n) {
         const float a_next = (2 * q + 3 < n) ? xo[q + 1] : 0.0f;
         const float old = ae[j];
-        ae[j] = bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
+        ae[j] = ANY ? bca_alpha_any(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M)
+                    : bca_alpha(s_hi[j], s_nx[j], wgt(2 * q + 1), wgt(2 * q + 2), ao[j], a_next, M);
         chg = fmaxf(chg, fabsf(ae[j] - old));
       }
       xe[q] = ae[j];
@@ -526,15 +595,23 @@ __global__ void __launch_bounds__(MAXT, MINB) tk_cta_bca_kernel(const Problem P)
   for (int j = 0; j < H; ++j) {
     const int q = t + j * T;
     const float a_im1 = q > 0 ? xe[q - 1] : 0.0f;
-    y_lo[j] = wgt(2 * q) - ao[j] + a_im1;
-    y_hi[j] = wgt(2 * q + 1) - ae[j] + ao[j];
+    y_lo[j] = ANY ? bca_output(M, s_lo[j], wgt(2 * q), a_im1, ao[j]) : wgt(2 * q) - ao[j] + a_im1;
+    y_hi[j] = ANY ? bca_output(M, s_hi[j], wgt(2 * q + 1), ao[j], ae[j]) : wgt(2 * q + 1) - ae[j] + ao[j];
   }
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < H; ++j) {
     const int q = t + j * T;
-    if (2 * q < n) { const int idx = un_idx(keys[pad(2 * q)]); if (idx < n) stage[idx] = y_lo[j]; }
-    if (2 * q + 1 < n) { const int idx = un_idx(keys[pad(2 * q + 1)]); if (idx < n) stage[idx] = y_hi[j]; }
+    if (2 * q < n) {
+      const unsigned long long e = keys[pad(2 * q)];
+      const int idx = un_idx(e);
+      if (idx < n) stage[idx] = (ANY && M.mag && un_neg(e)) ? -y_lo[j] : y_lo[j];
+    }
+    if (2 * q + 1 < n) {
+      const unsigned long long e = keys[pad(2 * q + 1)];
+      const int idx = un_idx(e);
+      if (idx < n) stage[idx] = (ANY && M.mag && un_neg(e)) ? -y_hi[j] : y_hi[j];
+    }
   }
   __syncthreads();
   float* o_row = P.out + row * (long long)n;
@@ -647,15 +724,23 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
     P.N = G * EPL;
     const long long groups = 128 / G;
     const unsigned blocks = (unsigned)((P.rows + groups - 1) / groups);
-    if (P.q4 && P.mode != TK_TOPKMAG) {        // p = 4/3: pairs dealt round-robin to the row's lanes
+    const bool closed = P.q4 && P.mode != TK_TOPKMAG && !(P.qm1 > 0.0f);   // p = 4/3, phi = x: closed-form pair step
+    const bool any = P.qm1 > 0.0f || (P.q4 && P.mode == TK_TOPKMAG);         // any other q != 2: root-solving pair step
+    if (closed || any) {                       // dual coordinate ascent, pairs dealt round-robin to the row's lanes
+#define TK_GROUP_BCA(GG)                                                     \
+  do {                                                                       \
+    if (any) tk_group_bca_kernel<GG, true><<<blocks, 128, 0, stream>>>(P);   \
+    else tk_group_bca_kernel<GG, false><<<blocks, 128, 0, stream>>>(P);      \
+  } while (0)
       switch (G) {
-        case 1: tk_group_bca_kernel<1><<<blocks, 128, 0, stream>>>(P); break;
-        case 2: tk_group_bca_kernel<2><<<blocks, 128, 0, stream>>>(P); break;
-        case 4: tk_group_bca_kernel<4><<<blocks, 128, 0, stream>>>(P); break;
-        case 8: tk_group_bca_kernel<8><<<blocks, 128, 0, stream>>>(P); break;
-        case 16: tk_group_bca_kernel<16><<<blocks, 128, 0, stream>>>(P); break;
-        default: tk_group_bca_kernel<32><<<blocks, 128, 0, stream>>>(P); break;
+        case 1: TK_GROUP_BCA(1); break;
+        case 2: TK_GROUP_BCA(2); break;
+        case 4: TK_GROUP_BCA(4); break;
+        case 8: TK_GROUP_BCA(8); break;
+        case 16: TK_GROUP_BCA(16); break;
+        default: TK_GROUP_BCA(32); break;
       }
+#undef TK_GROUP_BCA
       return cudaGetLastError();
     }
     switch (G) {
@@ -683,20 +768,23 @@ cudaError_t launch_dykstra(const Problem& P0, cudaStream_t stream) {
       break;
   }
   size_t smem_used = smem;
-  if (P.q4 && P.mode != TK_TOPKMAG) {
-    // p = 4/3: the pairs dealt round-robin (one dual per pair and family in shared memory)
+  const bool closed = P.q4 && P.mode != TK_TOPKMAG && !(P.qm1 > 0.0f);
+  const bool any = P.qm1 > 0.0f || (P.q4 && P.mode == TK_TOPKMAG);
+  if (closed || any) {
+    // q != 2: dual coordinate ascent with the pairs dealt round-robin (one dual per pair and family in shared memory)
     smem_used = (size_t)(P.N + (P.N >> PAD_SHIFT) + 1) * 8 + (size_t)P.N * 4 + 16;
     switch (E) {
-      case 4: kern = tk_cta_bca_kernel<4, 128, 6>; slot = 4; break;
-      case 8: kern = tk_cta_bca_kernel<8, 256, 3>; slot = 5; break;
+      case 4: kern = any ? tk_cta_bca_kernel<4, 128, 4, true> : tk_cta_bca_kernel<4, 128, 6, false>; slot = 4; break;
+      case 8: kern = any ? tk_cta_bca_kernel<8, 256, 2, true> : tk_cta_bca_kernel<8, 256, 3, false>; slot = 5; break;
       default:
-        if (T > 512) { kern = tk_cta_bca_kernel<16, 1024, 1>; slot = 7; }
-        else if (T > 256) { kern = tk_cta_bca_kernel<16, 512, 1>; slot = 6; }
-        else { kern = tk_cta_bca_kernel<16, 256, 3>; slot = 8; }     // three rows per SM: 85 registers
+        if (T > 512) { kern = any ? tk_cta_bca_kernel<16, 1024, 1, true> : tk_cta_bca_kernel<16, 1024, 1, false>; slot = 7; }
+        else if (T > 256) { kern = any ? tk_cta_bca_kernel<16, 512, 1, true> : tk_cta_bca_kernel<16, 512, 1, false>; slot = 6; }
+        else { kern = any ? tk_cta_bca_kernel<16, 256, 2, true> : tk_cta_bca_kernel<16, 256, 3, false>; slot = 8; }
         break;
     }
+    if (any) slot += 5;
   }
-  static bool configured[9][64] = {};
+  static bool configured[14][64] = {};
   int dev = 0;
   cudaError_t err = cudaGetDevice(&dev);
   if (err != cudaSuccess) return err;

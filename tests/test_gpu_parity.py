@@ -344,6 +344,33 @@ def test_dykstra_path_matches_oracle_sweeps(p):
                 assert err <= TOL, (mode, n, k, lam, sweeps, err)
 
 
+@pytest.mark.parametrize("p,mode", [(1.5, tk.TK_MASK), (1.5, tk.TK_TOPK), (1.5, tk.TK_TOPKMAG), (1.2, tk.TK_MASK),
+                                    (P43, tk.TK_TOPKMAG)])
+def test_dykstra_path_root_solving_pair_step_matches_oracle_sweeps(p, mode):
+    """The dual coordinate ascent of App. A.8 for the cases without a closed-form pair step -- any q other
+    than 2 and 4, and phi even with p = 4/3: every coordinate solves its two-variable problem by a bracketed
+    Newton iteration.  Same sweep count in the oracle (whose pair solve is a bisection), <= 1e-5."""
+    from oracle import tko
+    from parity import rel_err, TOL
+    shapes = [(1, 1, 1.0), (2, 1, 0.5), (7, 3, 1.0), (8, 8, 1.0), (33, 7, 0.3), (64, 8, 1.0), (200, 20, 1.0),
+              (257, 40, 0.5), (1000, 5, 0.5), (4096, 512, 1.0)]
+    for n, k, lam in shapes:
+        for sweeps in (1, 10, 100):
+            if n > 1000 and sweeps != 10:
+                continue
+            rows = 5 if n <= 1000 else 2
+            x = rows_of(n, rows, 340 + n)
+            th = torch.from_numpy(x).cuda()
+            out = torch.full_like(th, float("nan"))
+            tk.tk_fwd_ex(th, rows, n, k, p, lam, mode, out, solver=tk.TK_SOLVER_DYKSTRA, sweeps=sweeps)
+            torch.cuda.synchronize()
+            ref = tko.dykstra(x, k, p, lam, mode, sweeps=sweeps)
+            got = out.cpu().numpy()
+            assert np.isfinite(got).all()
+            err = rel_err(got, ref).max()
+            assert err <= TOL, (mode, p, n, k, lam, sweeps, err)
+
+
 @pytest.mark.parametrize("p", [2.0, P43])
 def test_dykstra_cluster_rows_match_oracle_sweeps(p):
     """Rows of 16385..131072 elements: the iterate is shared by a thread-block cluster (2, 3, 5 and 8
@@ -566,8 +593,11 @@ def test_dykstra_default_sweeps_and_limits():
     assert np.max(np.abs(out.cpu().numpy() - ref)) <= 1e-5
     exact = tko.fwd(x, 2, 2.0, 0.3, tko.MASK)
     assert np.max(np.abs(out.cpu().numpy() - exact)) <= 1e-4       # small blocks: 100 sweeps reach PAV
-    with pytest.raises(tk.TkError) as e:
-        tk.tk_fwd_ex(th, 16, 64, 2, P43, 0.3, tk.TK_TOPKMAG, out, solver=tk.TK_SOLVER_DYKSTRA)
+    big = torch.zeros(2, 20000, device="cuda")
+    ws = torch.empty(tk.tk_workspace_bytes(2, 20000, 5, P43, tk.TK_TOPKMAG, tk.TK_SOLVER_DYKSTRA), dtype=torch.uint8, device="cuda")
+    with pytest.raises(tk.TkError) as e:          # phi even with p = 4/3: rows of one thread block only
+        tk.tk_fwd_ex(big, 2, 20000, 5, P43, 0.3, tk.TK_TOPKMAG, torch.empty_like(big), solver=tk.TK_SOLVER_DYKSTRA,
+                     workspace=ws)
     assert e.value.status == tk.TK_ERR_UNSUPPORTED
     with pytest.raises(tk.TkError) as e:
         tk.tk_fwd_ex(th, 16, 64, 2, 2.0, 0.3, tk.TK_MASK, out, solver=tk.TK_SOLVER_DYKSTRA,
@@ -699,7 +729,7 @@ def test_general_p_limits():
     with pytest.raises(tk.TkError) as e:
         tk.tk_vjp(th2, g2, 4, 300, 9, 1.5, 1.0, tk.TK_MASK, out2)          # no saved state on a row of more than 128:
     assert e.value.status == tk.TK_ERR_WORKSPACE                           # the forward pass runs again and needs room
-    for kwargs in ({"solver": tk.TK_SOLVER_PAV}, {"solver": tk.TK_SOLVER_DYKSTRA},
+    for kwargs in ({"solver": tk.TK_SOLVER_PAV},
                    {"perm_out": torch.empty((4, 64), dtype=torch.int32, device="cuda")}):
         with pytest.raises(tk.TkError) as e:
             tk.tk_fwd_ex(th, 4, 64, 2, 1.5, 1.0, tk.TK_MASK, out, **kwargs)
