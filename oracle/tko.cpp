@@ -617,8 +617,13 @@ int tko_fwd_w(const float* theta, const double* w, int64_t rows, int64_t n, int6
 
 // grad_theta = J^T g of y_R(., w) at theta (Prop. 7 with phi(x) = x: D_B = sum_B rho', no w term),
 // chained through y^s_i = rho(s_i - gamma_B): o_j = rho'_j (g^s_j - A_B / D_B), 0 where D_B = 0.
+// grad_w (may be null): the cotangent pulled back to w, per row and in w's own (sorted) order.  Inside a
+// pooled block B the value gamma solves sum_B rho(s_i - gamma) = sum_B w_i (stationarity of the block, Prop. 5
+// with phi(x) = x), so d gamma / d w_j = -1 / D_B and d y_i / d w_j = rho'_i / D_B for i, j in B: the pulled-back
+// cotangent of every w_j of the block is A_B / D_B.  A singleton has y_j = w_j: its entry is g_j also where
+// rho' vanishes.
 int tko_vjp_w(const float* theta, const double* w, const float* gout, int64_t rows, int64_t n,
-              int64_t w_rows, double p, double lambda, double* grad) {
+              int64_t w_rows, double p, double lambda, double* grad, double* grad_w) {
   if (check_args_w(rows, n, p, lambda, w, w_rows)) return 1;
   const Params P = make_params(p, lambda, MASK);
 #pragma omp parallel
@@ -642,6 +647,8 @@ int tko_vjp_w(const float* theta, const double* w, const float* gout, int64_t ro
         for (int64_t i = b.lo; i < b.hi; ++i) {
           double d = drho(P, s[i] - b.gamma);
           grad[r * n + pm[i]] = (D > 0.0) ? d * ((double)g[pm[i]] - A / D) : 0.0;
+          if (grad_w)
+            grad_w[r * n + i] = (D > 0.0) ? A / D : (b.hi - b.lo == 1 ? (double)g[pm[i]] : 0.0);
         }
       }
     }

@@ -60,7 +60,7 @@ def _load() -> ctypes.CDLL:
     lib.tko_dykstra.argtypes = [f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double,
                                 ctypes.c_int, ctypes.c_int, ctypes.c_int, f64p, f64p]
     lib.tko_fwd_w.argtypes = [f32p, f64p, i64, i64, i64, ctypes.c_double, ctypes.c_double, f64p, i32p, f64p, i32p, i32p]
-    lib.tko_vjp_w.argtypes = [f32p, f64p, f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double, f64p]
+    lib.tko_vjp_w.argtypes = [f32p, f64p, f32p, i64, i64, i64, ctypes.c_double, ctypes.c_double, f64p, f64p]
     for fn in (lib.tko_argsort, lib.tko_fwd, lib.tko_vjp, lib.tko_dykstra, lib.tko_fwd_w, lib.tko_vjp_w):
         fn.restype = ctypes.c_int
     _lib = lib
@@ -198,18 +198,21 @@ def fwd_w(theta, w, p: float, lam: float, details: bool = False):
     return out
 
 
-def vjp_w(theta, w, gout, p: float, lam: float) -> np.ndarray:
-    """J^T g of y_R(., w) at theta (gradient in theta only)."""
+def vjp_w(theta, w, gout, p: float, lam: float, with_w: bool = False):
+    """J^T g of y_R(., w) at theta.  with_w=True also returns the cotangent pulled back to w, (rows, n) in
+    w's own order (one row per row of theta, also when w is shared)."""
     x = _f32(theta)
     g = _f32(gout)
     rows, n = x.shape
     ww = _w64(w, rows, n)
     grad = np.empty((rows, n), np.float64)
+    gw = np.empty((rows, n), np.float64) if with_w else None
     rc = _load().tko_vjp_w(_ptr(x, ctypes.c_float), _ptr(ww, ctypes.c_double), _ptr(g, ctypes.c_float), rows, n,
-                           ww.shape[0], p, lam, _ptr(grad, ctypes.c_double))
+                           ww.shape[0], p, lam, _ptr(grad, ctypes.c_double),
+                           _ptr(gw, ctypes.c_double) if with_w else None)
     if rc:
         raise ValueError("tko_vjp_w: invalid argument")
-    return grad
+    return (grad, gw) if with_w else grad
 
 
 def soft_rank(theta, p: float, lam: float) -> np.ndarray:

@@ -706,7 +706,7 @@ def test_general_p_vjp_without_saved_state_recomputes_the_forward_pass(mode):
         assert torch.equal(grad, grad2), (n, mode)
         ref = tko.vjp(x, g, k, p, lam, mode)
         a = grad.cpu().numpy().astype(np.float64)
-        # rows whose block edge is a near-tie are judged by the full harness elsewhere; here the bulk must agree
+        # rows whose block edge is a near-tie are handled by the full harness elsewhere; here the bulk must agree
         err = np.abs(a - ref) / np.maximum(1.0, np.abs(ref))
         assert np.median(err.max(axis=1)) <= 1e-5, (n, mode, err.max())
 

@@ -648,6 +648,43 @@ def test_general_w_vjp_matches_finite_differences(p):
         tko.fwd_w(np.zeros((1, 3), np.float32), [1.0, 2.0, 0.0], 2.0, 1.0)
 
 
+@pytest.mark.parametrize("p", [2.0, P43])
+def test_general_w_cotangent_pulled_back_to_w(p):
+    """The gradient in w (what makes the relaxed sort of Sec. 3 differentiable in its input, which enters as
+    w).  Pins: (1) every point of P(w) has sum y = sum w, so the cotangent g = 1 must pull back to 1 for every
+    w_j; (2) central differences of the forward pass in w (w is a float64 input: small steps that keep it
+    sorted), away from the kinks where the partition changes; (3) a singleton has y_j = w_j."""
+    rng = np.random.default_rng(41)
+    n = 7
+    for lam in (0.5, 2.0):
+        x = (rng.standard_normal((1, n)) * 1.2).astype(np.float32)
+        w = np.array([3.0, 2.6, 2.1, 1.9, 1.0, 0.2, 0.0])
+        _, gw1 = tko.vjp_w(x, w, np.ones((1, n), np.float32), p, lam, with_w=True)
+        assert np.max(np.abs(gw1 - 1.0)) < 1e-12
+        g = rng.standard_normal((1, n)).astype(np.float32)
+        _, gw = tko.vjp_w(x, w, g, p, lam, with_w=True)
+        _, d0 = tko.fwd_w(x, w, p, lam, details=True)
+        h = 1e-6
+        fd = np.empty(n)
+        same = True
+        for j in range(n):
+            wp = w.copy(); wm = w.copy()
+            wp[j] += h; wm[j] -= h
+            yp, dp = tko.fwd_w(x, wp, p, lam, details=True)
+            ym, dm = tko.fwd_w(x, wm, p, lam, details=True)
+            same &= np.array_equal(d0["block_lo"], dp["block_lo"]) and np.array_equal(d0["block_lo"], dm["block_lo"])
+            fd[j] = float(np.dot(g[0].astype(np.float64), (yp[0] - ym[0]))) / (2 * h)
+        if same:
+            assert np.max(np.abs(fd - gw[0])) < 1e-6, (lam, fd, gw)
+    # lambda -> 0: nothing pools, y = w through the permutation, so the pull-back is g in sorted order
+    x = np.array([[0.3, -1.0, 2.0, 0.9]], np.float32)
+    w = np.array([4.0, 3.0, 2.0, 1.0])
+    g = np.array([[1.0, 2.0, 3.0, 4.0]], np.float32)
+    _, gw = tko.vjp_w(x, w, g, p, 1e-3, with_w=True)
+    order = np.argsort(-x[0], kind="stable")
+    assert np.allclose(gw[0], g[0][order], atol=1e-9)
+
+
 # --------------------------------------------------------------------------
 # VJP
 # --------------------------------------------------------------------------
