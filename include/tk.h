@@ -227,12 +227,16 @@ tk_status tk_vjp_cols(const float *theta, const float *grad_out, int64_t n, int6
  * an unsorted w gives an unspecified result).  p = 2 or p = 4/3, n <= 2048 (else
  * TK_ERR_UNSUPPORTED).  opts may carry status_out; the other fields must be unset.
  * tk_vjp_w: grad_theta[r, :] = J(theta[r, :])^T grad_out[r, :], the Jacobian of Prop. 7 (block
- * diagonal over the pooled blocks) in theta, w held fixed; the row is sorted and solved again.  */
+ * diagonal over the pooled blocks) in theta; the row is sorted and solved again.  grad_w (may be
+ * NULL): device [rows*n], the cotangent pulled back to w, per row and in w's own order -- inside a
+ * pooled block B the value solves sum_B rho(s_i - gamma) = sum_B w_i, so every w_j of the block
+ * receives sum_B rho' g / sum_B rho'.  It is what the relaxed sort needs, whose input enters as w;
+ * for a w shared by all rows the caller adds the rows up.                                         */
 tk_status tk_fwd_w(const float *theta, const float *w, int64_t rows, int64_t n, int64_t w_rows, double p,
                    double lambda, float *out, const tk_opts *opts, tk_stream stream);
 tk_status tk_vjp_w(const float *theta, const float *w, const float *grad_out, int64_t rows, int64_t n,
-                   int64_t w_rows, double p, double lambda, float *grad_theta, const tk_opts *opts,
-                   tk_stream stream);
+                   int64_t w_rows, double p, double lambda, float *grad_theta, float *grad_w,
+                   const tk_opts *opts, tk_stream stream);
 
 /* Segmented stable descending argsort (Sec. 3, argsort/sort): per row,
  * perm_out[i] = index of the i-th largest key (theta, or |theta| for

@@ -97,7 +97,7 @@ def load() -> ctypes.CDLL:
     lib.tk_fwd_w.restype = ci
     lib.tk_fwd_w.argtypes = [vp, vp, i64, i64, i64, dbl, dbl, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_vjp_w.restype = ci
-    lib.tk_vjp_w.argtypes = [vp, vp, vp, i64, i64, i64, dbl, dbl, vp, ctypes.POINTER(TkOpts), vp]
+    lib.tk_vjp_w.argtypes = [vp, vp, vp, i64, i64, i64, dbl, dbl, vp, vp, ctypes.POINTER(TkOpts), vp]
     lib.tk_argsort.restype = ci
     lib.tk_argsort.argtypes = [vp, i64, i64, ci, vp, vp, ctypes.POINTER(TkOpts), vp]
     _lib = lib
@@ -253,11 +253,13 @@ def tk_fwd_w(theta, w, rows, n, p, lam, out, *, status_out=None) -> None:
         raise TkError(rc, "tk_fwd_w")
 
 
-def tk_vjp_w(theta, w, grad_out, rows, n, p, lam, grad_theta, *, status_out=None) -> None:
+def tk_vjp_w(theta, w, grad_out, rows, n, p, lam, grad_theta, *, grad_w=None, status_out=None) -> None:
+    """grad_w (optional): [rows, n], the cotangent pulled back to w (per row, in w's order)."""
     w_rows = 1 if w.numel() == n and rows != 1 else (rows if w.numel() >= rows * n else 1)
     o = _opts(status_out=status_out)
     rc = load().tk_vjp_w(_dev(theta, torch.float32, "theta", rows * n), _dev(w, torch.float32, "w", w_rows * n),
                          _dev(grad_out, torch.float32, "grad_out", rows * n), rows, n, w_rows, p, lam,
-                         _dev(grad_theta, torch.float32, "grad_theta", rows * n), ctypes.byref(o), _stream())
+                         _dev(grad_theta, torch.float32, "grad_theta", rows * n),
+                         _dev(grad_w, torch.float32, "grad_w", rows * n), ctypes.byref(o), _stream())
     if rc != TK_OK:
         raise TkError(rc, "tk_vjp_w")

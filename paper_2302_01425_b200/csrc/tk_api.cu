@@ -438,8 +438,8 @@ tk_status tk_vjp_cols(const float* theta, const float* grad_out, int64_t n, int6
 
 // ---- any sorted w: relaxed linear maximisation over the permutahedron P(w)
 static tk_status run_w(const float* theta, const float* w, const float* grad_out, int64_t rows, int64_t n,
-                       int64_t w_rows, double p, double lambda, float* out, const tk_opts* opts, tk_stream stream,
-                       int what) {
+                       int64_t w_rows, double p, double lambda, float* out, float* grad_w, const tk_opts* opts,
+                       tk_stream stream, int what) {
   int q4 = 0;
   double qm1 = 0.0;
   tk_status s = check_common(theta, rows, n, 1, p, lambda, TK_MASK, &q4, &qm1);
@@ -452,6 +452,7 @@ static tk_status run_w(const float* theta, const float* w, const float* grad_out
   fill(P, theta, rows, n, 1, q4, 0.0, lambda, TK_MASK);
   P.out = out;
   P.gout = grad_out;
+  P.sorted_out = grad_w;
   P.what = what;
   if (opts) P.status = opts->status_out;
   cudaError_t e = tk::launch_w(P, w, w_rows, (cudaStream_t)stream);
@@ -460,13 +461,13 @@ static tk_status run_w(const float* theta, const float* w, const float* grad_out
 
 tk_status tk_fwd_w(const float* theta, const float* w, int64_t rows, int64_t n, int64_t w_rows, double p,
                    double lambda, float* out, const tk_opts* opts, tk_stream stream) {
-  return run_w(theta, w, nullptr, rows, n, w_rows, p, lambda, out, opts, stream, tk::W_FWD);
+  return run_w(theta, w, nullptr, rows, n, w_rows, p, lambda, out, nullptr, opts, stream, tk::W_FWD);
 }
 
 tk_status tk_vjp_w(const float* theta, const float* w, const float* grad_out, int64_t rows, int64_t n,
-                   int64_t w_rows, double p, double lambda, float* grad_theta, const tk_opts* opts,
+                   int64_t w_rows, double p, double lambda, float* grad_theta, float* grad_w, const tk_opts* opts,
                    tk_stream stream) {
-  return run_w(theta, w, grad_out, rows, n, w_rows, p, lambda, grad_theta, opts, stream, tk::W_VJP);
+  return run_w(theta, w, grad_out, rows, n, w_rows, p, lambda, grad_theta, grad_w, opts, stream, tk::W_VJP);
 }
 
 tk_status tk_argsort(const float* theta, int64_t rows, int64_t n, int mode, int32_t* perm_out,

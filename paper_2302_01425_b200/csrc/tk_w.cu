@@ -279,7 +279,13 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
       const float a = tt * inv_lam;
       const double dr = Q4 ? 3.0 * (double)a * (double)a * (double)inv_lam : (double)inv_lam;
       const double gs = (double)__ldg(g_row + A.idx[i]);
-      out_s[A.idx[i]] = D > 0.0 ? (float)(dr * (gs - Ab / D)) : 0.0f;
+      // a singleton's own mean is its g (the difference of two prefix sums would return rounding noise there)
+      const double mean = hi - lo == 1 ? gs : (D > 0.0 ? Ab / D : 0.0);
+      out_s[A.idx[i]] = (hi - lo > 1 && D > 0.0) ? (float)(dr * (gs - mean)) : 0.0f;
+      // the cotangent pulled back to w, in w's own order: A_B / D_B for every rank of the block (a
+      // singleton has y = w: its entry is g also where rho' vanishes)
+      if (P.sorted_out && TK_IN_BOUNDS(row * (long long)n + i, 1, P.rows * (long long)n, P.status))
+        P.sorted_out[row * (long long)n + i] = (float)mean;
     }
   }
   __syncthreads();
@@ -293,8 +299,8 @@ __global__ void __launch_bounds__(kWThreads) tk_w_kernel(const Problem P, const 
 
 int w_max_n() { return kWMaxN; }
 
-// Forward pass (P.what == W_FWD) or VJP in theta (W_VJP, cotangent in P.gout) of the relaxed operator
-// over P(w); w: device [w_rows * n], every row non-increasing; w_rows is 1 or P.rows.
+// Forward pass (P.what == W_FWD) or VJP (W_VJP, cotangent in P.gout; in theta, and in w when P.sorted_out
+// is given) of the relaxed operator over P(w); w: device [w_rows * n], every row non-increasing; w_rows is 1 or P.rows.
 cudaError_t launch_w(const Problem& P, const float* w, long long w_rows, cudaStream_t stream) {
   int N = 32;
   while (N < P.n) N <<= 1;

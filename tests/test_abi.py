@@ -120,8 +120,8 @@ def test_general_w_arguments_are_rejected_on_the_host(lib):
     assert fw(4, 8, 1, 1.5, 1.0) == b.TK_ERR_UNSUPPORTED            # p = 2 and p = 4/3 only
     assert fw(4, 4096, 1, 2.0, 1.0) == b.TK_ERR_UNSUPPORTED         # rows of up to 2048 elements
     assert fw(0, 8, 1, 2.0, 1.0) == b.TK_OK
-    assert lib.tk_vjp_w(fake, fake, None, 4, 8, 1, 2.0, 1.0, fake, None, None) == b.TK_ERR_INVALID_ARG
-    assert lib.tk_vjp_w(fake, fake, fake, 0, 8, 1, 2.0, 1.0, fake, None, None) == b.TK_OK
+    assert lib.tk_vjp_w(fake, fake, None, 4, 8, 1, 2.0, 1.0, fake, None, None, None) == b.TK_ERR_INVALID_ARG
+    assert lib.tk_vjp_w(fake, fake, fake, 0, 8, 1, 2.0, 1.0, fake, fake, None, None) == b.TK_OK
 
 
 class FakeDeviceTensor:
@@ -182,6 +182,8 @@ def test_binding_refuses_buffers_shorter_than_the_call_needs(lib, monkeypatch):
         b.tk_fwd_w(ok(32), ok(8), 1, 32, 2.0, 1.0, ok(32))
     with pytest.raises(ValueError, match="grad_theta"):
         b.tk_vjp_w(ok(32), ok(8), ok(32), 4, 8, 2.0, 1.0, ok(31))
+    with pytest.raises(ValueError, match="grad_w"):
+        b.tk_vjp_w(ok(32), ok(8), ok(32), 4, 8, 2.0, 1.0, ok(32), grad_w=ok(31))
     # wrong dtype, host memory and strided views are refused too
     with pytest.raises(ValueError, match="contiguous CUDA tensor"):
         b.tk_fwd(T(32, "float64"), 4, 8, 2, 2.0, 1.0, 0, ok(32))

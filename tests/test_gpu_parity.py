@@ -908,14 +908,21 @@ def test_general_sorted_w_matches_oracle(p):
         g = wl.cotangent_like(x, 77)
         gt = torch.from_numpy(g).cuda()
         grad = torch.full((rows, n), float("nan"), device="cuda")
-        tk.tk_vjp_w(th, wt, gt, rows, n, p, lam, grad)
+        gw = torch.full((rows, n), float("nan"), device="cuda")
+        tk.tk_vjp_w(th, wt, gt, rows, n, p, lam, grad, grad_w=gw)
         torch.cuda.synchronize()
-        gref = tko.vjp_w(x, w64, g, p, lam)
+        gref, gwref = tko.vjp_w(x, w64, g, p, lam, with_w=True)
         ok = stable_elements(x, w64, lam)
         assert ok.mean() >= 0.5, f"{label}: only {ok.mean():.2f} of the elements away from a merge"
         eg = rel(grad.cpu().numpy().astype(np.float64), gref)[ok]
         assert np.isfinite(grad.cpu().numpy()).all()
         assert eg.max() <= TOL, f"{label}: vjp {eg.max()}"
+        # the cotangent pulled back to w is indexed by sorted rank: the same filter, through the oracle's permutation
+        _, det = tko.fwd_w(x, w64, p, lam, details=True)
+        ok_rank = np.take_along_axis(ok, det["perm"].astype(np.int64), axis=1)
+        assert np.isfinite(gw.cpu().numpy()).all()
+        ew = rel(gw.cpu().numpy().astype(np.float64), gwref)[ok_rank]
+        assert ew.max() <= TOL, f"{label}: cotangent in w {ew.max()}"
         return out
 
     for n, rows in ((5, 33), (64, 40), (100, 17), (1000, 9), (2048, 5)):
