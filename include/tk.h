@@ -166,7 +166,10 @@ tk_status tk_fwd_ex(const float *theta, int64_t rows, int64_t n, int64_t k, doub
 
 /* Vector-Jacobian product (Prop. 7 chained through y = grad R*(x - u)):
  * grad_theta[r, :] = J(theta[r, :])^T grad_out[r, :].  All device, [rows*n] fp32.
- * With opts->state_out from a forward call the rows are not sorted again.       */
+ * With opts->state_out from a forward call nothing is solved again.  Without it the
+ * row is solved again: by the sort-free forward pass when opts->workspace has room
+ * for the row state (rows * sizeof(tk_rowstate) bytes, 256-byte aligned; rows of up
+ * to 32768 elements), inside a sorting kernel otherwise.                         */
 tk_status tk_vjp(const float *theta, const float *grad_out, int64_t rows, int64_t n, int64_t k,
                  double p, double lambda, int mode, float *grad_theta, const tk_opts *opts,
                  tk_stream stream);

@@ -278,10 +278,14 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   // otherwise the forward pass runs again here -- its output goes to grad_theta, which the VJP overwrites
   // afterwards, its row state to the caller's workspace
   const tk_rowstate* recomputed = nullptr;
-  if (qm1 > 0.0 && !(opts && opts->state_out) && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG)) {
-    if (!opts || !opts->workspace || (reinterpret_cast<uintptr_t>(opts->workspace) & 255u) ||
-        opts->workspace_bytes < (size_t)rows * sizeof(tk_rowstate))
-      return TK_ERR_WORKSPACE;
+  const bool room_for_state = opts && opts->workspace && !(reinterpret_cast<uintptr_t>(opts->workspace) & 255u) &&
+                              opts->workspace_bytes >= (size_t)rows * sizeof(tk_rowstate);
+  const bool must_recompute = qm1 > 0.0 && (n > tk::kMaxGeneralSortedN || mode == TK_TOPKMAG);
+  // p = 2 and p = 4/3 on rows the threshold form serves: with room for the row state the forward pass that
+  // needs no sort runs again; without it the sorting kernels recompute inside the VJP kernel
+  const bool may_recompute = qm1 == 0.0 && n <= tk::newton_max_n() && room_for_state;
+  if (!(opts && opts->state_out) && (must_recompute || may_recompute)) {
+    if (!room_for_state) return TK_ERR_WORKSPACE;
     tk_opts f = {};
     f.solver = TK_SOLVER_AUTO;
     f.state_out = static_cast<tk_rowstate*>(opts->workspace);
@@ -298,9 +302,9 @@ tk_status tk_vjp(const float* theta, const float* grad_out, int64_t rows, int64_
   if (opts) P.status = opts->status_out;
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(grad_out) && aligned16(grad_theta);
   cudaError_t e;
-  if (n > tk::kMaxOnChipN && n <= tk::kMaxKeyOnlyN && opts && opts->state_out) {
-    // from saved state a row of this length is streamed by one thread block: no scratch
-    P.state_in = opts->state_out;
+  if (n > tk::kMaxOnChipN && n <= tk::kMaxKeyOnlyN && (recomputed || (opts && opts->state_out))) {
+    // from row state (saved, or just recomputed) a row of this length needs no scratch
+    P.state_in = recomputed ? recomputed : opts->state_out;
     e = tk::launch_vjp_state(P, (cudaStream_t)stream);
   } else if (n > tk::kMaxOnChipN) {
     s = check_workspace(opts, rows, n);

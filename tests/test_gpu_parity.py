@@ -711,6 +711,32 @@ def test_general_p_vjp_without_saved_state_recomputes_the_forward_pass(mode):
         assert np.median(err.max(axis=1)) <= 1e-5, (n, mode, err.max())
 
 
+def test_vjp_without_saved_state_uses_the_sort_free_forward_when_given_room():
+    """tk_vjp with no saved row state but a workspace of rows * 16 bytes: the threshold-form forward pass runs
+    again and the VJP is the one from state, bit for bit; without the workspace the sorting kernels recompute,
+    and both agree to rounding."""
+    for n, k, rows, mode, p in ((64, 8, 500, tk.TK_MASK, 2.0), (1000, 5, 40, tk.TK_TOPK, P43),
+                                (4096, 512, 9, tk.TK_TOPKMAG, 2.0), (20000, 300, 3, tk.TK_MASK, P43)):
+        x = rows_of(n, rows, 590 + n)
+        g = wl.cotangent_like(x, 590 + n)
+        th, gt = torch.from_numpy(x).cuda(), torch.from_numpy(g).cuda()
+        ws = torch.empty(((rows * 16 + 255) // 256) * 256, dtype=torch.uint8, device="cuda")
+        fast, ref, slow = (torch.full_like(th, float("nan")) for _ in range(3))
+        tk.tk_vjp(th, gt, rows, n, k, p, 0.7, mode, fast, workspace=ws)
+        st = tk.new_state(rows)
+        out = torch.empty_like(th)
+        tk.tk_fwd_ex(th, rows, n, k, p, 0.7, mode, out, state_out=st)
+        tk.tk_vjp(th, gt, rows, n, k, p, 0.7, mode, ref, state=st)
+        torch.cuda.synchronize()
+        assert torch.equal(fast, ref), (n, mode)
+        if n <= 16384:
+            tk.tk_vjp(th, gt, rows, n, k, p, 0.7, mode, slow)
+            torch.cuda.synchronize()
+            d = ((slow - ref).abs() / ref.abs().clamp(min=1.0))
+            # rows whose block edge is a near-tie may differ between the two solves: the bulk must agree
+            assert float(d.max(dim=1).values.median()) <= 1e-5, (n, mode)
+
+
 def test_general_p_limits():
     th = torch.randn((4, 64), device="cuda")
     out = torch.empty_like(th)
