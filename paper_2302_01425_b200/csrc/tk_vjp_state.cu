@@ -149,10 +149,24 @@ __global__ void __launch_bounds__(256) tk_vjp_long_partial(const Problem P, doub
     const float* x_row = P.theta + row * (long long)n;
     const float* g_row = P.gout + row * (long long)n;
     const int start = tile * kLongTile;
+    if (P.vec4) {                               // n % 4 == 0 and aligned rows: 128-bit loads
+      const float4* x4 = reinterpret_cast<const float4*>(x_row + start);
+      const float4* g4 = reinterpret_cast<const float4*>(g_row + start);
+#pragma unroll
+      for (int j = 0; j < kLongTile / 1024; ++j) {
+        const int v = j * 256 + t;
+        if (start + 4 * v < n) {
+          const float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
+          accumulate_f64(P, M, c, x.x, g.x, A, D); accumulate_f64(P, M, c, x.y, g.y, A, D);
+          accumulate_f64(P, M, c, x.z, g.z, A, D); accumulate_f64(P, M, c, x.w, g.w, A, D);
+        }
+      }
+    } else {
 #pragma unroll 4
-    for (int j = 0; j < kLongTile / 256; ++j) {
-      const int i = start + j * 256 + t;
-      if (i < n) accumulate_f64(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+      for (int j = 0; j < kLongTile / 256; ++j) {
+        const int i = start + j * 256 + t;
+        if (i < n) accumulate_f64(P, M, c, __ldg(x_row + i), __ldg(g_row + i), A, D);
+      }
     }
   }
   A = warp_sum(A); D = warp_sum(D);
@@ -185,6 +199,23 @@ __global__ void __launch_bounds__(256) tk_vjp_long_finish(const Problem P, const
   const float* g_row = P.gout + row * (long long)n;
   float* o_row = P.out + row * (long long)n;
   const int start = tile * kLongTile;
+  if (P.vec4) {
+    const float4* x4 = reinterpret_cast<const float4*>(x_row + start);
+    const float4* g4 = reinterpret_cast<const float4*>(g_row + start);
+    float4* o4 = reinterpret_cast<float4*>(o_row + start);
+#pragma unroll
+    for (int j = 0; j < kLongTile / 1024; ++j) {
+      const int v = j * 256 + t;
+      if (start + 4 * v < n) {
+        const float4 x = __ldg(x4 + v), g = __ldg(g4 + v);
+        float4 o;
+        o.x = finish(P, M, c, x.x, g.x, ratio, delta); o.y = finish(P, M, c, x.y, g.y, ratio, delta);
+        o.z = finish(P, M, c, x.z, g.z, ratio, delta); o.w = finish(P, M, c, x.w, g.w, ratio, delta);
+        o4[v] = o;
+      }
+    }
+    return;
+  }
 #pragma unroll 4
   for (int j = 0; j < kLongTile / 256; ++j) {
     const int i = start + j * 256 + t;
