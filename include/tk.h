@@ -66,7 +66,7 @@ typedef enum {
 
 typedef enum {
   TK_SOLVER_AUTO = 0,     /* the fastest exact path for the request: the threshold form when
-                             only values are asked for (rows of more than 16 elements, up to
+                             only values are asked for (rows of more than 8 elements -- 16 for p = 4/3 --, up to
                              32768; longer rows when there are at most 16 of them), else the
                              sort and TK_SOLVER_PAV                                          */
   TK_SOLVER_PAV = 1,      /* sort, then exact pooling of adjacent violators (Sec. 5, App. B.2) */

@@ -184,8 +184,8 @@ static tk_status fwd_relaxed(const float* theta, int64_t rows, int64_t n, int64_
   P.vec4 = (n % 4 == 0) && aligned16(theta) && aligned16(out);
   // phi(x) = x with a closed-form block solve, nothing but values asked for: the threshold form needs no
   // order at all (TK_SOLVER_PAV keeps the sort)
-  // (rows of up to 16 elements sort faster than they iterate: AUTO keeps the sort there)
-  const bool by_threshold = (solver == TK_SOLVER_THRESHOLD || (solver == TK_SOLVER_AUTO && n > 16)) &&
+  // (very short rows sort faster than they iterate: AUTO keeps the sort up to 8 elements, up to 16 for p = 4/3)
+  const bool by_threshold = (solver == TK_SOLVER_THRESHOLD || (solver == TK_SOLVER_AUTO && n > (q4 ? 16 : 8))) &&
                             qm1 == 0.0 && P.perm_out == nullptr && n <= tk::newton_max_n();
   if (by_threshold) {
     cudaError_t en = tk::launch_newton(P, (cudaStream_t)stream);
