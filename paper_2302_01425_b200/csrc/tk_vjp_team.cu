@@ -258,7 +258,7 @@ cudaError_t launch_vjp_team(const Problem& P, cudaStream_t stream) {
   if (n <= 128) return vt_launch_mode<8, 16, 1>(P, stream);
   if (n <= 256) return vt_launch_mode<16, 16, 1>(P, stream);
   if (n <= 512) return vt_launch_mode<32, 16, 1>(P, stream);
-  if (n <= 1024) return vt_launch_mode<32, 16, 2>(P, stream);
+  if (n <= 1024) return vt_launch_mode<32, 8, 4>(P, stream);
   if (n <= 2048) return vt_launch_mode<32, 16, 4>(P, stream);
   if (n <= 4096) return vt_launch_mode<32, 16, 8>(P, stream);
   if (n <= 8192) return vt_launch_mode<32, 16, 16>(P, stream);
